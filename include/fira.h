@@ -1,0 +1,191 @@
+/*
+ * fira.h -- C ABI of the Fira optimizer update (arXiv 2410.01623) for one NVIDIA
+ * B200 (sm_100a).
+ *
+ * What the library computes.  For every registered weight matrix W (m x n, row
+ * major) and its gradient G, one call of fira_step() performs one pass of the
+ * loop body of the paper's Algorithm 1 ("Fira with Adam", Appendix A.1):
+ *
+ *   R = P^T G,  S = (I - P P^T) G                    (Section 4.1, "Challenge analysis")
+ *   M <- b1 M + (1-b1) R,  V <- b2 V + (1-b2) R^2
+ *   N = sqrt(1-b2^s)/(1-b1^s) * M / (sqrt(V) + eps)   (Eq. 2-4 on R; s = steps taken incl. this one)
+ *   k_i = ||N[:,i]|| / (||R[:,i]|| + eps),  S[:,i] <- k_i S[:,i]      (Eq. 11, Algorithm 1 form)
+ *   S <- S * gamma / max(||S|| / (||S_prev|| + eps), gamma)            (Eq. 12, Algorithm 1 form)
+ *   W <- W - lr * alpha * (P N + S)                                     (Algorithm 1, last two lines)
+ *
+ * Orientation.  For m <= n the projection is a left one, P is m x r and the
+ * factors k are per column of G (n of them).  For m > n the footnote of Section
+ * 3.3 applies: a right projection Q (n x r), R = G Q (m x r); the whole algorithm
+ * is applied to the transposed problem, so the factors are per row of G (m of
+ * them).  Below, d = min(m,n) is the projected extent and l = max(m,n) the other
+ * one; "the projection" is the d x r matrix P or Q.
+ *
+ * Conventions fixed where the paper leaves a choice: the bias-correction exponent
+ * is s = t + 1; the remembered norm ||S_prev|| is the norm after limiting; a
+ * matrix's first step is not limited; gamma = +inf disables the limiter; a
+ * projection switch keeps M, V, ||S_prev|| and t; alpha multiplies both terms
+ * unless FIRA_FLAG_ALPHA_LOWRANK_ONLY is set; no weight decay.
+ *
+ * Memory and ownership.  Every pointer whose name ends in _dev is a device pointer
+ * on the context's GPU; every other pointer is a host pointer.  The caller owns W,
+ * G, the state buffer and the scratch buffer and keeps them alive for the lifetime
+ * of the context; the library allocates no device memory.  The state buffer holds,
+ * per matrix, the projection (d x r, row major, in the matrix's dtype), M and V
+ * (each l x r, row major, float: row i belongs to column i of G when m <= n and to
+ * row i of G when m > n, i.e. the transpose of the paper's r x n layout in the
+ * first case), ||S_prev|| (float) and t (int64): the d r + 2 l r + 1 numbers of the
+ * paper's comparison table plus the step count.  The scratch buffer holds
+ * intermediates and is overwritten by every call.
+ *
+ * Streams and errors.  All device work is enqueued on the stream given to
+ * fira_init() and calls return without waiting for it unless stated otherwise.
+ * Host-side argument errors are returned at once and leave the state untouched.
+ * Device-side conditions (a bounded wait that ran out, a non-finite norm) are
+ * recorded in a status word that fira_poll() reads.  No entry point throws, aborts
+ * or traps.  A context is not thread safe.
+ */
+#ifndef FIRA_H_
+#define FIRA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define FIRA_API __attribute__((visibility("default")))
+#else
+#define FIRA_API
+#endif
+
+typedef enum {
+  FIRA_OK = 0,
+  FIRA_ERR_INVALID_ARG = 1,
+  FIRA_ERR_WORKSPACE_TOO_SMALL = 2,
+  FIRA_ERR_UNSUPPORTED = 3,
+  FIRA_ERR_CUDA = 4,
+  FIRA_ERR_DEVICE_TIMEOUT = 5,
+  FIRA_ERR_NONFINITE = 6
+} fira_status;
+
+typedef enum { FIRA_F32 = 0, FIRA_BF16 = 1 } fira_dtype;
+
+/* fira_hparams.flags */
+#define FIRA_FLAG_ALPHA_LOWRANK_ONLY 1u /* G~ = alpha P N + S instead of alpha (P N + S) */
+#define FIRA_FLAG_AUTO_REFRESH 2u       /* fira_step() refreshes a matrix's projection when t mod T == 0 */
+#define FIRA_FLAG_FORCE_SIMT 4u         /* bf16 matrices also use the fp32 CUDA-core kernels */
+
+/* Inputs of Algorithm 1.  eps > 0; 0 <= beta < 1; gamma >= 1 or +inf; T >= 0 (0: never). */
+typedef struct {
+  float beta1, beta2, eps;
+  float lr;     /* eta; fira_step() can override it per call */
+  float alpha;  /* GaLore scale */
+  float gamma;  /* limiter threshold */
+  int32_t T;    /* projection refresh gap in steps */
+  uint32_t flags;
+} fira_hparams;
+
+/* One weight matrix: m x n, row major with leading dimension ld (elements, >= n;
+ * 0 means n), W and G of type dtype (fira_dtype), rank 1 <= r <= min(m, n). */
+typedef struct {
+  int32_t m, n, r;
+  int32_t dtype;
+  int64_t ld;
+} fira_matrix_desc;
+
+/* Per-matrix numbers of the most recent step. */
+typedef struct {
+  float norm_scaled;  /* ||S|| after the column factors, before the limiter */
+  float lambda;       /* limiter factor applied (1 = not limited) */
+  float norm_prev;    /* ||S_prev|| now stored (norm after limiting); < 0 = unset */
+  float k_min, k_max; /* range of the factors k */
+  int64_t t;          /* steps taken */
+  int32_t engine;     /* 0 = fp32 CUDA-core kernels, 1 = bf16 tensor-core kernels */
+} fira_diag;
+
+typedef struct fira_ctx fira_ctx;
+
+/* Bytes needed for the state and scratch buffers of a matrix list (Algorithm 1's
+ * "Input" line fixes what a matrix is; the state is the paper's comparison-table
+ * count).  Both are rounded up to 256-byte multiples per section. */
+FIRA_API fira_status fira_query_workspace(const fira_hparams* hp, const fira_matrix_desc* descs,
+                                          int32_t count, size_t* state_bytes, size_t* scratch_bytes);
+
+/* Algorithm 1, initialisation: M_0 = V_0 = 0, t = 0, ||S_prev|| unset, projection
+ * zero (set it with fira_set_projection() or fira_refresh_projection() before the
+ * first step).  state_dev and scratch_dev must be 256-byte aligned and at least as
+ * large as fira_query_workspace() reports.  cuda_stream is a cudaStream_t (NULL =
+ * the default stream).  Waits for the stream once the state has been cleared. */
+FIRA_API fira_status fira_init(fira_ctx** out, const fira_hparams* hp, const fira_matrix_desc* descs,
+                               int32_t count, void* state_dev, size_t state_bytes, void* scratch_dev,
+                               size_t scratch_bytes, void* cuda_stream);
+
+/* One pass of Algorithm 1's loop body over every matrix.  W_dev and G_dev are host
+ * arrays of `count` device pointers (16-byte aligned).  W is updated in place, G is
+ * only read.  lr < 0 uses hparams.lr.  With FIRA_FLAG_AUTO_REFRESH the projection of
+ * every matrix whose t is a multiple of T is first recomputed from its G (the
+ * "if t mod T = 0" branch). */
+FIRA_API fira_status fira_step(fira_ctx* ctx, void* const* W_dev, const void* const* G_dev, float lr);
+
+/* The same pass as fira_step() (Algorithm 1's loop body) for callers whose weights
+ * and gradients live in HOST memory: W_host and G_host are host arrays of `count`
+ * host pointers (m x ld elements each; page-locked memory makes the copies
+ * asynchronous).  Every G and W is copied into staging_dev, the step runs there,
+ * and every W is copied back, all on the context's stream.  staging_dev is a
+ * 256-byte aligned device buffer of at least fira_staging_bytes() bytes, owned by
+ * the caller.  The host W buffers hold the result once the stream has been
+ * synchronised. */
+FIRA_API fira_status fira_step_host(fira_ctx* ctx, void* const* W_host, const void* const* G_host,
+                                    float lr, void* staging_dev, size_t staging_bytes);
+FIRA_API size_t fira_staging_bytes(const fira_ctx* ctx);
+
+/* Eq. 7: replace the projection of the selected matrices by an orthonormal basis of
+ * the dominant rank-r left (m <= n) or right (m > n) singular subspace of the given
+ * gradients, found on the device by `iters` rounds of blocked subspace iteration
+ * started from a seeded Gaussian matrix (iters < 0: library default).  which = NULL
+ * selects all matrices; G_dev always has `count` entries (entries of unselected
+ * matrices may be NULL).  M, V, ||S_prev|| and t are kept.  The result spans the
+ * subspace; its columns are not the individual singular vectors.  Waits for the
+ * stream before returning. */
+FIRA_API fira_status fira_refresh_projection(fira_ctx* ctx, const void* const* G_dev,
+                                             const int32_t* which, int32_t nwhich, uint64_t seed,
+                                             int32_t iters);
+
+/* Copy a projection (d x r, row major, the matrix's dtype) from / to device memory
+ * (the P_t of Algorithm 1, given by the caller instead of Eq. 7). */
+FIRA_API fira_status fira_set_projection(fira_ctx* ctx, int32_t idx, const void* P_dev);
+FIRA_API fira_status fira_get_projection(fira_ctx* ctx, int32_t idx, void* P_dev);
+
+/* Checkpointing of Algorithm 1's state: copy M and V (l x r floats each, device
+ * pointers, may be NULL to skip) and the two scalars.  Both wait for the stream. */
+FIRA_API fira_status fira_get_state(fira_ctx* ctx, int32_t idx, float* M_dev, float* V_dev,
+                                    float* norm_prev_host, int64_t* t_host);
+FIRA_API fira_status fira_set_state(fira_ctx* ctx, int32_t idx, const float* M_dev, const float* V_dev,
+                                    float norm_prev, int64_t t);
+
+/* Number of optimizer-state elements held for matrix idx: d r + 2 l r + 1 (the
+ * "Optimizer States" row of the paper's comparison table). */
+FIRA_API int64_t fira_state_elements(const fira_ctx* ctx, int32_t idx);
+
+/* Waits for the stream and copies the diagnostics of matrix idx (the quantities of
+ * Eq. 11 and Eq. 12 of the latest step) to the host. */
+FIRA_API fira_status fira_get_diagnostics(fira_ctx* ctx, int32_t idx, fira_diag* out_host);
+
+/* Reads the device status word (waits for the stream): FIRA_OK, or the first
+ * device-side condition recorded since the last poll, which it clears. */
+FIRA_API fira_status fira_poll(fira_ctx* ctx);
+
+/* Number of kernel launches enqueued by the most recent fira_step() call. */
+FIRA_API int32_t fira_last_step_launches(const fira_ctx* ctx);
+
+FIRA_API const char* fira_status_string(fira_status s);
+/* Text of the most recent error on this thread ("" if none). */
+FIRA_API const char* fira_last_error(void);
+FIRA_API void fira_destroy(fira_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FIRA_H_ */

@@ -1,0 +1,96 @@
+// Shared declarations of the Fira library's translation units: the per-matrix
+// device table and small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/fira.h"
+
+namespace fira {
+
+// Scalars kept per matrix in the state buffer.  prev_norm and t are optimizer
+// state (the "+1" of the paper's comparison table and the step count); the rest
+// are diagnostics of the latest step.
+struct MatScalars {
+  float prev_norm;    // ||S_prev|| after limiting; < 0 means "not set yet"
+  float lambda;       // limiter factor of the latest step
+  float norm_scaled;  // ||S|| before the limiter
+  float k_min, k_max;
+  float pad;
+  long long t;        // steps taken
+};
+static_assert(sizeof(MatScalars) == 32, "MatScalars layout");
+
+// One entry of the device-resident problem table.  l = max(m,n) indexes the
+// unprojected extent, d = min(m,n) the projected one.
+struct MatDev {
+  void* W;
+  const void* G;
+  void* P;            // d x r, row major, dtype
+  float* M;           // l x r
+  float* V;           // l x r
+  MatScalars* sc;
+  float* Rt;          // scratch: l x r fp32 low-rank gradient (transposed layout)
+  float* Xt;          // scratch: l x r fp32, first N then X = a_low N - a_res lambda k R
+  float* kvec;        // scratch: l factors
+  float* part;        // scratch: partial sums of ||S||^2
+  __nv_bfloat16* Nb;  // scratch of the tensor-core path: l x r bf16 N
+  __nv_bfloat16* Rb;  //   "      l x r bf16 R
+  __nv_bfloat16* Xb;  //   "      l x r bf16 X
+  float* colpart;     //   "      per (r-tile, l) partial sums of N^2 and R^2
+  float* gsq;         //   "      per-l sums of G^2
+  long long ld;
+  int m, n, r;
+  int left;           // 1: m <= n (left projection), 0: right projection
+  int bf16;           // storage type of W, G, P
+  int engine;         // 0 CUDA-core fp32, 1 tcgen05 bf16
+  int l, d;
+};
+
+struct Hyper {
+  float beta1, beta2, eps, lr, a_low, a_res, gamma;
+};
+
+enum DeviceStatusBits : unsigned {
+  DEV_STATUS_TIMEOUT = 1u,
+  DEV_STATUS_NONFINITE = 2u,
+};
+
+template <typename T>
+__device__ __forceinline__ float to_float(T v);
+template <>
+__device__ __forceinline__ float to_float<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) {
+  return __bfloat162float(v);
+}
+template <typename T>
+__device__ __forceinline__ T from_float(float v);
+template <>
+__device__ __forceinline__ float from_float<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float v) {
+  return __float2bfloat16_rn(v);
+}
+
+// Index of the matrix whose tile range contains `tile`: the largest i with
+// start[i] <= tile (start has count + 1 ascending entries).
+__device__ __forceinline__ int find_matrix(const int* __restrict__ start, int count, int tile) {
+  int lo = 0, hi = count;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (start[mid] <= tile) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+void set_error(const std::string& msg);
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+}  // namespace fira

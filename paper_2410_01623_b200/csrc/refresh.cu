@@ -1,0 +1,401 @@
+// Projection refresh (Eq. 7): an orthonormal basis of the dominant rank-r singular
+// subspace of G, by blocked subspace iteration on the device.
+//
+// With A = G seen as a d x l matrix (d = projected extent):
+//   Z <- Gaussian (l x r);  Y <- orth(A Z)
+//   repeat `iters` times:   Z <- orth(A^T Y);  Y <- orth(A Z)
+//   projection <- Y  (d x r)
+// orth() is CholeskyQR applied twice: C = Y^T Y, C = L L^T, Y <- Y L^-T.  It
+// changes the basis, never the spanned subspace, so a small diagonal shift in the
+// first pass (which keeps the factorisation defined for ill-conditioned Y) costs
+// no accuracy of the subspace.  The paper calls a library SVD here; the iteration
+// converges to the same subspace at the rate (sigma_{r+1}/sigma_r)^2 per round.
+//
+// Random numbers: Philox4x32-10 (Salmon et al., "Parallel random numbers: as easy
+// as 1, 2, 3", SC'11), keyed by the caller's seed, turned into normals by the
+// Box-Muller transform.
+#include <algorithm>
+
+#include "context.cuh"
+#include "simt_gemm.cuh"
+
+namespace fira {
+
+namespace {
+
+struct RefreshMat {
+  const void* G;
+  void* P;
+  float* Y;   // d x r
+  float* Z;   // l x r
+  float* C;   // r x r
+  long long ld;
+  int d, l, r;
+  int left, bf16;
+  unsigned long long key;
+};
+
+struct GemmDesc {
+  const void* A; long long sAi, sAk; int a_bf16;
+  const float* B; long long sBk, sBj;
+  float* C; long long sCi;
+  int I, J, K;
+};
+
+// ------------------------------------------------------------------ Philox4x32-10
+__device__ __forceinline__ void philox4x32_10(unsigned c0, unsigned c1, unsigned c2, unsigned c3,
+                                              unsigned k0, unsigned k1, unsigned (&out)[4]) {
+  const unsigned M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const unsigned hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+    const unsigned hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+    const unsigned n0 = hi1 ^ c1 ^ k0, n1 = lo1, n2 = hi0 ^ c3 ^ k1, n3 = lo0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += W0; k1 += W1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+__global__ void __launch_bounds__(256)
+k_gauss(const RefreshMat* __restrict__ rm) {
+  const RefreshMat m = rm[blockIdx.y];
+  const long long total = (long long)m.l * m.r;
+  const long long quads = (total + 3) / 4;
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < quads;
+       q += (long long)gridDim.x * blockDim.x) {
+    unsigned o[4];
+    philox4x32_10((unsigned)q, (unsigned)(q >> 32), 0u, 0u, (unsigned)m.key, (unsigned)(m.key >> 32), o);
+    // two Box-Muller pairs; the radius uniforms lie in (0, 1]
+    const float u0 = ((float)(o[0] >> 8) + 1.0f) * (1.0f / 16777216.0f);
+    const float u1 = (float)(o[1] >> 8) * (1.0f / 16777216.0f);
+    const float u2 = ((float)(o[2] >> 8) + 1.0f) * (1.0f / 16777216.0f);
+    const float u3 = (float)(o[3] >> 8) * (1.0f / 16777216.0f);
+    const float ra = sqrtf(-2.0f * logf(u0)), rb = sqrtf(-2.0f * logf(u2));
+    float s0, c0, s1, c1;
+    sincospif(2.0f * u1, &s0, &c0);
+    sincospif(2.0f * u3, &s1, &c1);
+    const float v[4] = {ra * c0, ra * s0, rb * c1, rb * s1};
+    for (int e = 0; e < 4; ++e) {
+      const long long idx = q * 4 + e;
+      if (idx < total) m.Z[idx] = v[e];
+    }
+  }
+}
+
+// ------------------------------------------------------------------ grouped product
+__global__ void __launch_bounds__(GEMM_THREADS)
+k_rgemm(const GemmDesc* __restrict__ descs, int ndesc, const int* __restrict__ tile_start) {
+  __shared__ __align__(16) float As[TK][TM + 4];
+  __shared__ __align__(16) float Bs[TK][TN + 4];
+  const int p = find_matrix(tile_start, ndesc, blockIdx.x);
+  const GemmDesc g = descs[p];
+  const int tile = blockIdx.x - tile_start[p];
+  const int jt = (g.J + TN - 1) / TN;
+  const int i0 = (tile / jt) * TM, j0 = (tile % jt) * TN;
+  float acc[4][4] = {};
+  if (g.a_bf16)
+    gemm_tile<__nv_bfloat16, float>((const __nv_bfloat16*)g.A, g.sAi, g.sAk, g.B, g.sBk, g.sBj,
+                                    g.I, g.J, g.K, i0, j0, acc, As, Bs);
+  else
+    gemm_tile<float, float>((const float*)g.A, g.sAi, g.sAk, g.B, g.sBk, g.sBj, g.I, g.J, g.K,
+                            i0, j0, acc, As, Bs);
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+#pragma unroll
+  for (int x = 0; x < 4; ++x) {
+    const int i = i0 + ty * 4 + x;
+    if (i >= g.I) continue;
+#pragma unroll
+    for (int y = 0; y < 4; ++y) {
+      const int j = j0 + tx * 4 + y;
+      if (j < g.J) g.C[(long long)i * g.sCi + j] = acc[x][y];
+    }
+  }
+}
+
+// ------------------------------------------------------------------ Cholesky
+// One block per matrix: C (r x r, symmetric, row major) -> lower factor L in
+// place (the strict upper triangle is left as it was).  Left-looking over 64-wide
+// block columns.  shift_rel * trace(C)/r is added to the diagonal first.  A
+// non-positive or non-finite pivot is replaced and flagged.
+constexpr int CB = 64;
+
+__global__ void __launch_bounds__(GEMM_THREADS)
+k_cholesky(const RefreshMat* __restrict__ rm, float shift_rel, unsigned* __restrict__ status) {
+  __shared__ __align__(16) float As[TK][TM + 4];
+  __shared__ __align__(16) float Bs[TK][TN + 4];
+  __shared__ float D[CB][CB + 1];
+  __shared__ float red[GEMM_THREADS];
+  const RefreshMat m = rm[blockIdx.x];
+  const int r = m.r;
+  float* C = m.C;
+  const int tid = threadIdx.x;
+  float tr = 0.f;
+  for (int i = tid; i < r; i += GEMM_THREADS) tr += C[(long long)i * r + i];
+  red[tid] = tr;
+  __syncthreads();
+  for (int o = GEMM_THREADS / 2; o > 0; o >>= 1) {
+    if (tid < o) red[tid] += red[tid + o];
+    __syncthreads();
+  }
+  const float mean_diag = red[0] / (float)r;
+  const float shift = shift_rel * mean_diag;
+  const float floor_pivot = fmaxf(1e-30f, 1e-12f * mean_diag);
+  __syncthreads();
+  for (int i = tid; i < r; i += GEMM_THREADS) C[(long long)i * r + i] += shift;
+  __syncthreads();
+
+  const int tx = tid & 15, ty = tid >> 4;
+  for (int J0 = 0; J0 < r; J0 += CB) {
+    const int jb = min(CB, r - J0);
+    // (a) C[I, J] -= L[I, :J0] L[J, :J0]^T for every row tile I >= J
+    for (int I0 = J0; I0 < r; I0 += TM) {
+      float acc[4][4] = {};
+      gemm_tile<float, float>(C, r, 1, C, 1, r, r, J0 + jb, J0, I0, J0, acc, As, Bs);
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        const int i = I0 + ty * 4 + x;
+        if (i >= r) continue;
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+          const int j = J0 + tx * 4 + y;
+          if (j < J0 + jb) C[(long long)i * r + j] -= acc[x][y];
+        }
+      }
+    }
+    __syncthreads();
+    // (b) factor the diagonal block in shared memory
+    for (int e = tid; e < CB * CB; e += GEMM_THREADS) {
+      const int i = e / CB, j = e % CB;
+      D[i][j] = (i < jb && j < jb) ? C[(long long)(J0 + i) * r + J0 + j] : (i == j ? 1.f : 0.f);
+    }
+    __syncthreads();
+    for (int k = 0; k < jb; ++k) {
+      if (tid == 0) {
+        float pv = D[k][k];
+        if (!(pv > floor_pivot) || !isfinite(pv)) { pv = floor_pivot; atomicOr(status, DEV_STATUS_NONFINITE); }
+        D[k][k] = sqrtf(pv);
+      }
+      __syncthreads();
+      const float dk = D[k][k];
+      if (tid > k && tid < jb) D[tid][k] /= dk;
+      __syncthreads();
+      const int rem = jb - k - 1;
+      for (int e = tid; e < rem * rem; e += GEMM_THREADS) {
+        const int i = k + 1 + e / rem, j = k + 1 + e % rem;
+        if (j <= i) D[i][j] -= D[i][k] * D[j][k];
+      }
+      __syncthreads();
+    }
+    for (int e = tid; e < jb * jb; e += GEMM_THREADS) {
+      const int i = e / jb, j = e % jb;
+      if (j <= i) C[(long long)(J0 + i) * r + J0 + j] = D[i][j];
+    }
+    // (c) rows below: L[i, J] = C[i, J] L_JJ^-T, one thread per row
+    for (int i = J0 + jb + tid; i < r; i += GEMM_THREADS) {
+      float* row = C + (long long)i * r + J0;
+      for (int c = 0; c < jb; ++c) {
+        float v = row[c];
+        for (int k = 0; k < c; ++k) v -= row[k] * D[c][k];
+        row[c] = v / D[c][c];
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------ X <- X L^-T
+// One block per tile of 64 rows of X (rows x r, in place).  For each 64-wide
+// block column J: X_J = (X_J - X_{<J} L[J, <J]^T) L_JJ^-T.
+struct TrsmDesc { float* X; const float* L; int rows, r; };
+
+__global__ void __launch_bounds__(GEMM_THREADS)
+k_trsm_rows(const TrsmDesc* __restrict__ descs, int ndesc, const int* __restrict__ tile_start) {
+  __shared__ __align__(16) float As[TK][TM + 4];
+  __shared__ __align__(16) float Bs[TK][TN + 4];
+  __shared__ float T[TM][CB + 1];
+  __shared__ float D[CB][CB + 1];
+  const int p = find_matrix(tile_start, ndesc, blockIdx.x);
+  const TrsmDesc t = descs[p];
+  const int I0 = (blockIdx.x - tile_start[p]) * TM;
+  const int r = t.r;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  for (int J0 = 0; J0 < r; J0 += CB) {
+    const int jb = min(CB, r - J0);
+    float acc[4][4] = {};
+    gemm_tile<float, float>(t.X, r, 1, t.L, 1, r, t.rows, J0 + jb, J0, I0, J0, acc, As, Bs);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const int il = ty * 4 + x;
+#pragma unroll
+      for (int y = 0; y < 4; ++y) {
+        const int jl = tx * 4 + y;
+        float v = 0.f;
+        if (I0 + il < t.rows && jl < jb) v = t.X[(long long)(I0 + il) * r + J0 + jl] - acc[x][y];
+        T[il][jl] = v;
+      }
+    }
+    for (int e = tid; e < CB * CB; e += GEMM_THREADS) {
+      const int i = e / CB, j = e % CB;
+      D[i][j] = (i < jb && j < jb) ? t.L[(long long)(J0 + i) * r + J0 + j] : (i == j ? 1.f : 0.f);
+    }
+    __syncthreads();
+    if (tid < TM && I0 + tid < t.rows) {
+      float* row = T[tid];
+      for (int c = 0; c < jb; ++c) {
+        float v = row[c];
+        for (int k = 0; k < c; ++k) v -= row[k] * D[c][k];
+        v /= D[c][c];
+        row[c] = v;
+        t.X[(long long)(I0 + tid) * r + J0 + c] = v;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(256)
+k_store_projection(const RefreshMat* __restrict__ rm) {
+  const RefreshMat m = rm[blockIdx.y];
+  const long long total = (long long)m.d * m.r;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    if (m.bf16) ((__nv_bfloat16*)m.P)[i] = __float2bfloat16_rn(m.Y[i]);
+    else ((float*)m.P)[i] = m.Y[i];
+  }
+}
+
+// descriptor tables of a chunk: per-matrix entries plus alignment slack
+constexpr size_t TABLE_PER_MATRIX = 1024;
+constexpr size_t TABLE_SLACK = 16 * 1024;
+static_assert(sizeof(RefreshMat) + 4 * sizeof(GemmDesc) + 2 * sizeof(TrsmDesc) + 8 * sizeof(int) <= TABLE_PER_MATRIX, "table allowance");
+
+}  // namespace
+
+static size_t refresh_data_bytes(const fira_matrix_desc& d) {
+  const size_t dd = std::min(d.m, d.n), ll = std::max(d.m, d.n), r = d.r;
+  return align_up(dd * r * 4) + align_up(ll * r * 4) + align_up(r * r * 4);
+}
+
+size_t refresh_bytes_per_matrix(const fira_matrix_desc& d) {
+  return refresh_data_bytes(d) + TABLE_PER_MATRIX + TABLE_SLACK;
+}
+
+#define RF_CUDA(call)                                                          \
+  do {                                                                         \
+    cudaError_t e_ = (call);                                                   \
+    if (e_ != cudaSuccess) {                                                   \
+      set_error(std::string(#call) + ": " + cudaGetErrorString(e_));           \
+      return FIRA_ERR_CUDA;                                                    \
+    }                                                                          \
+  } while (0)
+
+// Refreshes the matrices of `which` in chunks that fit the work area.  The work
+// area is shared with the step's scratch, whose contents are dead between steps.
+fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vector<int>& which,
+                         uint64_t seed, int iters) {
+  if (iters < 0) iters = 4;
+  cudaStream_t st = c->stream;
+  size_t pos = 0;
+  while (pos < which.size()) {
+    // ---- carve a chunk: as many matrices as fit (data regions first, then tables)
+    std::vector<size_t> offs;
+    size_t off = 0, q = pos;
+    for (; q < which.size(); ++q) {
+      const size_t data = refresh_data_bytes(c->descs[which[q]]);
+      if (off + data + (q - pos + 1) * TABLE_PER_MATRIX + TABLE_SLACK > c->work_bytes) break;
+      offs.push_back(off);
+      off += data;
+    }
+    if (q == pos) { set_error("scratch buffer too small for the projection refresh"); return FIRA_ERR_WORKSPACE_TOO_SMALL; }
+    const int nm = (int)(q - pos);
+    std::vector<RefreshMat> rms;
+    size_t data_end = 0;
+    for (int a = 0; a < nm; ++a) {
+      const int idx = which[pos + a];
+      const MatDev& mt = c->mats[idx];
+      RefreshMat rm;
+      rm.G = G_dev[idx]; rm.P = mt.P;
+      char* base = c->work_base + offs[a];
+      rm.Y = (float*)base; base += align_up((size_t)mt.d * mt.r * 4);
+      rm.Z = (float*)base; base += align_up((size_t)mt.l * mt.r * 4);
+      rm.C = (float*)base; base += align_up((size_t)mt.r * mt.r * 4);
+      data_end = std::max(data_end, (size_t)(base - c->work_base));
+      rm.ld = mt.ld; rm.d = mt.d; rm.l = mt.l; rm.r = mt.r; rm.left = mt.left; rm.bf16 = mt.bf16;
+      rm.key = seed * 0x9E3779B97F4A7C15ull + (unsigned long long)idx * 0xD1B54A32D192ED03ull + 1ull;
+      rms.push_back(rm);
+    }
+    // ---- descriptor tables: AZ->Y, A^T Y->Z, Y^T Y->C, Z^T Z->C, trsm(Y), trsm(Z)
+    std::vector<GemmDesc> gAZ, gAtY, gYY, gZZ;
+    std::vector<TrsmDesc> tY, tZ;
+    std::vector<int> sAZ{0}, sAtY{0}, sYY{0}, sTY{0}, sTZ{0};
+    auto tiles = [](int I, int J) { return ((I + TM - 1) / TM) * ((J + TN - 1) / TN); };
+    for (const RefreshMat& m : rms) {
+      GemmDesc g;
+      // Y[d][j] = sum_l A(d,l) Z[l][j]
+      g.A = m.G; g.a_bf16 = m.bf16;
+      g.sAi = m.left ? m.ld : 1; g.sAk = m.left ? 1 : m.ld;
+      g.B = m.Z; g.sBk = m.r; g.sBj = 1; g.C = m.Y; g.sCi = m.r; g.I = m.d; g.J = m.r; g.K = m.l;
+      gAZ.push_back(g); sAZ.push_back(sAZ.back() + tiles(g.I, g.J));
+      // Z[l][j] = sum_d A(d,l) Y[d][j]
+      g.sAi = m.left ? 1 : m.ld; g.sAk = m.left ? m.ld : 1;
+      g.B = m.Y; g.C = m.Z; g.I = m.l; g.K = m.d;
+      gAtY.push_back(g); sAtY.push_back(sAtY.back() + tiles(g.I, g.J));
+      // C = Y^T Y and C = Z^T Z
+      g.a_bf16 = 0; g.sAi = 1; g.sAk = m.r; g.sBk = m.r; g.sBj = 1; g.C = m.C; g.sCi = m.r; g.I = m.r; g.J = m.r;
+      g.A = m.Y; g.B = m.Y; g.K = m.d; gYY.push_back(g);
+      g.A = m.Z; g.B = m.Z; g.K = m.l; gZZ.push_back(g);
+      sYY.push_back(sYY.back() + tiles(m.r, m.r));
+      tY.push_back(TrsmDesc{m.Y, m.C, m.d, m.r}); sTY.push_back(sTY.back() + (m.d + TM - 1) / TM);
+      tZ.push_back(TrsmDesc{m.Z, m.C, m.l, m.r}); sTZ.push_back(sTZ.back() + (m.l + TM - 1) / TM);
+    }
+    char* tp = c->work_base + align_up(data_end);
+    cudaError_t cerr = cudaSuccess;
+    auto put = [&](const void* src, size_t bytes) -> char* {
+      char* dst = tp;
+      if ((size_t)(tp + align_up(bytes) - c->work_base) > c->work_bytes) { cerr = cudaErrorInvalidValue; return dst; }
+      cudaError_t e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st);
+      if (e != cudaSuccess) cerr = e;
+      tp += align_up(bytes);
+      return dst;
+    };
+    const RefreshMat* rm_dev = (const RefreshMat*)put(rms.data(), rms.size() * sizeof(RefreshMat));
+    const GemmDesc* dAZ = (const GemmDesc*)put(gAZ.data(), gAZ.size() * sizeof(GemmDesc));
+    const GemmDesc* dAtY = (const GemmDesc*)put(gAtY.data(), gAtY.size() * sizeof(GemmDesc));
+    const GemmDesc* dYY = (const GemmDesc*)put(gYY.data(), gYY.size() * sizeof(GemmDesc));
+    const GemmDesc* dZZ = (const GemmDesc*)put(gZZ.data(), gZZ.size() * sizeof(GemmDesc));
+    const TrsmDesc* dTY = (const TrsmDesc*)put(tY.data(), tY.size() * sizeof(TrsmDesc));
+    const TrsmDesc* dTZ = (const TrsmDesc*)put(tZ.data(), tZ.size() * sizeof(TrsmDesc));
+    const int* dsAZ = (const int*)put(sAZ.data(), sAZ.size() * sizeof(int));
+    const int* dsAtY = (const int*)put(sAtY.data(), sAtY.size() * sizeof(int));
+    const int* dsYY = (const int*)put(sYY.data(), sYY.size() * sizeof(int));
+    const int* dsTY = (const int*)put(sTY.data(), sTY.size() * sizeof(int));
+    const int* dsTZ = (const int*)put(sTZ.data(), sTZ.size() * sizeof(int));
+    if (cerr != cudaSuccess) { set_error(std::string("refresh tables: ") + cudaGetErrorString(cerr)); return FIRA_ERR_CUDA; }
+
+    auto orth = [&](const GemmDesc* gram, const TrsmDesc* tr, const int* tr_start, int tr_tiles) {
+      for (int pass = 0; pass < 2; ++pass) {
+        k_rgemm<<<sYY.back(), GEMM_THREADS, 0, st>>>(gram, nm, dsYY);
+        k_cholesky<<<nm, GEMM_THREADS, 0, st>>>(rm_dev, pass == 0 ? 1e-6f : 0.f, c->status_dev);
+        k_trsm_rows<<<tr_tiles, GEMM_THREADS, 0, st>>>(tr, nm, tr_start);
+      }
+    };
+    k_gauss<<<dim3(296, nm), 256, 0, st>>>(rm_dev);
+    k_rgemm<<<sAZ.back(), GEMM_THREADS, 0, st>>>(dAZ, nm, dsAZ);
+    orth(dYY, dTY, dsTY, sTY.back());
+    for (int it = 0; it < iters; ++it) {
+      k_rgemm<<<sAtY.back(), GEMM_THREADS, 0, st>>>(dAtY, nm, dsAtY);
+      orth(dZZ, dTZ, dsTZ, sTZ.back());
+      k_rgemm<<<sAZ.back(), GEMM_THREADS, 0, st>>>(dAZ, nm, dsAZ);
+      orth(dYY, dTY, dsTY, sTY.back());
+    }
+    k_store_projection<<<dim3(296, nm), 256, 0, st>>>(rm_dev);
+    RF_CUDA(cudaGetLastError());
+    // the next chunk reuses the work area, and the host tables above die here
+    RF_CUDA(cudaStreamSynchronize(st));
+    pos = q;
+  }
+  return FIRA_OK;
+}
+
+}  // namespace fira

@@ -1,0 +1,243 @@
+// fp32 CUDA-core kernels of the Fira step (Algorithm 1's loop body), grouped over
+// a list of matrices: one launch per phase covers every matrix of the list.
+//
+// Phases (l = unprojected index, d = projected index, Pi = the d x r projection):
+//   1. project      Rt[l][j]   = sum_d G(d,l) Pi[d][j]                      (R = P^T G)
+//   2. adam_rows    M,V update, N, k_l = ||N_l|| / (||R_l|| + eps)           (Eq. 2-4, Eq. 11)
+//   3. back_project mode NORM:   part = sum (k_l (G - Pi R))^2               (||S||, literal residual)
+//   4. finalize     lambda, ||S_prev||, t                                    (Eq. 12)
+//   5. form_x       Xt = a_low N - a_res lambda k_l R
+//   6. back_project mode UPDATE: W -= lr (Pi X + a_res lambda k_l G)
+// Phase 6 uses the identity alpha (P N + lambda (G - P R) diag k) =
+// P (alpha N - alpha lambda R diag k) + alpha lambda G diag k, so that the update
+// needs one product instead of two.
+#include "common.cuh"
+#include "simt_gemm.cuh"
+#include "step_simt.cuh"
+
+namespace fira {
+
+namespace {
+
+// ---------------------------------------------------------------- phase 1
+template <typename T>
+__device__ __forceinline__ void project_tile(const MatDev& mt, int tile, float (*As)[TM + 4],
+                                             float (*Bs)[TN + 4]) {
+  const int rt = (mt.r + TN - 1) / TN;
+  const int i0 = (tile / rt) * TM, j0 = (tile % rt) * TN;
+  float acc[4][4] = {};
+  const T* G = static_cast<const T*>(mt.G);
+  const T* P = static_cast<const T*>(mt.P);
+  // A(i = l, k = d): G[d][l] when left, G[l][d] when right.
+  const long long sAi = mt.left ? 1 : mt.ld, sAk = mt.left ? mt.ld : 1;
+  gemm_tile<T, T>(G, sAi, sAk, P, mt.r, 1, mt.l, mt.r, mt.d, i0, j0, acc, As, Bs);
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+#pragma unroll
+  for (int x = 0; x < 4; ++x) {
+    const int i = i0 + ty * 4 + x;
+    if (i >= mt.l) continue;
+#pragma unroll
+    for (int y = 0; y < 4; ++y) {
+      const int j = j0 + tx * 4 + y;
+      if (j < mt.r) mt.Rt[(long long)i * mt.r + j] = acc[x][y];
+    }
+  }
+}
+
+__global__ void __launch_bounds__(GEMM_THREADS)
+k_project(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+          const int* __restrict__ tile_start) {
+  __shared__ __align__(16) float As[TK][TM + 4];
+  __shared__ __align__(16) float Bs[TK][TN + 4];
+  const int p = find_matrix(tile_start, nlist, blockIdx.x);
+  const MatDev mt = mats[list[p]];
+  const int tile = blockIdx.x - tile_start[p];
+  if (mt.bf16) project_tile<__nv_bfloat16>(mt, tile, As, Bs);
+  else project_tile<float>(mt, tile, As, Bs);
+}
+
+// ---------------------------------------------------------------- phase 2
+// One warp per unprojected index l.  N goes to Xt.
+__global__ void __launch_bounds__(256)
+k_adam_rows(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+            const int* __restrict__ row_start, int rows_total, Hyper hp) {
+  const int warps_per_block = blockDim.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  if (row >= rows_total) return;
+  const int p = find_matrix(row_start, nlist, row);
+  const MatDev mt = mats[list[p]];
+  const int l = row - row_start[p];
+  // bias correction sqrt(1 - b2^s) / (1 - b1^s), s = t + 1, in double
+  const double s = (double)(mt.sc->t + 1);
+  const float bias = (float)(sqrt(1.0 - pow((double)hp.beta2, s)) / (1.0 - pow((double)hp.beta1, s)));
+  const long long base = (long long)l * mt.r;
+  float nn = 0.f, rn = 0.f;
+  for (int j = lane; j < mt.r; j += 32) {
+    const float rv = mt.Rt[base + j];
+    const float mv = hp.beta1 * mt.M[base + j] + (1.f - hp.beta1) * rv;
+    const float vv = hp.beta2 * mt.V[base + j] + (1.f - hp.beta2) * rv * rv;
+    mt.M[base + j] = mv;
+    mt.V[base + j] = vv;
+    const float nv = bias * mv / (sqrtf(vv) + hp.eps);
+    mt.Xt[base + j] = nv;
+    nn = fmaf(nv, nv, nn);
+    rn = fmaf(rv, rv, rn);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    nn += __shfl_xor_sync(0xffffffffu, nn, o);
+    rn += __shfl_xor_sync(0xffffffffu, rn, o);
+  }
+  if (lane == 0) mt.kvec[l] = sqrtf(nn) / (sqrtf(rn) + hp.eps);
+}
+
+// ---------------------------------------------------------------- phases 3 and 6
+enum { MODE_NORM = 0, MODE_UPDATE = 1 };
+
+template <typename T, int MODE>
+__device__ __forceinline__ void back_tile(const MatDev& mt, int tile, float lr, float a_res,
+                                          float (*As)[TM + 4], float (*Bs)[TN + 4], float* red) {
+  const int ct = (mt.n + TN - 1) / TN;
+  const int i0 = (tile / ct) * TM, j0 = (tile % ct) * TN;
+  float acc[4][4] = {};
+  const T* P = static_cast<const T*>(mt.P);
+  const float* X = (MODE == MODE_NORM) ? mt.Rt : mt.Xt;
+  const long long r = mt.r;
+  if (mt.left) {
+    // D[d][l] = sum_j Pi[d][j] X[l][j]
+    gemm_tile<T, float>(P, r, 1, X, 1, r, mt.m, mt.n, mt.r, i0, j0, acc, As, Bs);
+  } else {
+    // D[l][d] = sum_j X[l][j] Pi[d][j]
+    gemm_tile<float, T>(X, r, 1, P, 1, r, mt.m, mt.n, mt.r, i0, j0, acc, As, Bs);
+  }
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const T* G = static_cast<const T*>(mt.G);
+  T* W = static_cast<T*>(mt.W);
+  const float lam = (MODE == MODE_UPDATE) ? mt.sc->lambda : 1.f;
+  float ss = 0.f;
+#pragma unroll
+  for (int x = 0; x < 4; ++x) {
+    const int i = i0 + ty * 4 + x;
+    if (i >= mt.m) continue;
+#pragma unroll
+    for (int y = 0; y < 4; ++y) {
+      const int j = j0 + tx * 4 + y;
+      if (j >= mt.n) continue;
+      const float kf = mt.kvec[mt.left ? j : i];
+      const long long off = (long long)i * mt.ld + j;
+      const float g = to_float<T>(G[off]);
+      if (MODE == MODE_NORM) {
+        const float sv = kf * (g - acc[x][y]);
+        ss = fmaf(sv, sv, ss);
+      } else {
+        const float w = to_float<T>(W[off]);
+        W[off] = from_float<T>(w - lr * (acc[x][y] + a_res * lam * kf * g));
+      }
+    }
+  }
+  if (MODE == MODE_NORM) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float tot = 0.f;
+      for (int w = 0; w < GEMM_THREADS / 32; ++w) tot += red[w];
+      mt.part[tile] = tot;
+    }
+  }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(GEMM_THREADS)
+k_back_project(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+               const int* __restrict__ tile_start, float lr, float a_res) {
+  __shared__ __align__(16) float As[TK][TM + 4];
+  __shared__ __align__(16) float Bs[TK][TN + 4];
+  __shared__ float red[GEMM_THREADS / 32];
+  const int p = find_matrix(tile_start, nlist, blockIdx.x);
+  const MatDev mt = mats[list[p]];
+  const int tile = blockIdx.x - tile_start[p];
+  if (mt.bf16) back_tile<__nv_bfloat16, MODE>(mt, tile, lr, a_res, As, Bs, red);
+  else back_tile<float, MODE>(mt, tile, lr, a_res, As, Bs, red);
+}
+
+// ---------------------------------------------------------------- phase 5
+__global__ void __launch_bounds__(256)
+k_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+         const int* __restrict__ row_start, int rows_total, float a_low, float a_res) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows_total) return;
+  const int p = find_matrix(row_start, nlist, row);
+  const MatDev mt = mats[list[p]];
+  const int l = row - row_start[p];
+  const float c = a_res * mt.sc->lambda * mt.kvec[l];
+  const long long base = (long long)l * mt.r;
+  for (int j = lane; j < mt.r; j += 32) mt.Xt[base + j] = a_low * mt.Xt[base + j] - c * mt.Rt[base + j];
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------- phase 4
+__global__ void __launch_bounds__(256)
+k_finalize(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+           const int* __restrict__ npart_of, Hyper hp, unsigned* __restrict__ status) {
+  __shared__ double sred[256];
+  __shared__ float smin[256], smax[256];
+  const MatDev mt = mats[list[blockIdx.x]];
+  const int npart = npart_of[blockIdx.x];
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < npart; i += 256) acc += (double)mt.part[i];
+  float kmin = INFINITY, kmax = -INFINITY;
+  for (int i = threadIdx.x; i < mt.l; i += 256) {
+    const float kv = mt.kvec[i];
+    kmin = fminf(kmin, kv);
+    kmax = fmaxf(kmax, kv);
+  }
+  sred[threadIdx.x] = acc; smin[threadIdx.x] = kmin; smax[threadIdx.x] = kmax;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) {
+      sred[threadIdx.x] += sred[threadIdx.x + o];
+      smin[threadIdx.x] = fminf(smin[threadIdx.x], smin[threadIdx.x + o]);
+      smax[threadIdx.x] = fmaxf(smax[threadIdx.x], smax[threadIdx.x + o]);
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const double tot = sred[0] > 0.0 ? sred[0] : 0.0;
+    const float norm = (float)sqrt(tot);
+    const float prev = mt.sc->prev_norm;
+    float lam = 1.f;
+    if (prev >= 0.f && !isinf(hp.gamma)) {
+      const float ratio = norm / (prev + hp.eps);
+      lam = hp.gamma / fmaxf(ratio, hp.gamma);
+    }
+    if (!isfinite((float)sred[0]) || !isfinite(smax[0])) atomicOr(status, DEV_STATUS_NONFINITE);
+    mt.sc->norm_scaled = norm;
+    mt.sc->lambda = lam;
+    mt.sc->prev_norm = lam * norm;
+    mt.sc->k_min = smin[0];
+    mt.sc->k_max = smax[0];
+    mt.sc->t = mt.sc->t + 1;
+  }
+}
+
+int launch_simt_step(const SimtPlan& pl, const Hyper& hp, unsigned* status_dev, cudaStream_t st) {
+  if (pl.nlist == 0) return 0;
+  k_project<<<pl.proj_tiles, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.proj_tile_start);
+  const int row_blocks = (pl.rows_total + 7) / 8;
+  k_adam_rows<<<row_blocks, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.row_start, pl.rows_total, hp);
+  k_back_project<MODE_NORM><<<pl.w_tiles, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist,
+                                                                 pl.w_tile_start, 0.f, hp.a_res);
+  k_finalize<<<pl.nlist, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.npart, hp, status_dev);
+  k_form_x<<<row_blocks, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.row_start, pl.rows_total,
+                                       hp.a_low, hp.a_res);
+  k_back_project<MODE_UPDATE><<<pl.w_tiles, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist,
+                                                                   pl.w_tile_start, hp.lr, hp.a_res);
+  return 6;
+}
+
+}  // namespace fira

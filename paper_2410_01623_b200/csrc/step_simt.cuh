@@ -1,0 +1,32 @@
+// Launch interface of the grouped fp32 CUDA-core step kernels.
+#pragma once
+#include "common.cuh"
+
+namespace fira {
+
+// Device-resident schedule of one list of matrices.  `list` holds indices into
+// `mats`; the *_start arrays have nlist + 1 ascending entries (prefix sums).
+struct SimtPlan {
+  const MatDev* mats = nullptr;
+  const int* list = nullptr;
+  int nlist = 0;
+  const int* proj_tile_start = nullptr;  // 64 x 64 tiles of Rt (l x r)
+  int proj_tiles = 0;
+  const int* row_start = nullptr;        // rows l
+  int rows_total = 0;
+  const int* w_tile_start = nullptr;     // 64 x 64 tiles of W (m x n)
+  int w_tiles = 0;
+  const int* npart = nullptr;            // partial sums per matrix (= its W tiles)
+};
+
+// Enqueues the six phases; returns the number of launches.
+int launch_simt_step(const SimtPlan& pl, const Hyper& hp, unsigned* status_dev, cudaStream_t st);
+
+// One block of 256 threads per matrix of the list: sums the matrix's partial sums
+// of ||S||^2 (npart_of[i] floats at mt.part) in a fixed order, applies the limiter
+// rule (Eq. 12 in Algorithm 1's form), stores lambda and the new ||S_prev||,
+// records the range of k and advances t.
+__global__ void k_finalize(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+                           const int* __restrict__ npart_of, Hyper hp, unsigned* __restrict__ status);
+
+}  // namespace fira

@@ -1,0 +1,28 @@
+// Launch interface of the bf16 tensor-core (tcgen05) step kernels.
+#pragma once
+#include <vector>
+
+#include "common.cuh"
+
+struct fira_ctx;
+
+namespace fira {
+
+// Whether the tensor-core kernels can take this matrix (shape and alignment rules
+// of the TMA loads); otherwise it runs on the fp32 CUDA-core kernels.
+bool tc_supported(const fira_matrix_desc& d);
+// Scratch sizes (floats) of the per-(r-tile, l) column partial sums and of the
+// partial sums of ||S||^2.
+size_t tc_colpart_floats(const fira_matrix_desc& d);
+size_t tc_part_floats(const fira_matrix_desc& d);
+// Appends this engine's schedule arrays to `ints` (host image of the device int
+// block) and records where they are.
+fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints);
+void tc_destroy_plan(fira_ctx* c);
+// Called when W / G pointers changed: re-encodes what depends on them.
+fira_status tc_update_pointers(fira_ctx* c);
+// Enqueues the tensor-core phases for the matrices of the tc list; returns the
+// number of launches (negative: error, message set).
+int launch_tc_step(fira_ctx* c, const Hyper& hp);
+
+}  // namespace fira
