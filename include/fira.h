@@ -180,6 +180,19 @@ FIRA_API fira_status fira_poll(fira_ctx* ctx);
 /* Number of kernel launches enqueued by the most recent fira_step() call. */
 FIRA_API int32_t fira_last_step_launches(const fira_ctx* ctx);
 
+/* Per-kernel timing of fira_step() (measurement aid; the paper has no counterpart).
+ * While enabled, every step records CUDA events on the context's stream before and
+ * after each of its kernels (the last FIRA_TIMING_MAX_STEPS steps are kept).
+ * fira_get_phase_times() waits for the stream and returns, per kernel ("phase") in
+ * launch order, the mean duration in milliseconds over the recorded steps; ms_out
+ * has room for FIRA_TIMING_MAX_PHASES floats.  fira_phase_name() names a phase. */
+#define FIRA_TIMING_MAX_PHASES 16
+#define FIRA_TIMING_MAX_STEPS 64
+FIRA_API fira_status fira_enable_phase_timing(fira_ctx* ctx, int32_t enable);
+FIRA_API fira_status fira_get_phase_times(fira_ctx* ctx, int32_t* nphases, float* ms_out,
+                                          int32_t* steps_recorded);
+FIRA_API const char* fira_phase_name(const fira_ctx* ctx, int32_t phase);
+
 FIRA_API const char* fira_status_string(fira_status s);
 /* Text of the most recent error on this thread ("" if none). */
 FIRA_API const char* fira_last_error(void);

@@ -67,6 +67,10 @@ SIGNATURES = {
     "fira_get_diagnostics": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(Diag)]),
     "fira_poll": (C.c_int, [C.c_void_p]),
     "fira_last_step_launches": (C.c_int32, [C.c_void_p]),
+    "fira_enable_phase_timing": (C.c_int, [C.c_void_p, C.c_int32]),
+    "fira_get_phase_times": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_float),
+                                       C.POINTER(C.c_int32)]),
+    "fira_phase_name": (C.c_char_p, [C.c_void_p, C.c_int32]),
     "fira_status_string": (C.c_char_p, [C.c_int]),
     "fira_last_error": (C.c_char_p, []),
     "fira_destroy": (None, [C.c_void_p]),
@@ -220,3 +224,13 @@ class Fira:
 
     def last_step_launches(self) -> int:
         return self.L.fira_last_step_launches(self.ctx)
+
+    def enable_phase_timing(self, enable: bool = True):
+        check(self.L.fira_enable_phase_timing(self.ctx, 1 if enable else 0))
+
+    def phase_times(self):
+        """[(kernel name, mean ms per step)] over the steps recorded since enabling."""
+        n, steps = C.c_int32(), C.c_int32()
+        ms = (C.c_float * 16)()
+        check(self.L.fira_get_phase_times(self.ctx, C.byref(n), ms, C.byref(steps)))
+        return [(self.L.fira_phase_name(self.ctx, i).decode(), ms[i]) for i in range(n.value)], steps.value

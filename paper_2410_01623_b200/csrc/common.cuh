@@ -91,6 +91,22 @@ __device__ __forceinline__ int find_matrix(const int* __restrict__ start, int co
 
 void set_error(const std::string& msg);
 
+// Optional per-kernel timing of a step: marks are CUDA events recorded between the
+// launches.  slot = the step's row of the event ring, next = the next mark.
+struct PhaseTimer {
+  bool on = false;
+  std::vector<cudaEvent_t> events;   // FIRA_TIMING_MAX_STEPS x (FIRA_TIMING_MAX_PHASES + 1)
+  std::vector<const char*> names;    // phase names in launch order
+  int slot = 0, next = 0;
+  long long steps = 0;               // steps recorded since enabling
+  void begin_step() { next = 0; slot = (int)(steps % FIRA_TIMING_MAX_STEPS); }
+  void mark(cudaStream_t st) {
+    if (!on || next > FIRA_TIMING_MAX_PHASES) return;
+    cudaEventRecord(events[(size_t)slot * (FIRA_TIMING_MAX_PHASES + 1) + next], st);
+    ++next;
+  }
+};
+
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
 }  // namespace fira

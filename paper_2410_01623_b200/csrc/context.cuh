@@ -29,6 +29,7 @@ struct fira_ctx {
   fira::TcPlan* tc = nullptr;            // matrices on the tensor-core kernels
   std::vector<int> simt_list, tc_list;
   std::vector<long long> t_host;         // host mirror of every matrix's step count
+  fira::PhaseTimer timer;
   bool table_dirty = true;
   int last_launches = 0;
 };

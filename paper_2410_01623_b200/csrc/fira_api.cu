@@ -285,10 +285,13 @@ fira_status fira_step(fira_ctx* c, void* const* W_dev, const void* const* G_dev,
   }
   if (c->table_dirty) { fira_status s = upload_table(c); if (s != FIRA_OK) return s; }
   const Hyper h = make_hyper(c->hp, lr);
-  int launches = launch_simt_step(c->simt, h, c->status_dev, c->stream);
+  c->timer.begin_step();
+  int launches = launch_simt_step(c->simt, h, c->status_dev, c->stream, &c->timer);
+  if (c->simt.nlist == 0) c->timer.mark(c->stream);
   const int tcl = launch_tc_step(c, h);
   if (tcl < 0) return FIRA_ERR_CUDA;
   launches += tcl;
+  if (c->timer.on) c->timer.steps += 1;
   c->last_launches = launches;
   for (int i = 0; i < count; ++i) c->t_host[i] += 1;
   FIRA_CUDA(cudaGetLastError());
@@ -436,6 +439,49 @@ fira_status fira_poll(fira_ctx* c) {
 
 int32_t fira_last_step_launches(const fira_ctx* c) { return c ? c->last_launches : -1; }
 
+fira_status fira_enable_phase_timing(fira_ctx* c, int32_t enable) {
+  if (!c) { set_error("null context"); return FIRA_ERR_INVALID_ARG; }
+  PhaseTimer& tm = c->timer;
+  if (enable && tm.events.empty()) {
+    tm.events.resize((size_t)FIRA_TIMING_MAX_STEPS * (FIRA_TIMING_MAX_PHASES + 1));
+    for (auto& ev : tm.events) FIRA_CUDA(cudaEventCreate(&ev));
+    if (c->simt.nlist) for (int i = 0; i < 6; ++i) tm.names.push_back(kSimtPhaseNames[i]);
+    if (!c->tc_list.empty()) {
+      const char* nm[8];
+      const int k = tc_phase_names(nm);
+      for (int i = 0; i < k; ++i) tm.names.push_back(nm[i]);
+    }
+  }
+  tm.on = enable != 0;
+  tm.steps = 0;
+  return FIRA_OK;
+}
+
+fira_status fira_get_phase_times(fira_ctx* c, int32_t* nphases, float* ms_out, int32_t* steps_recorded) {
+  if (!c || !nphases || !ms_out || !steps_recorded) { set_error("null argument"); return FIRA_ERR_INVALID_ARG; }
+  PhaseTimer& tm = c->timer;
+  FIRA_CUDA(cudaStreamSynchronize(c->stream));
+  const int np = (int)tm.names.size();
+  const int ns = (int)std::min<long long>(tm.steps, FIRA_TIMING_MAX_STEPS);
+  *nphases = np; *steps_recorded = ns;
+  for (int p = 0; p < np; ++p) {
+    double acc = 0.0;
+    for (int s = 0; s < ns; ++s) {
+      float ms = 0.f;
+      const size_t base = (size_t)s * (FIRA_TIMING_MAX_PHASES + 1);
+      FIRA_CUDA(cudaEventElapsedTime(&ms, tm.events[base + p], tm.events[base + p + 1]));
+      acc += ms;
+    }
+    ms_out[p] = ns ? (float)(acc / ns) : 0.f;
+  }
+  return FIRA_OK;
+}
+
+const char* fira_phase_name(const fira_ctx* c, int32_t phase) {
+  if (!c || phase < 0 || phase >= (int)c->timer.names.size()) return "";
+  return c->timer.names[phase];
+}
+
 const char* fira_status_string(fira_status s) {
   switch (s) {
     case FIRA_OK: return "ok";
@@ -454,6 +500,7 @@ const char* fira_last_error(void) { return g_last_error.c_str(); }
 void fira_destroy(fira_ctx* c) {
   if (!c) return;
   tc_destroy_plan(c);
+  for (auto& ev : c->timer.events) cudaEventDestroy(ev);
   delete c;
 }
 

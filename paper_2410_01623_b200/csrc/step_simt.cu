@@ -225,18 +225,29 @@ k_finalize(const MatDev* __restrict__ mats, const int* __restrict__ list, int nl
   }
 }
 
-int launch_simt_step(const SimtPlan& pl, const Hyper& hp, unsigned* status_dev, cudaStream_t st) {
+const char* const kSimtPhaseNames[6] = {"k_project", "k_adam_rows", "k_back_project<norm>",
+                                        "k_finalize", "k_form_x", "k_back_project<update>"};
+
+int launch_simt_step(const SimtPlan& pl, const Hyper& hp, unsigned* status_dev, cudaStream_t st,
+                     PhaseTimer* tm) {
   if (pl.nlist == 0) return 0;
+  tm->mark(st);
   k_project<<<pl.proj_tiles, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.proj_tile_start);
+  tm->mark(st);
   const int row_blocks = (pl.rows_total + 7) / 8;
   k_adam_rows<<<row_blocks, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.row_start, pl.rows_total, hp);
+  tm->mark(st);
   k_back_project<MODE_NORM><<<pl.w_tiles, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist,
                                                                  pl.w_tile_start, 0.f, hp.a_res);
+  tm->mark(st);
   k_finalize<<<pl.nlist, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.npart, hp, status_dev);
+  tm->mark(st);
   k_form_x<<<row_blocks, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.row_start, pl.rows_total,
                                        hp.a_low, hp.a_res);
+  tm->mark(st);
   k_back_project<MODE_UPDATE><<<pl.w_tiles, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist,
                                                                    pl.w_tile_start, hp.lr, hp.a_res);
+  tm->mark(st);
   return 6;
 }
 

@@ -20,7 +20,9 @@ struct SimtPlan {
 };
 
 // Enqueues the six phases; returns the number of launches.
-int launch_simt_step(const SimtPlan& pl, const Hyper& hp, unsigned* status_dev, cudaStream_t st);
+int launch_simt_step(const SimtPlan& pl, const Hyper& hp, unsigned* status_dev, cudaStream_t st,
+                     PhaseTimer* tm);
+extern const char* const kSimtPhaseNames[6];
 
 // One block of 256 threads per matrix of the list: sums the matrix's partial sums
 // of ||S||^2 (npart_of[i] floats at mt.part) in a fixed order, applies the limiter

@@ -12,5 +12,6 @@ fira_status tc_build_plan(fira_ctx*, std::vector<int>&) { return FIRA_OK; }
 void tc_destroy_plan(fira_ctx*) {}
 fira_status tc_update_pointers(fira_ctx*) { return FIRA_OK; }
 int launch_tc_step(fira_ctx*, const Hyper&) { return 0; }
+int tc_phase_names(const char**) { return 0; }
 
 }  // namespace fira

@@ -24,5 +24,7 @@ fira_status tc_update_pointers(fira_ctx* c);
 // Enqueues the tensor-core phases for the matrices of the tc list; returns the
 // number of launches (negative: error, message set).
 int launch_tc_step(fira_ctx* c, const Hyper& hp);
+// Names of this engine's kernels in launch order (at most 8).
+int tc_phase_names(const char** out);
 
 }  // namespace fira

@@ -1,0 +1,214 @@
+"""GPU parity of fira_step against the fp64 oracle (through the C ABI)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import fira_oracle as fo
+from paper_2410_01623_b200 import binding as fb
+from paper_2410_01623_b200 import workloads as wk
+from tests.parity_util import Trajectory, rel_err, to_np64, workload_trajectory
+
+pytestmark = pytest.mark.gpu
+
+
+def test_single_matrix_workload_with_spike():
+    """The single 512 x 1376, r = 128 fp32 matrix: 10 steps, spike at step 6."""
+    wl = wk.workload("single-60m")
+    tr = workload_trajectory(wl, wl.steps)
+    tr.assert_ok()
+    lams = [row[0] for row in tr.lams]
+    assert lams[5] < 1.0                      # the spike step is limited
+    assert all(l == 1.0 for l in lams[:5])
+    d = tr.f.diagnostics(0)
+    assert d["t"] == wl.steps and d["engine"] == 0
+    assert d["norm_prev"] == pytest.approx(tr.st[0].prev_norm, rel=1e-4)
+    assert tr.f.state_elements(0) == 512 * 128 + 2 * 1376 * 128 + 1
+
+
+def _random_case(shapes, r, dtype, steps, seed, hp=None, spike=None, flags=0):
+    g = torch.Generator().manual_seed(seed)
+    hp = hp or fb.make_hparams(lr=1e-2, alpha=0.25, gamma=1.01, flags=flags)
+    W0 = [(torch.randn(m, n, generator=g) * 0.02).to(dtype) for (m, n) in shapes]
+    tr = Trajectory(shapes, r, dtype, hp, W0)
+    for i, (m, n) in enumerate(shapes):
+        q, _ = torch.linalg.qr(torch.randn(min(m, n), tr.f.ranks[i], generator=g, dtype=torch.float64))
+        tr.f.set_projection(i, q.to(dtype).cuda())
+    scales = [torch.exp(torch.randn(n, generator=g)) for (_, n) in shapes]
+    for s in range(1, steps + 1):
+        mult = 10.0 if spike and s in spike else 1.0
+        Gs = [(torch.randn(m, n, generator=g) * scales[i][None, :] * mult).to(dtype)
+              for i, (m, n) in enumerate(shapes)]
+        tr.step(Gs)
+    return tr
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_ragged_shapes_both_orientations(dtype):
+    # several 64-wide tiles plus ragged tails in every extent; left, right and square
+    shapes = [(150, 333), (333, 150), (130, 130), (64, 200), (7, 9), (9, 7)]
+    ranks = [37, 37, 64, 64, 3, 7]
+    tr = _random_case(shapes, ranks, dtype, steps=6, seed=3, spike=(4,))
+    tr.assert_ok()
+    assert any(l < 1.0 for row in tr.lams for l in row)
+
+
+def test_full_rank_projection_has_no_residual():
+    # r = d with an orthonormal basis: S = 0, the step is Adam through the projection
+    tr = _random_case([(48, 80)], 48, torch.float32, steps=3, seed=5)
+    tr.assert_ok()
+    assert tr.f.diagnostics(0)["norm_prev"] < 1e-4
+
+
+def test_alpha_lowrank_only_flag():
+    tr = _random_case([(96, 160), (160, 96)], 16, torch.float32, steps=4, seed=7,
+                      flags=fb.FLAG_ALPHA_LOWRANK_ONLY)
+    tr.assert_ok()
+
+
+@pytest.mark.parametrize("gamma", [math.inf, 1.0])
+def test_gamma_extremes(gamma):
+    hp = fb.make_hparams(gamma=gamma)
+    tr = _random_case([(100, 140)], 20, torch.float32, steps=5, seed=11, hp=hp, spike=(3,))
+    tr.assert_ok()
+    lams = [row[0] for row in tr.lams]
+    if math.isinf(gamma):
+        assert all(l == 1.0 for l in lams)
+    else:
+        assert lams[2] < 1.0
+
+
+def test_zero_gradient_and_zero_columns():
+    shapes = [(40, 70)]
+    hp = fb.make_hparams()
+    g = torch.Generator().manual_seed(1)
+    W0 = [torch.randn(40, 70, generator=g) * 0.02]
+    tr = Trajectory(shapes, 8, torch.float32, hp, W0)
+    q, _ = torch.linalg.qr(torch.randn(40, 8, generator=g, dtype=torch.float64))
+    tr.f.set_projection(0, q.float().cuda())
+    G = torch.randn(40, 70, generator=g)
+    G[:, 5] = 0.0
+    tr.step([G])
+    tr.step([torch.zeros(40, 70)])          # k = ||N|| / eps is huge, S = 0: finite result
+    tr.step([G])
+    tr.assert_ok()
+    assert torch.isfinite(tr.W[0]).all()
+
+
+def test_per_call_learning_rate_and_pointer_change():
+    shapes = [(70, 90)]
+    g = torch.Generator().manual_seed(2)
+    W0 = [torch.randn(70, 90, generator=g) * 0.02]
+    tr = Trajectory(shapes, 10, torch.float32, fb.make_hparams(lr=1e-2), W0)
+    q, _ = torch.linalg.qr(torch.randn(70, 10, generator=g, dtype=torch.float64))
+    tr.f.set_projection(0, q.float().cuda())
+    tr.step([torch.randn(70, 90, generator=g)], lr=3e-3)
+    # move W to a new allocation: the library must follow the new pointer
+    tr.W = [tr.W[0].clone()]
+    tr.step([torch.randn(70, 90, generator=g)], lr=5e-2)
+    tr.assert_ok()
+
+
+def test_checkpoint_resume_is_bitwise():
+    shapes = [(96, 130), (130, 96)]
+    hp = fb.make_hparams()
+    g = torch.Generator().manual_seed(4)
+    W0 = [torch.randn(m, n, generator=g) * 0.02 for (m, n) in shapes]
+    Ps = [torch.linalg.qr(torch.randn(96, 12, generator=g, dtype=torch.float64))[0].float().cuda()
+          for _ in shapes]
+    Gs = [[torch.randn(m, n, generator=g).cuda() for (m, n) in shapes] for _ in range(6)]
+
+    def run(n_first):
+        f = fb.Fira(shapes, 12, torch.float32, hp)
+        for i in range(2):
+            f.set_projection(i, Ps[i])
+        W = [w.cuda().clone() for w in W0]
+        for s in range(n_first):
+            f.step(W, Gs[s])
+        return f, W
+
+    f_all, W_all = run(6)
+    f_a, W_a = run(3)
+    saved = [f_a.get_state(i) for i in range(2)]
+    projs = [f_a.get_projection(i) for i in range(2)]
+    f_b = fb.Fira(shapes, 12, torch.float32, hp)
+    for i in range(2):
+        f_b.set_projection(i, projs[i])
+        M, V, pn, t = saved[i]
+        assert t == 3 and pn is not None
+        f_b.set_state(i, M, V, pn, t)
+    for s in range(3, 6):
+        f_b.step(W_a, Gs[s])
+    torch.cuda.synchronize()
+    for i in range(2):
+        assert torch.equal(W_a[i], W_all[i])
+        Ma, Va, pa, ta = f_all.get_state(i)
+        Mb, Vb, pb, tb = f_b.get_state(i)
+        assert torch.equal(Ma, Mb) and torch.equal(Va, Vb) and pa == pb and ta == tb == 6
+
+
+def test_moments_match_oracle_layout():
+    tr = _random_case([(60, 100), (100, 60)], 9, torch.float32, steps=3, seed=13)
+    for i, (m, n) in enumerate(tr.shapes):
+        M, V, pn, t = tr.f.get_state(i)
+        Mo = tr.st[i].M.T if m <= n else tr.st[i].M      # library layout is l x r
+        Vo = tr.st[i].V.T if m <= n else tr.st[i].V
+        assert rel_err(to_np64(M), Mo) < 1e-5
+        assert rel_err(to_np64(V), Vo) < 1e-5
+        assert pn == pytest.approx(tr.st[i].prev_norm, rel=1e-4)
+        assert t == 3
+
+
+def test_run_twice_is_bitwise_deterministic():
+    a = _random_case([(150, 333), (333, 150)], 37, torch.bfloat16, steps=4, seed=21, spike=(3,))
+    b = _random_case([(150, 333), (333, 150)], 37, torch.bfloat16, steps=4, seed=21, spike=(3,))
+    for x, y in zip(a.W, b.W):
+        assert torch.equal(x, y)
+
+
+def test_nonfinite_gradient_is_flagged():
+    f = fb.Fira([(32, 48)], 4, torch.float32, fb.make_hparams())
+    W = [torch.zeros(32, 48, device="cuda")]
+    G = torch.ones(32, 48, device="cuda")
+    G[3, 3] = float("inf")
+    f.set_projection(0, torch.eye(32, 4, device="cuda"))
+    f.step(W, [G])
+    assert f.poll() == 6
+    assert f.poll() == 0      # cleared by the previous poll
+
+
+def test_step_argument_errors():
+    f = fb.Fira([(32, 48)], 4, torch.float32, fb.make_hparams())
+    W = torch.zeros(32, 48, device="cuda")
+    with pytest.raises(fb.FiraError) as e:
+        f.step([W], [None])
+    assert e.value.status == 1
+    with pytest.raises(fb.FiraError):
+        f.step([W], [W], lr=float("nan"))
+    assert f.L.fira_get_diagnostics(f.ctx, 5, None) == 1
+    assert f.diagnostics(0)["t"] == 0
+
+
+def test_step_host_matches_device_step():
+    shapes = [(96, 130), (130, 96)]
+    hp = fb.make_hparams()
+    g = torch.Generator().manual_seed(8)
+    W0 = [torch.randn(m, n, generator=g) * 0.02 for (m, n) in shapes]
+    Gs = [torch.randn(m, n, generator=g) for (m, n) in shapes]
+    Ps = [torch.linalg.qr(torch.randn(96, 12, generator=g, dtype=torch.float64))[0].float().cuda()
+          for _ in shapes]
+    fa = fb.Fira(shapes, 12, torch.float32, hp)
+    fh = fb.Fira(shapes, 12, torch.float32, hp)
+    for i in range(2):
+        fa.set_projection(i, Ps[i])
+        fh.set_projection(i, Ps[i])
+    Wd = [w.cuda().clone() for w in W0]
+    fa.step(Wd, [x.cuda() for x in Gs])
+    Wh = [w.clone().pin_memory() for w in W0]
+    Gh = [x.clone().pin_memory() for x in Gs]
+    staging = torch.empty(fh.staging_bytes(), dtype=torch.uint8, device="cuda")
+    fh.step_host(Wh, Gh, staging)
+    torch.cuda.synchronize()
+    for i in range(2):
+        assert torch.equal(Wh[i], Wd[i].cpu())
