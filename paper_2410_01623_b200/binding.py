@@ -184,7 +184,8 @@ class Fira:
 
     def set_projection(self, idx: int, P: torch.Tensor):
         d, _ = self._dl(idx)
-        assert P.shape == (d, self.ranks[idx]) and P.dtype == self.dtype and P.is_contiguous()
+        assert P.shape == (d, self.ranks[idx]) and P.dtype == self.dtype and P.is_cuda
+        P = P.contiguous()   # the copy below is ordered on the same stream as torch's allocator
         check(self.L.fira_set_projection(self.ctx, idx, P.data_ptr()))
 
     def get_projection(self, idx: int) -> torch.Tensor:

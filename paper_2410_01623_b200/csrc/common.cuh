@@ -21,7 +21,7 @@ struct MatScalars {
   float lambda;       // limiter factor of the latest step
   float norm_scaled;  // ||S|| before the limiter
   float k_min, k_max;
-  float pad;
+  float pad;          // bias factor sqrt(1-b2^s)/(1-b1^s) of the running step (tensor-core path)
   long long t;        // steps taken
 };
 static_assert(sizeof(MatScalars) == 32, "MatScalars layout");

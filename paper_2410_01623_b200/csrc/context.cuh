@@ -20,6 +20,7 @@ struct fira_ctx {
   // sections inside the scratch buffer
   fira::MatDev* mats_dev = nullptr;
   unsigned* status_dev = nullptr;
+  char* tc_maps_dev = nullptr;           // tensor maps of the tensor-core path
   int* ints_dev = nullptr;               // all schedule arrays, one block
   size_t ints_count = 0;
   char* work_base = nullptr;             // per-matrix step scratch, reused by the refresh
@@ -41,7 +42,7 @@ struct Layout {
   std::vector<size_t> offP, offM, offV, offS;
   size_t state_bytes = 0;
   // byte offsets inside the scratch buffer
-  size_t off_mats = 0, off_status = 0, off_ints = 0, off_work = 0;
+  size_t off_mats = 0, off_status = 0, off_ints = 0, off_tcmaps = 0, off_work = 0;
   size_t ints_count = 0;
   // byte offsets per matrix inside the work area
   std::vector<size_t> offRt, offXt, offK, offPart, offNb, offRb, offXb, offColpart, offGsq;

@@ -70,6 +70,7 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
   L.off_status = wo; wo += 256;
   L.ints_count = 16 * (size_t)(count + 1);
   L.off_ints = wo; wo += align_up(L.ints_count * sizeof(int));
+  L.off_tcmaps = wo; wo += tc_maps_bytes(count);
   L.off_work = wo;
   size_t w = 0;
   size_t refresh_max = 0;
@@ -91,7 +92,7 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
       L.offRb[i] = w; w += align_up(ll * r * 2);
       L.offXb[i] = w; w += align_up(ll * r * 2);
       L.offColpart[i] = w; w += align_up(tc_colpart_floats(d) * 4);
-      L.offGsq[i] = w; w += align_up(ll * 4);
+      L.offGsq[i] = w; w += align_up(tc_gsq_floats(d) * 4);
       L.offPart[i] = w; w += align_up(tc_part_floats(d) * 4);
     }
     refresh_max = std::max(refresh_max, refresh_bytes_per_matrix(d));
@@ -168,6 +169,7 @@ fira_status fira_init(fira_ctx** out, const fira_hparams* hp, const fira_matrix_
   c->status_dev = (unsigned*)(c->scratch_base + L.off_status);
   c->ints_dev = (int*)(c->scratch_base + L.off_ints);
   c->ints_count = L.ints_count;
+  c->tc_maps_dev = c->scratch_base + L.off_tcmaps;
   c->work_base = c->scratch_base + L.off_work;
   c->work_bytes = scratch_bytes - L.off_work;
 

@@ -1,17 +1,724 @@
-// bf16 tensor-core step kernels (placeholder until the tcgen05 path lands: every
-// matrix is routed to the fp32 CUDA-core kernels).
+// bf16 tensor-core kernels of the Fira step (Algorithm 1's loop body) for sm_100a:
+// TMA-fed tcgen05.mma with fp32 accumulators in tensor memory and fused epilogues,
+// grouped over a list of matrices (persistent CTAs walk a static tile list).
+//
+// l = unprojected index (columns of G when m <= n, rows otherwise), d = projected
+// index, Pi = the d x r projection.  Launches per step:
+//   k_tc_prep          bias factor sqrt(1-b2^s)/(1-b1^s) per matrix
+//   k_tc_gsq           partial sums of G^2 per l                          (for ||S||)
+//   k_tc_project       Rt = G^T Pi on the tensor cores; epilogue: M, V update (Eq. 2-3),
+//                      N (Eq. 4), bf16 copies of N and R, per-l partial ||N_l||^2, ||R_l||^2
+//   k_tc_colfactors    k_l (Eq. 11) and partial sums of ||S||^2 = sum_l k_l^2 (||G_l||^2 - ||R_l||^2)
+//   k_finalize         lambda, ||S_prev||, t (Eq. 12)
+//   k_tc_form_x        X = a_low N - a_res lambda k_l R  (bf16)
+//   k_tc_back_project  D = Pi X on the tensor cores; epilogue: W -= lr (D + a_res lambda k_l G)
+//
+// ||S_l||^2 = ||G_l||^2 - ||R_l||^2 holds for a projection with orthonormal columns;
+// with a bf16-rounded projection it is exact to about 2^-8 ||R_l||^2.  It only enters
+// the limiter factor lambda and the remembered norm.
+//
+// Tile shapes: 128 (TMEM lanes) x BN <= 256 (TMEM columns) x 64 (one 128-byte swizzle
+// row of bf16) per pipeline stage; two accumulators of 256 columns alternate so that
+// the epilogue of one tile overlaps the products of the next.
+#include <cuda.h>
+
+#include <algorithm>
+
 #include "context.cuh"
 #include "step_tc.cuh"
+#include "tc_ptx.cuh"
 
 namespace fira {
 
-bool tc_supported(const fira_matrix_desc&) { return false; }
-size_t tc_colpart_floats(const fira_matrix_desc&) { return 0; }
-size_t tc_part_floats(const fira_matrix_desc&) { return 0; }
-fira_status tc_build_plan(fira_ctx*, std::vector<int>&) { return FIRA_OK; }
-void tc_destroy_plan(fira_ctx*) {}
-fira_status tc_update_pointers(fira_ctx*) { return FIRA_OK; }
-int launch_tc_step(fira_ctx*, const Hyper&) { return 0; }
-int tc_phase_names(const char**) { return 0; }
+namespace {
+
+constexpr int BM = 128;           // tile rows = TMEM lanes
+constexpr int BN_MAX = 256;       // tile columns = TMEM columns per accumulator
+constexpr int BK = 64;            // k-block: 64 bf16 = 128 bytes
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;       // 16 KiB
+constexpr int B_STAGE_BYTES = BN_MAX * BK * 2;   // 32 KiB
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int CHUNK_BYTES = 64 * BK * 2;         // one 64 x 64 box: 8 KiB
+constexpr int EPI_WARPS = 8;
+constexpr int TC_THREADS = 32 * (2 + EPI_WARPS);
+constexpr int TMEM_COLS = 512;
+constexpr size_t TC_SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + 256;
+constexpr int GSQ_ROWS = 128;     // rows per partial sum of G^2 (left orientation)
+
+struct TcMaps {
+  CUtensorMap g1a;   // G, box for the projection product
+  CUtensorMap g1b;   // Pi [d][r], boxes of 64 r x 64 d
+  CUtensorMap g2a;   // back-projection A operand (Pi when left, X when right), box 64 x 128
+  CUtensorMap g2b;   // back-projection B operand (X when left, Pi when right), box 64 x 256
+};
+static_assert(sizeof(TcMaps) % 64 == 0, "tensor maps must stay 64-byte aligned");
+
+__device__ __forceinline__ int tile_bn(int r) {
+  return (r % 256 == 0) ? 256 : (r % 192 == 0) ? 192 : (r % 128 == 0) ? 128 : 64;
+}
+
+struct SharedCtl {
+  uint64_t full[STAGES];
+  uint64_t empty[STAGES];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// Common prologue: carve shared memory, init barriers, allocate TMEM.
+__device__ __forceinline__ void tc_prologue(unsigned char* smem_raw, unsigned char*& tiles, SharedCtl*& ctl) {
+  const uintptr_t base = (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023;
+  tiles = reinterpret_cast<unsigned char*>(base);
+  ctl = reinterpret_cast<SharedCtl*>(tiles + (size_t)STAGES * STAGE_BYTES);
+  const int warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&ctl->full[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(ptx::smem_u32(&ctl->tmem_full[b]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[b]), EPI_WARPS);
+    }
+    ctl->abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(&ctl->tmem_base), TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+}
+
+__device__ __forceinline__ void tc_epilogue_teardown(SharedCtl* ctl, unsigned* status) {
+  ptx::tc_fence_before();
+  __syncthreads();
+  if ((threadIdx.x >> 5) == 1) {
+    __syncwarp();
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(ctl->tmem_base, TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && ctl->abort_flag) atomicOr(status, DEV_STATUS_TIMEOUT);
+}
+
+// After an aborted run the producer gives its copies in flight a bounded time to land.
+__device__ __forceinline__ void drain_stage_waits(SharedCtl* ctl, int stage, uint32_t phase, int issued_any) {
+  if (!issued_any) return;
+  for (int s = 0; s < STAGES; ++s)
+    for (uint32_t it = 0; it < (1u << 16); ++it)
+      if (ptx::mbar_try_wait(ptx::smem_u32(&ctl->full[s]), (s < stage) ? phase : (phase ^ 1u))) break;
+}
+
+__device__ __forceinline__ uint4 pack8_bf16(const float (&v)[8]) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
+  __nv_bfloat162 b = __floats2bfloat162_rn(v[2], v[3]);
+  __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]);
+  __nv_bfloat162 d = __floats2bfloat162_rn(v[6], v[7]);
+  uint4 o;
+  o.x = *reinterpret_cast<uint32_t*>(&a); o.y = *reinterpret_cast<uint32_t*>(&b);
+  o.z = *reinterpret_cast<uint32_t*>(&c); o.w = *reinterpret_cast<uint32_t*>(&d);
+  return o;
+}
+__device__ __forceinline__ void unpack8_bf16(const uint4& u, float (&v)[8]) {
+  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __bfloat1622float2(p[i]);
+    v[2 * i] = f.x; v[2 * i + 1] = f.y;
+  }
+}
+
+// ============================================================================ projection product
+// Rt[l][j] = sum_d G(d,l) Pi[d][j].  Tile: 128 l x BN r.  A = G: left orientation
+// MN-major (G is [d][l], l contiguous: two 64 x 64 boxes), right orientation K-major
+// (G is [l][d]: one box of 64 d x 128 l).  B = Pi [d][r]: MN-major, BN/64 boxes.
+__global__ void __launch_bounds__(TC_THREADS, 1)
+k_tc_project(const MatDev* __restrict__ mats, const TcMaps* __restrict__ maps, const int* __restrict__ list,
+             int nlist, const int* __restrict__ tile_start, int total_tiles, Hyper hp,
+             unsigned* __restrict__ status) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* tiles;
+  SharedCtl* ctl;
+  tc_prologue(smem_raw, tiles, ctl);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &ctl->abort_flag;
+  const uint32_t tiles_u32 = ptx::smem_u32(tiles);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; int issued = 0; bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const int p = find_matrix(tile_start, nlist, t);
+        const MatDev& mt = mats[list[p]];
+        const TcMaps* mp = &maps[p];
+        const int r = mt.r, d = mt.d, left = mt.left;
+        const int bn = tile_bn(r), nrt = r / bn;
+        const int local = t - tile_start[p];
+        const int l0 = (local / nrt) * BM, r0 = (local % nrt) * bn;
+        const int nkb = (d + BK - 1) / BK;
+        const uint32_t bytes = A_STAGE_BYTES + bn * BK * 2;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
+          const uint32_t sa = tiles_u32 + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+          ptx::mbar_expect_tx(fb, bytes);
+          const int k0 = kb * BK;
+          if (left) {
+            ptx::tma_load_2d(sa, &mp->g1a, fb, l0, k0);
+            ptx::tma_load_2d(sa + CHUNK_BYTES, &mp->g1a, fb, l0 + 64, k0);
+          } else {
+            ptx::tma_load_2d(sa, &mp->g1a, fb, k0, l0);
+          }
+          for (int c = 0; c < bn / 64; ++c) ptx::tma_load_2d(sb + c * CHUNK_BYTES, &mp->g1b, fb, r0 + 64 * c, k0);
+          issued = 1;
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) drain_stage_waits(ctl, stage, phase, issued);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; int buf = 0; uint32_t bphase = 0; bool ok = true;
+      const uint32_t tmem = ctl->tmem_base;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const int p = find_matrix(tile_start, nlist, t);
+        const MatDev& mt = mats[list[p]];
+        const int left = mt.left, bn = tile_bn(mt.r);
+        const int nkb = (mt.d + BK - 1) / BK;
+        const uint32_t idesc = ptx::make_idesc_bf16(BM, bn, left, 1);
+        if (!ptx::mbar_wait(ptx::smem_u32(&ctl->tmem_empty[buf]), bphase ^ 1u, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t dcol = tmem + buf * BN_MAX;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t sa = tiles_u32 + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            // MN-major: 16 k-rows of 128 bytes per step; K-major: 32 bytes along the row
+            const uint64_t ad = left ? ptx::make_smem_desc(sa + k * 2048, CHUNK_BYTES, 1024)
+                                     : ptx::make_smem_desc(sa + k * 32, 0, 1024);
+            const uint64_t bd = ptx::make_smem_desc(sb + k * 2048, CHUNK_BYTES, 1024);
+            ptx::umma_bf16(dcol, ad, bd, idesc, (kb | k) ? 1u : 0u);
+          }
+          ptx::umma_commit(ptx::smem_u32(&ctl->empty[stage]));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::umma_commit(ptx::smem_u32(&ctl->tmem_full[buf]));
+        if (++buf == 2) { buf = 0; bphase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue: Adam on R
+    const int ew = warp - 2;
+    const int quarter = warp & 3;       // TMEM lanes 32*quarter .. +31 are this warp's
+    const int half = ew >> 2;           // which half of the tile's columns
+    int buf = 0; uint32_t bphase = 0;
+    const uint32_t tmem = ctl->tmem_base;
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+      const int p = find_matrix(tile_start, nlist, t);
+      const MatDev& mt = mats[list[p]];
+      const int r = mt.r, L = mt.l;
+      const int bn = tile_bn(r), nrt = r / bn;
+      const int local = t - tile_start[p];
+      const int rt = local % nrt;
+      const int l = (local / nrt) * BM + quarter * 32 + lane;
+      const int cols_half = bn / 2;                 // multiple of 32
+      const int cbase = half * cols_half;
+      const float bias = mt.sc->pad;
+      const bool row_ok = l < L;
+      if (!ptx::mbar_wait(ptx::smem_u32(&ctl->tmem_full[buf]), bphase, abort_flag)) break;
+      ptx::tc_fence_after();
+      float nn = 0.f, rn = 0.f;
+      const long long rowoff = (long long)l * r + rt * bn + cbase;
+      for (int c = 0; c < cols_half; c += 32) {
+        uint32_t rr[32];
+        ptx::tmem_ld_32x32b_x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX + cbase + c, rr);
+        ptx::tmem_ld_wait();
+        if (row_ok) {
+          float* Mp = mt.M + rowoff + c;
+          float* Vp = mt.V + rowoff + c;
+          __nv_bfloat16* Np = mt.Nb + rowoff + c;
+          __nv_bfloat16* Rp = mt.Rb + rowoff + c;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float4 m0 = *reinterpret_cast<const float4*>(Mp + 8 * q);
+            const float4 m1 = *reinterpret_cast<const float4*>(Mp + 8 * q + 4);
+            const float4 v0 = *reinterpret_cast<const float4*>(Vp + 8 * q);
+            const float4 v1 = *reinterpret_cast<const float4*>(Vp + 8 * q + 4);
+            float mo[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+            float vo[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+            float rv[8], nv[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              rv[e] = __uint_as_float(rr[8 * q + e]);
+              mo[e] = hp.beta1 * mo[e] + (1.f - hp.beta1) * rv[e];
+              vo[e] = hp.beta2 * vo[e] + (1.f - hp.beta2) * rv[e] * rv[e];
+              nv[e] = bias * mo[e] / (sqrtf(vo[e]) + hp.eps);
+              nn = fmaf(nv[e], nv[e], nn);
+              rn = fmaf(rv[e], rv[e], rn);
+            }
+            *reinterpret_cast<float4*>(Mp + 8 * q) = make_float4(mo[0], mo[1], mo[2], mo[3]);
+            *reinterpret_cast<float4*>(Mp + 8 * q + 4) = make_float4(mo[4], mo[5], mo[6], mo[7]);
+            *reinterpret_cast<float4*>(Vp + 8 * q) = make_float4(vo[0], vo[1], vo[2], vo[3]);
+            *reinterpret_cast<float4*>(Vp + 8 * q + 4) = make_float4(vo[4], vo[5], vo[6], vo[7]);
+            *reinterpret_cast<uint4*>(Np + 8 * q) = pack8_bf16(nv);
+            *reinterpret_cast<uint4*>(Rp + 8 * q) = pack8_bf16(rv);
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[buf]));
+      if (row_ok) {
+        // colpart[0][part][l] = partial ||N_l||^2, colpart[1][part][l] = partial ||R_l||^2
+        const int nparts = 2 * nrt, part = rt * 2 + half;
+        mt.colpart[(long long)part * L + l] = nn;
+        mt.colpart[(long long)(nparts + part) * L + l] = rn;
+      }
+      if (++buf == 2) { buf = 0; bphase ^= 1u; }
+    }
+  }
+  tc_epilogue_teardown(ctl, status);
+}
+
+// ============================================================================ back-projection product
+// D[i][j] = sum_q A(i,q) B(j,q) over the rank index q, both operands K-major:
+// left: A = Pi [d][r] (i = row of W), B = X [l][r] (j = column of W);
+// right: A = X [l][r], B = Pi [d][r].  Tile 128 x 256 of W.
+// Epilogue: W[i][j] -= lr (D + a_res lambda k G[i][j]), k taken per column (left) or
+// per row (right).
+__global__ void __launch_bounds__(TC_THREADS, 1)
+k_tc_back_project(const MatDev* __restrict__ mats, const TcMaps* __restrict__ maps,
+                  const int* __restrict__ list, int nlist, const int* __restrict__ tile_start,
+                  int total_tiles, Hyper hp, unsigned* __restrict__ status) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* tiles;
+  SharedCtl* ctl;
+  tc_prologue(smem_raw, tiles, ctl);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &ctl->abort_flag;
+  const uint32_t tiles_u32 = ptx::smem_u32(tiles);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; int issued = 0; bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const int p = find_matrix(tile_start, nlist, t);
+        const MatDev& mt = mats[list[p]];
+        const TcMaps* mp = &maps[p];
+        const int nct = (mt.n + BN_MAX - 1) / BN_MAX;
+        const int local = t - tile_start[p];
+        const int i0 = (local / nct) * BM, j0 = (local % nct) * BN_MAX;
+        const int nkb = mt.r / BK;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
+          const uint32_t sa = tiles_u32 + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+          ptx::mbar_expect_tx(fb, STAGE_BYTES);
+          ptx::tma_load_2d(sa, &mp->g2a, fb, kb * BK, i0);
+          ptx::tma_load_2d(sb, &mp->g2b, fb, kb * BK, j0);
+          issued = 1;
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) drain_stage_waits(ctl, stage, phase, issued);
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; int buf = 0; uint32_t bphase = 0; bool ok = true;
+      const uint32_t tmem = ctl->tmem_base;
+      const uint32_t idesc = ptx::make_idesc_bf16(BM, BN_MAX, 0, 0);
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const int p = find_matrix(tile_start, nlist, t);
+        const int nkb = mats[list[p]].r / BK;
+        if (!ptx::mbar_wait(ptx::smem_u32(&ctl->tmem_empty[buf]), bphase ^ 1u, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t dcol = tmem + buf * BN_MAX;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t sa = tiles_u32 + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t ad = ptx::make_smem_desc(sa + k * 32, 0, 1024);
+            const uint64_t bd = ptx::make_smem_desc(sb + k * 32, 0, 1024);
+            ptx::umma_bf16(dcol, ad, bd, idesc, (kb | k) ? 1u : 0u);
+          }
+          ptx::umma_commit(ptx::smem_u32(&ctl->empty[stage]));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::umma_commit(ptx::smem_u32(&ctl->tmem_full[buf]));
+        if (++buf == 2) { buf = 0; bphase ^= 1u; }
+      }
+    }
+  } else {
+    const int ew = warp - 2;
+    const int quarter = warp & 3;
+    const int half = ew >> 2;
+    int buf = 0; uint32_t bphase = 0;
+    const uint32_t tmem = ctl->tmem_base;
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+      const int p = find_matrix(tile_start, nlist, t);
+      const MatDev& mt = mats[list[p]];
+      const int n = mt.n, m = mt.m, left = mt.left;
+      const long long ld = mt.ld;
+      const int nct = (n + BN_MAX - 1) / BN_MAX;
+      const int local = t - tile_start[p];
+      const int i = (local / nct) * BM + quarter * 32 + lane;
+      const int jbase = (local % nct) * BN_MAX + half * (BN_MAX / 2);
+      const bool row_ok = i < m;
+      const float cres = hp.a_res * mt.sc->lambda;
+      const float krow = (!left && row_ok) ? mt.kvec[i] : 0.f;
+      const __nv_bfloat16* Gp = static_cast<const __nv_bfloat16*>(mt.G) + (long long)i * ld;
+      __nv_bfloat16* Wp = static_cast<__nv_bfloat16*>(mt.W) + (long long)i * ld;
+      if (!ptx::mbar_wait(ptx::smem_u32(&ctl->tmem_full[buf]), bphase, abort_flag)) break;
+      ptx::tc_fence_after();
+      for (int c = 0; c < BN_MAX / 2; c += 32) {
+        uint32_t dd[32];
+        ptx::tmem_ld_32x32b_x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX + half * (BN_MAX / 2) + c, dd);
+        ptx::tmem_ld_wait();
+        if (row_ok) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int j = jbase + c + 8 * q;
+            if (j < n) {            // n is a multiple of 8: the 8 columns are all inside
+              const uint4 gu = *reinterpret_cast<const uint4*>(Gp + j);
+              const uint4 wu = *reinterpret_cast<const uint4*>(Wp + j);
+              float g[8], w[8], kf[8];
+              unpack8_bf16(gu, g);
+              unpack8_bf16(wu, w);
+              if (left) {
+                const float4 k0 = *reinterpret_cast<const float4*>(mt.kvec + j);
+                const float4 k1 = *reinterpret_cast<const float4*>(mt.kvec + j + 4);
+                kf[0] = k0.x; kf[1] = k0.y; kf[2] = k0.z; kf[3] = k0.w;
+                kf[4] = k1.x; kf[5] = k1.y; kf[6] = k1.z; kf[7] = k1.w;
+              } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) kf[e] = krow;
+              }
+#pragma unroll
+              for (int e = 0; e < 8; ++e)
+                w[e] = w[e] - hp.lr * (__uint_as_float(dd[8 * q + e]) + cres * kf[e] * g[e]);
+              *reinterpret_cast<uint4*>(Wp + j) = pack8_bf16(w);
+            }
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[buf]));
+      if (++buf == 2) { buf = 0; bphase ^= 1u; }
+    }
+  }
+  tc_epilogue_teardown(ctl, status);
+}
+
+// ============================================================================ small kernels
+__global__ void k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist, Hyper hp) {
+  const int p = blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= nlist) return;
+  const MatDev& mt = mats[list[p]];
+  const double s = (double)(mt.sc->t + 1);
+  mt.sc->pad = (float)(sqrt(1.0 - pow((double)hp.beta2, s)) / (1.0 - pow((double)hp.beta1, s)));
+}
+
+// Sums of G^2 per unprojected index.  Left: gsq[rb][col] over blocks of GSQ_ROWS rows
+// (one block = GSQ_ROWS rows x 2048 columns, 8 columns per thread); right: gsq[0][row],
+// one warp per row.  `start` counts blocks.
+__global__ void __launch_bounds__(256)
+k_tc_gsq(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+         const int* __restrict__ start) {
+  const int p = find_matrix(start, nlist, blockIdx.x);
+  const MatDev& mt = mats[list[p]];
+  const int b = blockIdx.x - start[p];
+  const __nv_bfloat16* G = static_cast<const __nv_bfloat16*>(mt.G);
+  if (mt.left) {
+    const int ncb = (mt.n + 2047) / 2048;
+    const int rb = b / ncb, cb = b % ncb;
+    const int col = cb * 2048 + threadIdx.x * 8;
+    if (col >= mt.n) return;
+    float acc[8] = {};
+    const int row_end = min(mt.m, (rb + 1) * GSQ_ROWS);
+    for (int row = rb * GSQ_ROWS; row < row_end; ++row) {
+      const uint4 u = *reinterpret_cast<const uint4*>(G + (long long)row * mt.ld + col);
+      float g[8];
+      unpack8_bf16(u, g);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = fmaf(g[e], g[e], acc[e]);
+    }
+    float* out = mt.gsq + (long long)rb * mt.l + col;
+    *reinterpret_cast<float4*>(out) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    *reinterpret_cast<float4*>(out + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+  } else {
+    const int row = b * 8 + (threadIdx.x >> 5);
+    if (row >= mt.m) return;
+    const int lane = threadIdx.x & 31;
+    float acc = 0.f;
+    for (int col = lane * 8; col < mt.n; col += 256) {
+      const uint4 u = *reinterpret_cast<const uint4*>(G + (long long)row * mt.ld + col);
+      float g[8];
+      unpack8_bf16(u, g);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc = fmaf(g[e], g[e], acc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) mt.gsq[row] = acc;
+  }
+}
+
+// k_l and the partial sums of ||S||^2, 256 values of l per block.
+__global__ void __launch_bounds__(256)
+k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+                const int* __restrict__ start, Hyper hp) {
+  __shared__ float red[8];
+  const int p = find_matrix(start, nlist, blockIdx.x);
+  const MatDev& mt = mats[list[p]];
+  const int b = blockIdx.x - start[p];
+  const int l = b * 256 + threadIdx.x;
+  float contrib = 0.f;
+  if (l < mt.l) {
+    const int nparts = 2 * (mt.r / tile_bn(mt.r));
+    float nn = 0.f, rn = 0.f, gs = 0.f;
+    for (int q = 0; q < nparts; ++q) {
+      nn += mt.colpart[(long long)q * mt.l + l];
+      rn += mt.colpart[(long long)(nparts + q) * mt.l + l];
+    }
+    const int ngs = mt.left ? (mt.d + GSQ_ROWS - 1) / GSQ_ROWS : 1;
+    for (int q = 0; q < ngs; ++q) gs += mt.gsq[(long long)q * mt.l + l];
+    const float k = sqrtf(nn) / (sqrtf(rn) + hp.eps);
+    mt.kvec[l] = k;
+    contrib = k * k * fmaxf(gs - rn, 0.f);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xffffffffu, contrib, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = contrib;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    mt.part[b] = tot;
+  }
+}
+
+// X = a_low N - a_res lambda k_l R in bf16, one warp per l.
+__global__ void __launch_bounds__(256)
+k_tc_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+            const int* __restrict__ row_start, int rows_total, float a_low, float a_res) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= rows_total) return;
+  const int p = find_matrix(row_start, nlist, row);
+  const MatDev& mt = mats[list[p]];
+  const int l = row - row_start[p];
+  const float c = a_res * mt.sc->lambda * mt.kvec[l];
+  const long long base = (long long)l * mt.r;
+  for (int j = lane * 8; j < mt.r; j += 256) {
+    const uint4 nu = *reinterpret_cast<const uint4*>(mt.Nb + base + j);
+    const uint4 ru = *reinterpret_cast<const uint4*>(mt.Rb + base + j);
+    float nv[8], rv[8], x[8];
+    unpack8_bf16(nu, nv);
+    unpack8_bf16(ru, rv);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) x[e] = a_low * nv[e] - c * rv[e];
+    *reinterpret_cast<uint4*>(mt.Xb + base + j) = pack8_bf16(x);
+  }
+}
+
+// ============================================================================ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* sym = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(sym);
+  return fn;
+}
+
+// bf16 row-major matrix [rows][cols] with leading dimension ld; box = box_c x box_r.
+bool encode_map(CUtensorMap* out, const void* base, long long rows, long long cols, long long ld,
+                int box_c, int box_r) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) { set_error("cuTensorMapEncodeTiled is not available"); return false; }
+  const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t gstr[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)box_c, (cuuint32_t)box_r};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with code " + std::to_string((int)r)); return false; }
+  return true;
+}
+
+int host_tile_bn(int r) { return (r % 256 == 0) ? 256 : (r % 192 == 0) ? 192 : (r % 128 == 0) ? 128 : 64; }
+
+}  // namespace
+
+struct TcPlan {
+  std::vector<TcMaps> maps;          // host image, one entry per matrix of the tc list
+  TcMaps* maps_dev = nullptr;        // lives in the scratch buffer
+  const int* list = nullptr;
+  int nlist = 0;
+  const int* k1_start = nullptr; int k1_tiles = 0;
+  const int* k2_start = nullptr; int k2_tiles = 0;
+  const int* gsq_start = nullptr; int gsq_blocks = 0;
+  const int* col_start = nullptr; int col_blocks = 0;
+  const int* row_start = nullptr; int rows_total = 0;
+  const int* npart = nullptr;
+  int num_sms = 148;
+  bool attrs_set = false;
+};
+
+bool tc_supported(const fira_matrix_desc& d) {
+  const long long ld = d.ld ? d.ld : d.n;
+  return d.dtype == FIRA_BF16 && d.r % 64 == 0 && d.m >= 256 && d.n >= 256 && d.n % 8 == 0 && ld % 8 == 0;
+}
+
+size_t tc_colpart_floats(const fira_matrix_desc& d) {
+  const size_t l = std::max(d.m, d.n);
+  return 2 * (size_t)(2 * (d.r / host_tile_bn(d.r))) * l;
+}
+
+size_t tc_gsq_floats(const fira_matrix_desc& d) {
+  const size_t l = std::max(d.m, d.n), dd = std::min(d.m, d.n);
+  return (d.m <= d.n ? (dd + GSQ_ROWS - 1) / GSQ_ROWS : 1) * l;
+}
+
+size_t tc_part_floats(const fira_matrix_desc& d) { return ((size_t)std::max(d.m, d.n) + 255) / 256; }
+
+size_t tc_maps_bytes(int count) { return align_up(sizeof(TcMaps) * (size_t)count); }
+
+static bool encode_matrix_maps(const MatDev& mt, TcMaps& mp, bool only_g) {
+  // G is [m][n]: left -> boxes of 64 l x 64 d rows; right -> box of 64 d x 128 l rows
+  if (!encode_map(&mp.g1a, mt.G, mt.m, mt.n, mt.ld, 64, mt.left ? 64 : 128)) return false;
+  if (only_g) return true;
+  if (!encode_map(&mp.g1b, mt.P, mt.d, mt.r, mt.r, 64, 64)) return false;
+  const void* a2 = mt.left ? (const void*)mt.P : (const void*)mt.Xb;
+  const void* b2 = mt.left ? (const void*)mt.Xb : (const void*)mt.P;
+  const long long a2rows = mt.left ? mt.d : mt.l, b2rows = mt.left ? mt.l : mt.d;
+  if (!encode_map(&mp.g2a, a2, a2rows, mt.r, mt.r, 64, 128)) return false;
+  if (!encode_map(&mp.g2b, b2, b2rows, mt.r, mt.r, 64, 256)) return false;
+  return true;
+}
+
+fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
+  if (c->tc_list.empty()) return FIRA_OK;
+  TcPlan* pl = new TcPlan();
+  c->tc = pl;
+  cudaDeviceGetAttribute(&pl->num_sms, cudaDevAttrMultiProcessorCount, c->device);
+  const std::vector<int>& lst = c->tc_list;
+  std::vector<int> k1{0}, k2{0}, gs{0}, cs{0}, rs{0}, np;
+  for (int i : lst) {
+    const MatDev& mt = c->mats[i];
+    const int bn = host_tile_bn(mt.r);
+    k1.push_back(k1.back() + ((mt.l + BM - 1) / BM) * (mt.r / bn));
+    k2.push_back(k2.back() + ((mt.m + BM - 1) / BM) * ((mt.n + BN_MAX - 1) / BN_MAX));
+    const int gblocks = mt.left ? ((mt.d + GSQ_ROWS - 1) / GSQ_ROWS) * ((mt.n + 2047) / 2048) : (mt.m + 7) / 8;
+    gs.push_back(gs.back() + gblocks);
+    const int cb = (mt.l + 255) / 256;
+    cs.push_back(cs.back() + cb);
+    rs.push_back(rs.back() + mt.l);
+    np.push_back(cb);
+  }
+  auto push_block = [&](const std::vector<int>& v) {
+    size_t o = ints.size();
+    ints.insert(ints.end(), v.begin(), v.end());
+    return o;
+  };
+  const size_t o_list = push_block(lst), o_k1 = push_block(k1), o_k2 = push_block(k2), o_gs = push_block(gs),
+               o_cs = push_block(cs), o_rs = push_block(rs), o_np = push_block(np);
+  pl->list = c->ints_dev + o_list; pl->nlist = (int)lst.size();
+  pl->k1_start = c->ints_dev + o_k1; pl->k1_tiles = k1.back();
+  pl->k2_start = c->ints_dev + o_k2; pl->k2_tiles = k2.back();
+  pl->gsq_start = c->ints_dev + o_gs; pl->gsq_blocks = gs.back();
+  pl->col_start = c->ints_dev + o_cs; pl->col_blocks = cs.back();
+  pl->row_start = c->ints_dev + o_rs; pl->rows_total = rs.back();
+  pl->npart = c->ints_dev + o_np;
+  pl->maps.resize(lst.size());
+  pl->maps_dev = reinterpret_cast<TcMaps*>(c->tc_maps_dev);
+  // maps that do not depend on W / G; the G map is encoded when the pointers are known
+  for (size_t q = 0; q < lst.size(); ++q) {
+    MatDev mt = c->mats[lst[q]];
+    mt.G = mt.P;   // placeholder address with valid alignment; replaced in tc_update_pointers
+    if (!encode_matrix_maps(mt, pl->maps[q], false)) return FIRA_ERR_CUDA;
+  }
+  return FIRA_OK;
+}
+
+void tc_destroy_plan(fira_ctx* c) {
+  delete c->tc;
+  c->tc = nullptr;
+}
+
+fira_status tc_update_pointers(fira_ctx* c) {
+  TcPlan* pl = c->tc;
+  if (!pl) return FIRA_OK;
+  for (size_t q = 0; q < c->tc_list.size(); ++q)
+    if (!encode_matrix_maps(c->mats[c->tc_list[q]], pl->maps[q], true)) return FIRA_ERR_CUDA;
+  cudaError_t e = cudaMemcpyAsync(pl->maps_dev, pl->maps.data(), sizeof(TcMaps) * pl->maps.size(),
+                                  cudaMemcpyHostToDevice, c->stream);
+  if (e != cudaSuccess) { set_error(std::string("tensor map upload: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
+  return FIRA_OK;
+}
+
+int tc_phase_names(const char** out) {
+  static const char* names[7] = {"k_tc_prep", "k_tc_gsq", "k_tc_project", "k_tc_colfactors",
+                                 "k_finalize(tc)", "k_tc_form_x", "k_tc_back_project"};
+  for (int i = 0; i < 7; ++i) out[i] = names[i];
+  return 7;
+}
+
+int launch_tc_step(fira_ctx* c, const Hyper& hp) {
+  TcPlan* pl = c->tc;
+  if (!pl || pl->nlist == 0) return 0;
+  cudaStream_t st = c->stream;
+  if (!pl->attrs_set) {
+    cudaError_t e1 = cudaFuncSetAttribute(k_tc_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES);
+    cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES);
+    if (e1 != cudaSuccess || e2 != cudaSuccess) {
+      set_error(std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
+      return -1;
+    }
+    pl->attrs_set = true;
+  }
+  PhaseTimer* tm = &c->timer;
+  const MatDev* mats = c->mats_dev;
+  k_tc_prep<<<(pl->nlist + 127) / 128, 128, 0, st>>>(mats, pl->list, pl->nlist, hp);
+  tm->mark(st);
+  k_tc_gsq<<<pl->gsq_blocks, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->gsq_start);
+  tm->mark(st);
+  k_tc_project<<<std::min(pl->k1_tiles, pl->num_sms), TC_THREADS, TC_SMEM_BYTES, st>>>(
+      mats, pl->maps_dev, pl->list, pl->nlist, pl->k1_start, pl->k1_tiles, hp, c->status_dev);
+  tm->mark(st);
+  k_tc_colfactors<<<pl->col_blocks, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->col_start, hp);
+  tm->mark(st);
+  k_finalize<<<pl->nlist, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->npart, hp, c->status_dev);
+  tm->mark(st);
+  k_tc_form_x<<<(pl->rows_total + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start,
+                                                        pl->rows_total, hp.a_low, hp.a_res);
+  tm->mark(st);
+  k_tc_back_project<<<std::min(pl->k2_tiles, pl->num_sms), TC_THREADS, TC_SMEM_BYTES, st>>>(
+      mats, pl->maps_dev, pl->list, pl->nlist, pl->k2_start, pl->k2_tiles, hp, c->status_dev);
+  tm->mark(st);
+  return 7;
+}
 
 }  // namespace fira

@@ -137,7 +137,7 @@ def random_projection(wl: Workload, idx: int, device="cpu") -> torch.Tensor:
     d = min(m, n)
     a = torch.randn(d, wl.r, generator=_gen("cpu", 5, idx), dtype=torch.float64)
     q, _ = torch.linalg.qr(a)
-    return q.to(wl.torch_dtype).to(device)
+    return q.to(wl.torch_dtype).contiguous().to(device)
 
 
 def planted_gradient(m: int, n: int, r: int, seed: int, gap: float = 4.0,

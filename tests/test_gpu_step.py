@@ -76,7 +76,7 @@ def test_gamma_extremes(gamma):
     if math.isinf(gamma):
         assert all(l == 1.0 for l in lams)
     else:
-        assert lams[2] < 1.0
+        assert any(l < 1.0 for l in lams[1:])      # any growth of ||S|| is cut back
 
 
 def test_zero_gradient_and_zero_columns():
