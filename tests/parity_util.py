@@ -110,3 +110,13 @@ def workload_trajectory(wl: wk.Workload, steps: int, device="cuda", gen_device="
             tr.f.refresh_projection([g.to(device) for g in Gs], None, seed=s, iters=refresh_iters)
         tr.step(Gs)
     return tr
+
+
+def residual_jump(G: torch.Tensor, proj: torch.Tensor, mult: float = 9.0) -> torch.Tensor:
+    """G + mult * (the part of G outside the projection's subspace): a jump that the
+    column factors do not absorb (they scale with 1/||R||, and R is unchanged), so the
+    norm of the scaled residual grows by about 1 + mult and the limiter must act."""
+    G64, P64 = G.to(torch.float64), proj.to(torch.float64).cpu()
+    m, n = G.shape
+    resid = G64 - P64 @ (P64.T @ G64) if m <= n else G64 - (G64 @ P64) @ P64.T
+    return (G64 + mult * resid).to(G.dtype)

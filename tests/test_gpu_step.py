@@ -8,7 +8,7 @@ import torch
 from oracle import fira_oracle as fo
 from paper_2410_01623_b200 import binding as fb
 from paper_2410_01623_b200 import workloads as wk
-from tests.parity_util import Trajectory, rel_err, to_np64, workload_trajectory
+from tests.parity_util import Trajectory, rel_err, residual_jump, to_np64, workload_trajectory
 
 pytestmark = pytest.mark.gpu
 
@@ -32,14 +32,17 @@ def _random_case(shapes, r, dtype, steps, seed, hp=None, spike=None, flags=0):
     hp = hp or fb.make_hparams(lr=1e-2, alpha=0.25, gamma=1.01, flags=flags)
     W0 = [(torch.randn(m, n, generator=g) * 0.02).to(dtype) for (m, n) in shapes]
     tr = Trajectory(shapes, r, dtype, hp, W0)
+    Ps = []
     for i, (m, n) in enumerate(shapes):
         q, _ = torch.linalg.qr(torch.randn(min(m, n), tr.f.ranks[i], generator=g, dtype=torch.float64))
-        tr.f.set_projection(i, q.to(dtype).cuda())
+        Ps.append(q.to(dtype))
+        tr.f.set_projection(i, Ps[i].cuda())
     scales = [torch.exp(torch.randn(n, generator=g)) for (_, n) in shapes]
     for s in range(1, steps + 1):
-        mult = 10.0 if spike and s in spike else 1.0
-        Gs = [(torch.randn(m, n, generator=g) * scales[i][None, :] * mult).to(dtype)
+        Gs = [(torch.randn(m, n, generator=g) * scales[i][None, :]).to(dtype)
               for i, (m, n) in enumerate(shapes)]
+        if spike and s in spike:      # a jump outside the subspace, which the limiter must cut
+            Gs = [residual_jump(G, Ps[i]) for i, G in enumerate(Gs)]
         tr.step(Gs)
     return tr
 
@@ -76,7 +79,7 @@ def test_gamma_extremes(gamma):
     if math.isinf(gamma):
         assert all(l == 1.0 for l in lams)
     else:
-        assert any(l < 1.0 for l in lams[1:])      # any growth of ||S|| is cut back
+        assert lams[2] < 0.5                       # the jump at step 3 is cut back
 
 
 def test_zero_gradient_and_zero_columns():
