@@ -193,6 +193,38 @@ FIRA_API fira_status fira_get_phase_times(fira_ctx* ctx, int32_t* nphases, float
                                           int32_t* steps_recorded);
 FIRA_API const char* fira_phase_name(const fira_ctx* ctx, int32_t phase);
 
+/* One step of ONE matrix without any buffer from the caller beyond the inputs and
+ * outputs themselves.  (The paper has no counterpart: this is a deployment aid.)
+ *
+ * It exists for callers that are not allowed to allocate device memory -- code
+ * running inside another framework's memory pool, a latency-critical loop that must
+ * stay out of the driver's allocator, a process whose memory was budgeted at start
+ * -- and therefore cannot provide the state and scratch buffers of fira_init().  The
+ * intermediates live in a fixed array inside the library image instead:
+ * fira_noalloc_max_scratch_bytes() bytes (8 MiB), held on every GPU that loads the
+ * library until the process exits.  The call allocates nothing.
+ *
+ * desc: the matrix (fp32 or bf16; it always runs on the fp32 CUDA-core kernels).  Its
+ * intermediates must fit the array, roughly max(m,n) * r <= 1,000,000; larger
+ * matrices are rejected with FIRA_ERR_WORKSPACE_TOO_SMALL and a message giving the
+ * sizes.  W_dev (updated in place), G_dev, P_dev (the d x r projection), M_dev and
+ * V_dev (l x r floats, zero before the first step, updated in place) are 16-byte
+ * aligned device pointers; norm_prev_dev points to one float on the device (set it
+ * to -1 before the first step: "no remembered norm yet") and t_dev to one int64 on
+ * the device (0 before the first step); both are updated.  lr < 0 uses hp->lr.
+ * The result equals fira_step()'s for the same matrix on the CUDA-core kernels.
+ *
+ * The first call on a device looks up the array's device address; make that call
+ * before any stream capture starts.  All calls share the one array, which keeps the
+ * previous call's contents (each call rewrites or clears what it reads), so calls
+ * that overlap on the GPU -- from different streams or threads -- race: issue them on
+ * one stream or wait in between. */
+FIRA_API fira_status fira_step_single_noalloc(const fira_hparams* hp, const fira_matrix_desc* desc,
+                                              void* W_dev, const void* G_dev, const void* P_dev,
+                                              float* M_dev, float* V_dev, float* norm_prev_dev,
+                                              int64_t* t_dev, float lr, void* cuda_stream);
+FIRA_API size_t fira_noalloc_max_scratch_bytes(void);
+
 FIRA_API const char* fira_status_string(fira_status s);
 /* Text of the most recent error on this thread ("" if none). */
 FIRA_API const char* fira_last_error(void);

@@ -71,6 +71,10 @@ SIGNATURES = {
     "fira_get_phase_times": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_float),
                                        C.POINTER(C.c_int32)]),
     "fira_phase_name": (C.c_char_p, [C.c_void_p, C.c_int32]),
+    "fira_step_single_noalloc": (C.c_int, [C.POINTER(Hparams), C.POINTER(MatrixDesc), C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_float, C.c_void_p]),
+    "fira_noalloc_max_scratch_bytes": (C.c_size_t, []),
     "fira_status_string": (C.c_char_p, [C.c_int]),
     "fira_last_error": (C.c_char_p, []),
     "fira_destroy": (None, [C.c_void_p]),

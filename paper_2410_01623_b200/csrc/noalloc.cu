@@ -1,0 +1,171 @@
+// fira_step_single_noalloc(): one Fira step of one matrix for callers that cannot
+// allocate device memory.
+//
+// Who needs this.  Code that runs where cudaMalloc is off limits: a plug-in called
+// from inside another framework's memory pool that forbids side allocations, a
+// real-time loop that must not touch the driver's allocator, an environment whose
+// memory budget was fixed at start-up.  Such a caller cannot supply the state and
+// scratch buffers that fira_init() asks for, so the intermediates of the step live
+// in a fixed array that is part of the library image instead.
+//
+// The array costs kNoAllocScratchBytes on every GPU that loads the library, for the
+// life of the process.  All calls share it and it keeps what the previous call left
+// there: two calls that overlap on the GPU (different streams, or different host
+// threads) corrupt each other.  Whatever must start from zero is cleared by each call.
+#include <math.h>
+#include <string.h>
+
+#include <algorithm>
+
+#include "context.cuh"
+
+namespace fira {
+
+namespace {
+
+constexpr size_t kNoAllocScratchBytes = 8u << 20;   // 8 MiB
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+constexpr int kMaxDevices = 64;
+// Device addresses of g_noalloc_scratch, one per device, resolved on first use.  In
+// host code the name g_noalloc_scratch is only a handle for the runtime; the address
+// a kernel may dereference comes from cudaGetSymbolAddress on the current device.
+unsigned char* g_scratch_addr[kMaxDevices] = {};
+
+struct Carve {
+  size_t off_mats, off_status, off_ints, off_sc, off_rt, off_xt, off_k, off_part, total;
+};
+
+Carve carve(int m, int n, int r) {
+  const size_t l = std::max(m, n);
+  const size_t tiles = (size_t)((m + 63) / 64) * ((n + 63) / 64);
+  Carve c;
+  size_t o = 0;
+  c.off_mats = o; o += align_up(sizeof(MatDev));
+  c.off_status = o; o += 256;
+  c.off_ints = o; o += 256;
+  c.off_sc = o; o += align_up(sizeof(MatScalars));
+  c.off_rt = o; o += align_up(l * r * 4);
+  c.off_xt = o; o += align_up(l * r * 4);
+  c.off_k = o; o += align_up(l * 4);
+  c.off_part = o; o += align_up(tiles * 4);
+  c.total = o;
+  return c;
+}
+
+// Moves the two state scalars between the caller's memory and the MatScalars block
+// that the step kernels use.
+__global__ void k_noalloc_load_scalars(MatScalars* sc, const float* norm_prev, const long long* t) {
+  sc->prev_norm = (*norm_prev < 0.f) ? -1.f : *norm_prev;
+  sc->lambda = 1.f; sc->norm_scaled = 0.f; sc->k_min = 0.f; sc->k_max = 0.f; sc->pad = 0.f;
+  sc->t = *t;
+}
+__global__ void k_noalloc_store_scalars(const MatScalars* sc, float* norm_prev, long long* t) {
+  *norm_prev = sc->prev_norm;
+  *t = sc->t;
+}
+
+}  // namespace
+}  // namespace fira
+
+using namespace fira;
+
+extern "C" fira_status fira_step_single_noalloc(const fira_hparams* hp, const fira_matrix_desc* desc,
+                                                void* W_dev, const void* G_dev, const void* P_dev,
+                                                float* M_dev, float* V_dev, float* norm_prev_dev,
+                                                int64_t* t_dev, float lr, void* cuda_stream) {
+  fira_status vs = validate(hp, desc, 1);
+  if (vs != FIRA_OK) return vs;
+  if (!W_dev || !G_dev || !P_dev || !M_dev || !V_dev || !norm_prev_dev || !t_dev) {
+    set_error("null device pointer");
+    return FIRA_ERR_INVALID_ARG;
+  }
+  if (((uintptr_t)W_dev | (uintptr_t)G_dev | (uintptr_t)P_dev | (uintptr_t)M_dev | (uintptr_t)V_dev) & 15) {
+    set_error("W, G, P, M and V must be 16-byte aligned");
+    return FIRA_ERR_INVALID_ARG;
+  }
+  if (!(lr < 0.f) && !isfinite(lr)) { set_error("lr must be finite"); return FIRA_ERR_INVALID_ARG; }
+  const Carve cv = carve(desc->m, desc->n, desc->r);
+  if (cv.total > kNoAllocScratchBytes) {
+    set_error("fira_step_single_noalloc: this matrix needs " + std::to_string(cv.total) +
+              " bytes of scratch, the built-in array holds " + std::to_string(kNoAllocScratchBytes) +
+              " (roughly max(m,n) * r <= 1,000,000)");
+    return FIRA_ERR_WORKSPACE_TOO_SMALL;
+  }
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    set_error(std::string("cudaGetDevice: ") + cudaGetErrorString(e));
+    return FIRA_ERR_CUDA;
+  }
+  if (!g_scratch_addr[dev]) {
+    // once per device, with that device current
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess || !p) {
+      set_error(std::string("cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+      return FIRA_ERR_CUDA;
+    }
+    g_scratch_addr[dev] = static_cast<unsigned char*>(p);
+  }
+  unsigned char* base = g_scratch_addr[dev];
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+
+  MatDev mt;
+  memset(&mt, 0, sizeof(mt));
+  mt.W = W_dev; mt.G = G_dev; mt.P = const_cast<void*>(P_dev); mt.M = M_dev; mt.V = V_dev;
+  mt.sc = reinterpret_cast<MatScalars*>(base + cv.off_sc);
+  mt.Rt = reinterpret_cast<float*>(base + cv.off_rt);
+  mt.Xt = reinterpret_cast<float*>(base + cv.off_xt);
+  mt.kvec = reinterpret_cast<float*>(base + cv.off_k);
+  mt.part = reinterpret_cast<float*>(base + cv.off_part);
+  mt.m = desc->m; mt.n = desc->n; mt.r = desc->r;
+  mt.ld = desc->ld ? desc->ld : desc->n;
+  mt.left = desc->m <= desc->n;
+  mt.bf16 = desc->dtype == FIRA_BF16;
+  mt.l = std::max(desc->m, desc->n); mt.d = std::min(desc->m, desc->n);
+  mt.engine = 0;
+
+  const int ptiles = ((mt.l + 63) / 64) * ((mt.r + 63) / 64);
+  const int wtiles = ((mt.m + 63) / 64) * ((mt.n + 63) / 64);
+  // [list(1)] [proj_start(2)] [row_start(2)] [w_start(2)] [npart(1)]
+  const int ints[8] = {0, 0, ptiles, 0, mt.l, 0, wtiles, wtiles};
+  int* ints_dev = reinterpret_cast<int*>(base + cv.off_ints);
+  unsigned* status_dev = reinterpret_cast<unsigned*>(base + cv.off_status);
+
+#define NA_CUDA(call)                                                          \
+  do {                                                                         \
+    cudaError_t e_ = (call);                                                   \
+    if (e_ != cudaSuccess) {                                                   \
+      set_error(std::string(#call) + ": " + cudaGetErrorString(e_));           \
+      return FIRA_ERR_CUDA;                                                    \
+    }                                                                          \
+  } while (0)
+  // the array still holds the previous call's tables and status: rewrite and clear them
+  NA_CUDA(cudaMemcpyAsync(base + cv.off_mats, &mt, sizeof(mt), cudaMemcpyHostToDevice, st));
+  NA_CUDA(cudaMemcpyAsync(ints_dev, ints, sizeof(ints), cudaMemcpyHostToDevice, st));
+  NA_CUDA(cudaMemsetAsync(status_dev, 0, 256, st));
+  k_noalloc_load_scalars<<<1, 1, 0, st>>>(mt.sc, norm_prev_dev, reinterpret_cast<const long long*>(t_dev));
+
+  SimtPlan pl;
+  pl.mats = reinterpret_cast<const MatDev*>(base + cv.off_mats);
+  pl.list = ints_dev; pl.nlist = 1;
+  pl.proj_tile_start = ints_dev + 1; pl.proj_tiles = ptiles;
+  pl.row_start = ints_dev + 3; pl.rows_total = mt.l;
+  pl.w_tile_start = ints_dev + 5; pl.w_tiles = wtiles;
+  pl.npart = ints_dev + 7;
+  Hyper h;
+  h.beta1 = hp->beta1; h.beta2 = hp->beta2; h.eps = hp->eps;
+  h.lr = lr < 0.f ? hp->lr : lr;
+  h.a_low = hp->alpha;
+  h.a_res = (hp->flags & FIRA_FLAG_ALPHA_LOWRANK_ONLY) ? 1.f : hp->alpha;
+  h.gamma = hp->gamma;
+  PhaseTimer no_timer;
+  launch_simt_step(pl, h, status_dev, st, &no_timer);
+  k_noalloc_store_scalars<<<1, 1, 0, st>>>(mt.sc, norm_prev_dev, reinterpret_cast<long long*>(t_dev));
+  NA_CUDA(cudaGetLastError());
+#undef NA_CUDA
+  return FIRA_OK;
+}
+
+extern "C" size_t fira_noalloc_max_scratch_bytes(void) { return kNoAllocScratchBytes; }
