@@ -43,7 +43,10 @@ constexpr int CHUNK_BYTES = 64 * BK * 2;         // one 64 x 64 box: 8 KiB
 constexpr int EPI_WARPS = 8;
 constexpr int TC_THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
-constexpr size_t TC_SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + 256;
+constexpr int STG_PITCH = 32;                    // floats per staged row (16-byte slots XOR-swizzled)
+constexpr int STG_WARP_FLOATS = 32 * STG_PITCH;  // one warp's 32 x 32 fp32 staging tile
+constexpr size_t TC_SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 256 + (size_t)EPI_WARPS * STG_WARP_FLOATS * 4;
+static_assert(TC_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr int GSQ_ROWS = 128;     // rows per partial sum of G^2 (left orientation)
 
 struct TcMaps {
@@ -68,9 +71,11 @@ struct SharedCtl {
 };
 
 // Common prologue: carve shared memory, init barriers, allocate TMEM.
-__device__ __forceinline__ void tc_prologue(unsigned char* smem_raw, unsigned char*& tiles, SharedCtl*& ctl) {
-  const uintptr_t base = (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023;
-  tiles = reinterpret_cast<unsigned char*>(base);
+// Returns false (all threads alike) if the dynamic shared memory does not start on a
+// 1024-byte boundary, which the 128-byte swizzle of the TMA tiles needs.
+__device__ __forceinline__ bool tc_prologue(unsigned char* smem_raw, unsigned char*& tiles, SharedCtl*& ctl) {
+  tiles = smem_raw;
+  if (ptx::smem_u32(smem_raw) & 1023u) return false;
   ctl = reinterpret_cast<SharedCtl*>(tiles + (size_t)STAGES * STAGE_BYTES);
   const int warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) {
@@ -92,6 +97,7 @@ __device__ __forceinline__ void tc_prologue(unsigned char* smem_raw, unsigned ch
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
+  return true;
 }
 
 __device__ __forceinline__ void tc_epilogue_teardown(SharedCtl* ctl, unsigned* status) {
@@ -132,6 +138,8 @@ __device__ __forceinline__ void unpack8_bf16(const uint4& u, float (&v)[8]) {
   }
 }
 
+#include "tc_epilogue.cuh"
+
 // ============================================================================ projection product
 // Rt[l][j] = sum_d G(d,l) Pi[d][j].  Tile: 128 l x BN r.  A = G: left orientation
 // MN-major (G is [d][l], l contiguous: two 64 x 64 boxes), right orientation K-major
@@ -140,10 +148,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 k_tc_project(const MatDev* __restrict__ mats, const TcMaps* __restrict__ maps, const int* __restrict__ list,
              int nlist, const int* __restrict__ tile_start, int total_tiles, Hyper hp,
              unsigned* __restrict__ status) {
-  extern __shared__ unsigned char smem_raw[];
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* tiles;
   SharedCtl* ctl;
-  tc_prologue(smem_raw, tiles, ctl);
+  if (!tc_prologue(smem_raw, tiles, ctl)) {
+    if (threadIdx.x == 0) atomicOr(status, DEV_STATUS_TIMEOUT);
+    return;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &ctl->abort_flag;
   const uint32_t tiles_u32 = ptx::smem_u32(tiles);
@@ -220,69 +231,52 @@ k_tc_project(const MatDev* __restrict__ mats, const TcMaps* __restrict__ maps, c
     const int ew = warp - 2;
     const int quarter = warp & 3;       // TMEM lanes 32*quarter .. +31 are this warp's
     const int half = ew >> 2;           // which half of the tile's columns
+    float* stg = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(ctl) + 256) + ew * STG_WARP_FLOATS;
     int buf = 0; uint32_t bphase = 0;
     const uint32_t tmem = ctl->tmem_base;
+    ProjTile cur = proj_tile(mats, list, nlist, tile_start, blockIdx.x, total_tiles, quarter, half, lane);
+    MVHalf bufA, bufB;
+    if (cur.valid) load_mv(bufA, cur, 0);
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-      const int p = find_matrix(tile_start, nlist, t);
-      const MatDev& mt = mats[list[p]];
-      const int r = mt.r, L = mt.l;
-      const int bn = tile_bn(r), nrt = r / bn;
-      const int local = t - tile_start[p];
-      const int rt = local % nrt;
-      const int l = (local / nrt) * BM + quarter * 32 + lane;
-      const int cols_half = bn / 2;                 // multiple of 32
-      const int cbase = half * cols_half;
-      const float bias = mt.sc->pad;
-      const bool row_ok = l < L;
+      const ProjTile nxt = proj_tile(mats, list, nlist, tile_start, t + gridDim.x, total_tiles, quarter, half, lane);
       if (!ptx::mbar_wait(ptx::smem_u32(&ctl->tmem_full[buf]), bphase, abort_flag)) break;
       ptx::tc_fence_after();
-      float nn = 0.f, rn = 0.f;
-      const long long rowoff = (long long)l * r + rt * bn + cbase;
-      for (int c = 0; c < cols_half; c += 32) {
-        uint32_t rr[32];
-        ptx::tmem_ld_32x32b_x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX + cbase + c, rr);
-        ptx::tmem_ld_wait();
-        if (row_ok) {
-          float* Mp = mt.M + rowoff + c;
-          float* Vp = mt.V + rowoff + c;
-          __nv_bfloat16* Np = mt.Nb + rowoff + c;
-          __nv_bfloat16* Rp = mt.Rb + rowoff + c;
+      float nn[8] = {}, rn[8] = {};
+      const uint32_t tcol = tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX + half * cur.nch * 32;
+      for (int c = 0; c < cur.nch; ++c) {
+        stage_rows(stg, lane, tcol + 32 * c);
+        if (c == cur.nch - 1) {           // the accumulator has been read out completely
+          ptx::tc_fence_before();
+          if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[buf]));
+        }
+        load_mv(bufB, cur, 2 * c + 1);
+        adam_half(bufA, cur, 2 * c, stg, lane, hp, nn, rn);
+        if (c + 1 < cur.nch) load_mv(bufA, cur, 2 * c + 2);
+        else if (nxt.valid) load_mv(bufA, nxt, 0);
+        adam_half(bufB, cur, 2 * c + 1, stg, lane, hp, nn, rn);
+        __syncwarp();                     // the staging tile is free again
+      }
+      // row sums: the eight lanes of a row hold its partial sums
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const float4 m0 = *reinterpret_cast<const float4*>(Mp + 8 * q);
-            const float4 m1 = *reinterpret_cast<const float4*>(Mp + 8 * q + 4);
-            const float4 v0 = *reinterpret_cast<const float4*>(Vp + 8 * q);
-            const float4 v1 = *reinterpret_cast<const float4*>(Vp + 8 * q + 4);
-            float mo[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
-            float vo[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-            float rv[8], nv[8];
+      for (int i = 0; i < 8; ++i) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              rv[e] = __uint_as_float(rr[8 * q + e]);
-              mo[e] = hp.beta1 * mo[e] + (1.f - hp.beta1) * rv[e];
-              vo[e] = hp.beta2 * vo[e] + (1.f - hp.beta2) * rv[e] * rv[e];
-              nv[e] = bias * mo[e] / (sqrtf(vo[e]) + hp.eps);
-              nn = fmaf(nv[e], nv[e], nn);
-              rn = fmaf(rv[e], rv[e], rn);
-            }
-            *reinterpret_cast<float4*>(Mp + 8 * q) = make_float4(mo[0], mo[1], mo[2], mo[3]);
-            *reinterpret_cast<float4*>(Mp + 8 * q + 4) = make_float4(mo[4], mo[5], mo[6], mo[7]);
-            *reinterpret_cast<float4*>(Vp + 8 * q) = make_float4(vo[0], vo[1], vo[2], vo[3]);
-            *reinterpret_cast<float4*>(Vp + 8 * q + 4) = make_float4(vo[4], vo[5], vo[6], vo[7]);
-            *reinterpret_cast<uint4*>(Np + 8 * q) = pack8_bf16(nv);
-            *reinterpret_cast<uint4*>(Rp + 8 * q) = pack8_bf16(rv);
+        for (int o = 1; o < 8; o <<= 1) {
+          nn[i] += __shfl_xor_sync(0xffffffffu, nn[i], o);
+          rn[i] += __shfl_xor_sync(0xffffffffu, rn[i], o);
+        }
+      }
+      if ((lane & 7) == 0) {
+        // colpart[part][l] = partial ||N_l||^2, colpart[nparts + part][l] = partial ||R_l||^2
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int l = cur.l0 + 4 * i;
+          if (l < cur.L) {
+            cur.colpart[(long long)cur.part * cur.L + l] = nn[i];
+            cur.colpart[(long long)(cur.nparts + cur.part) * cur.L + l] = rn[i];
           }
         }
       }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[buf]));
-      if (row_ok) {
-        // colpart[0][part][l] = partial ||N_l||^2, colpart[1][part][l] = partial ||R_l||^2
-        const int nparts = 2 * nrt, part = rt * 2 + half;
-        mt.colpart[(long long)part * L + l] = nn;
-        mt.colpart[(long long)(nparts + part) * L + l] = rn;
-      }
+      cur = nxt;
       if (++buf == 2) { buf = 0; bphase ^= 1u; }
     }
   }
@@ -299,10 +293,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 k_tc_back_project(const MatDev* __restrict__ mats, const TcMaps* __restrict__ maps,
                   const int* __restrict__ list, int nlist, const int* __restrict__ tile_start,
                   int total_tiles, Hyper hp, unsigned* __restrict__ status) {
-  extern __shared__ unsigned char smem_raw[];
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* tiles;
   SharedCtl* ctl;
-  tc_prologue(smem_raw, tiles, ctl);
+  if (!tc_prologue(smem_raw, tiles, ctl)) {
+    if (threadIdx.x == 0) atomicOr(status, DEV_STATUS_TIMEOUT);
+    return;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &ctl->abort_flag;
   const uint32_t tiles_u32 = ptx::smem_u32(tiles);
@@ -363,59 +360,36 @@ k_tc_back_project(const MatDev* __restrict__ mats, const TcMaps* __restrict__ ma
   } else {
     const int ew = warp - 2;
     const int quarter = warp & 3;
-    const int half = ew >> 2;
     int buf = 0; uint32_t bphase = 0;
     const uint32_t tmem = ctl->tmem_base;
+    float* stg = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(ctl) + 256) + ew * STG_WARP_FLOATS;
+    const int half = ew >> 2;           // which half of the tile's columns
+    BackTile cur = back_tile_info(mats, list, nlist, tile_start, blockIdx.x, total_tiles, quarter, half, lane, hp);
+    GWChunk bufA, bufB;
+    load_gw(bufA, cur, 0);
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-      const int p = find_matrix(tile_start, nlist, t);
-      const MatDev& mt = mats[list[p]];
-      const int n = mt.n, m = mt.m, left = mt.left;
-      const long long ld = mt.ld;
-      const int nct = (n + BN_MAX - 1) / BN_MAX;
-      const int local = t - tile_start[p];
-      const int i = (local / nct) * BM + quarter * 32 + lane;
-      const int jbase = (local % nct) * BN_MAX + half * (BN_MAX / 2);
-      const bool row_ok = i < m;
-      const float cres = hp.a_res * mt.sc->lambda;
-      const float krow = (!left && row_ok) ? mt.kvec[i] : 0.f;
-      const __nv_bfloat16* Gp = static_cast<const __nv_bfloat16*>(mt.G) + (long long)i * ld;
-      __nv_bfloat16* Wp = static_cast<__nv_bfloat16*>(mt.W) + (long long)i * ld;
+      const BackTile nxt = back_tile_info(mats, list, nlist, tile_start, t + gridDim.x, total_tiles, quarter,
+                                          half, lane, hp);
       if (!ptx::mbar_wait(ptx::smem_u32(&ctl->tmem_full[buf]), bphase, abort_flag)) break;
       ptx::tc_fence_after();
-      for (int c = 0; c < BN_MAX / 2; c += 32) {
-        uint32_t dd[32];
-        ptx::tmem_ld_32x32b_x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX + half * (BN_MAX / 2) + c, dd);
-        ptx::tmem_ld_wait();
-        if (row_ok) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int j = jbase + c + 8 * q;
-            if (j < n) {            // n is a multiple of 8: the 8 columns are all inside
-              const uint4 gu = *reinterpret_cast<const uint4*>(Gp + j);
-              const uint4 wu = *reinterpret_cast<const uint4*>(Wp + j);
-              float g[8], w[8], kf[8];
-              unpack8_bf16(gu, g);
-              unpack8_bf16(wu, w);
-              if (left) {
-                const float4 k0 = *reinterpret_cast<const float4*>(mt.kvec + j);
-                const float4 k1 = *reinterpret_cast<const float4*>(mt.kvec + j + 4);
-                kf[0] = k0.x; kf[1] = k0.y; kf[2] = k0.z; kf[3] = k0.w;
-                kf[4] = k1.x; kf[5] = k1.y; kf[6] = k1.z; kf[7] = k1.w;
-              } else {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) kf[e] = krow;
-              }
-#pragma unroll
-              for (int e = 0; e < 8; ++e)
-                w[e] = w[e] - hp.lr * (__uint_as_float(dd[8 * q + e]) + cres * kf[e] * g[e]);
-              *reinterpret_cast<uint4*>(Wp + j) = pack8_bf16(w);
-            }
-          }
+      const uint32_t tcol = tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX + half * (BN_MAX / 2);
+      constexpr int NCH = BN_MAX / 64;    // chunks of 32 columns in this warp's half
+#pragma unroll 1
+      for (int c = 0; c < NCH; c += 2) {
+        stage_rows(stg, lane, tcol + 32 * c);
+        load_gw(bufB, cur, c + 1);
+        update_chunk(bufA, cur, c, stg, lane, hp.lr);
+        __syncwarp();
+        stage_rows(stg, lane, tcol + 32 * (c + 1));
+        if (c + 2 == NCH) {               // the accumulator has been read out completely
+          ptx::tc_fence_before();
+          if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[buf]));
         }
+        if (c + 2 < NCH) load_gw(bufA, cur, c + 2); else load_gw(bufA, nxt, 0);
+        update_chunk(bufB, cur, c + 1, stg, lane, hp.lr);
+        __syncwarp();
       }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[buf]));
+      cur = nxt;
       if (++buf == 2) { buf = 0; bphase ^= 1u; }
     }
   }
