@@ -70,7 +70,7 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
   L.off_status = wo; wo += 256;
   L.ints_count = 16 * (size_t)(count + 1);
   L.off_ints = wo; wo += align_up(L.ints_count * sizeof(int));
-  L.off_tcmaps = wo; wo += tc_maps_bytes(count);
+  L.off_tcmaps = wo; wo += tc_tables_bytes(hp, descs, count);
   L.off_work = wo;
   size_t w = 0;
   size_t refresh_max = 0;

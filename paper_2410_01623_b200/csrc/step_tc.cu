@@ -54,6 +54,14 @@ struct TcMaps {
   CUtensorMap g1b;   // Pi [d][r], boxes of 64 r x 64 d
   CUtensorMap g2a;   // back-projection A operand (Pi when left, X when right), box 64 x 128
   CUtensorMap g2b;   // back-projection B operand (X when left, Pi when right), box 64 x 256
+  // maps used only to prefetch epilogue operands into L2 ahead of the epilogue
+  CUtensorMap pg;    // G [m][n] bf16, box 64 x 128
+  CUtensorMap pw;    // W [m][n] bf16, box 64 x 128
+  CUtensorMap pm;    // M [l][r] fp32, box 64 x 128
+  CUtensorMap pv;    // V [l][r] fp32, box 64 x 128
+  // boxes of the back-projection epilogue (64-byte swizzle)
+  CUtensorMap eg;    // G [m][n] bf16, box 32 x 128
+  CUtensorMap ew;    // W [m][n] bf16, box 32 x 128 (loaded and stored)
 };
 static_assert(sizeof(TcMaps) % 64 == 0, "tensor maps must stay 64-byte aligned");
 
@@ -173,6 +181,11 @@ k_tc_project(const MatDev* __restrict__ mats, const TcMaps* __restrict__ maps, c
         const int l0 = (local / nrt) * BM, r0 = (local % nrt) * bn;
         const int nkb = (d + BK - 1) / BK;
         const uint32_t bytes = A_STAGE_BYTES + bn * BK * 2;
+        // the epilogue of this tile reads M and V; start moving them from HBM to L2 now
+        for (int c = 0; c < bn / 64; ++c) {
+          ptx::tma_prefetch_l2_2d(&mp->pm, r0 + 64 * c, l0);
+          ptx::tma_prefetch_l2_2d(&mp->pv, r0 + 64 * c, l0);
+        }
         for (int kb = 0; kb < nkb; ++kb) {
           if (!ptx::mbar_wait(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
@@ -283,118 +296,7 @@ k_tc_project(const MatDev* __restrict__ mats, const TcMaps* __restrict__ maps, c
   tc_epilogue_teardown(ctl, status);
 }
 
-// ============================================================================ back-projection product
-// D[i][j] = sum_q A(i,q) B(j,q) over the rank index q, both operands K-major:
-// left: A = Pi [d][r] (i = row of W), B = X [l][r] (j = column of W);
-// right: A = X [l][r], B = Pi [d][r].  Tile 128 x 256 of W.
-// Epilogue: W[i][j] -= lr (D + a_res lambda k G[i][j]), k taken per column (left) or
-// per row (right).
-__global__ void __launch_bounds__(TC_THREADS, 1)
-k_tc_back_project(const MatDev* __restrict__ mats, const TcMaps* __restrict__ maps,
-                  const int* __restrict__ list, int nlist, const int* __restrict__ tile_start,
-                  int total_tiles, Hyper hp, unsigned* __restrict__ status) {
-  extern __shared__ __align__(1024) unsigned char smem_raw[];
-  unsigned char* tiles;
-  SharedCtl* ctl;
-  if (!tc_prologue(smem_raw, tiles, ctl)) {
-    if (threadIdx.x == 0) atomicOr(status, DEV_STATUS_TIMEOUT);
-    return;
-  }
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  volatile int* abort_flag = &ctl->abort_flag;
-  const uint32_t tiles_u32 = ptx::smem_u32(tiles);
-
-  if (warp == 0) {
-    if (lane == 0) {
-      int stage = 0; uint32_t phase = 0; int issued = 0; bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const int p = find_matrix(tile_start, nlist, t);
-        const MatDev& mt = mats[list[p]];
-        const TcMaps* mp = &maps[p];
-        const int nct = (mt.n + BN_MAX - 1) / BN_MAX;
-        const int local = t - tile_start[p];
-        const int i0 = (local / nct) * BM, j0 = (local % nct) * BN_MAX;
-        const int nkb = mt.r / BK;
-        for (int kb = 0; kb < nkb; ++kb) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
-          const uint32_t sa = tiles_u32 + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
-          ptx::mbar_expect_tx(fb, STAGE_BYTES);
-          ptx::tma_load_2d(sa, &mp->g2a, fb, kb * BK, i0);
-          ptx::tma_load_2d(sb, &mp->g2b, fb, kb * BK, j0);
-          issued = 1;
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-        }
-      }
-      if (!ok) drain_stage_waits(ctl, stage, phase, issued);
-    }
-  } else if (warp == 1) {
-    if (lane == 0) {
-      int stage = 0; uint32_t phase = 0; int buf = 0; uint32_t bphase = 0; bool ok = true;
-      const uint32_t tmem = ctl->tmem_base;
-      const uint32_t idesc = ptx::make_idesc_bf16(BM, BN_MAX, 0, 0);
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const int p = find_matrix(tile_start, nlist, t);
-        const int nkb = mats[list[p]].r / BK;
-        if (!ptx::mbar_wait(ptx::smem_u32(&ctl->tmem_empty[buf]), bphase ^ 1u, abort_flag)) { ok = false; break; }
-        ptx::tc_fence_after();
-        const uint32_t dcol = tmem + buf * BN_MAX;
-        for (int kb = 0; kb < nkb; ++kb) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
-          ptx::tc_fence_after();
-          const uint32_t sa = tiles_u32 + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
-#pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            const uint64_t ad = ptx::make_smem_desc(sa + k * 32, 0, 1024);
-            const uint64_t bd = ptx::make_smem_desc(sb + k * 32, 0, 1024);
-            ptx::umma_bf16(dcol, ad, bd, idesc, (kb | k) ? 1u : 0u);
-          }
-          ptx::umma_commit(ptx::smem_u32(&ctl->empty[stage]));
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-        }
-        if (!ok) break;
-        ptx::umma_commit(ptx::smem_u32(&ctl->tmem_full[buf]));
-        if (++buf == 2) { buf = 0; bphase ^= 1u; }
-      }
-    }
-  } else {
-    const int ew = warp - 2;
-    const int quarter = warp & 3;
-    int buf = 0; uint32_t bphase = 0;
-    const uint32_t tmem = ctl->tmem_base;
-    float* stg = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(ctl) + 256) + ew * STG_WARP_FLOATS;
-    const int half = ew >> 2;           // which half of the tile's columns
-    BackTile cur = back_tile_info(mats, list, nlist, tile_start, blockIdx.x, total_tiles, quarter, half, lane, hp);
-    GWChunk bufA, bufB;
-    load_gw(bufA, cur, 0);
-    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-      const BackTile nxt = back_tile_info(mats, list, nlist, tile_start, t + gridDim.x, total_tiles, quarter,
-                                          half, lane, hp);
-      if (!ptx::mbar_wait(ptx::smem_u32(&ctl->tmem_full[buf]), bphase, abort_flag)) break;
-      ptx::tc_fence_after();
-      const uint32_t tcol = tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX + half * (BN_MAX / 2);
-      constexpr int NCH = BN_MAX / 64;    // chunks of 32 columns in this warp's half
-#pragma unroll 1
-      for (int c = 0; c < NCH; c += 2) {
-        stage_rows(stg, lane, tcol + 32 * c);
-        load_gw(bufB, cur, c + 1);
-        update_chunk(bufA, cur, c, stg, lane, hp.lr);
-        __syncwarp();
-        stage_rows(stg, lane, tcol + 32 * (c + 1));
-        if (c + 2 == NCH) {               // the accumulator has been read out completely
-          ptx::tc_fence_before();
-          if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[buf]));
-        }
-        if (c + 2 < NCH) load_gw(bufA, cur, c + 2); else load_gw(bufA, nxt, 0);
-        update_chunk(bufB, cur, c + 1, stg, lane, hp.lr);
-        __syncwarp();
-      }
-      cur = nxt;
-      if (++buf == 2) { buf = 0; bphase ^= 1u; }
-    }
-  }
-  tc_epilogue_teardown(ctl, status);
-}
+#include "tc_back_project.cuh"
 
 // ============================================================================ small kernels
 __global__ void k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist, Hyper hp) {
@@ -487,14 +389,17 @@ k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, i
 // X = a_low N - a_res lambda k_l R in bf16, one warp per l.
 __global__ void __launch_bounds__(256)
 k_tc_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
-            const int* __restrict__ row_start, int rows_total, float a_low, float a_res) {
+            const int* __restrict__ row_start, int rows_total, float a_low, float a_res,
+            float* __restrict__ fast) {
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (row >= rows_total) return;
   const int p = find_matrix(row_start, nlist, row);
   const MatDev& mt = mats[list[p]];
   const int l = row - row_start[p];
-  const float c = a_res * mt.sc->lambda * mt.kvec[l];
+  const float lambda = mt.sc->lambda;
+  if (l == 0 && lane == 0) fast[2 * p + 1] = lambda;   // read by the back-projection epilogue
+  const float c = a_res * lambda * mt.kvec[l];
   const long long base = (long long)l * mt.r;
   for (int j = lane * 8; j < mt.r; j += 256) {
     const uint4 nu = *reinterpret_cast<const uint4*>(mt.Nb + base + j);
@@ -528,15 +433,20 @@ EncodeTiledFn get_encode_fn() {
 
 // bf16 row-major matrix [rows][cols] with leading dimension ld; box = box_c x box_r.
 bool encode_map(CUtensorMap* out, const void* base, long long rows, long long cols, long long ld,
-                int box_c, int box_r) {
+                int box_c, int box_r, int mode = 0) {
+  // mode 0: bf16, 128-byte swizzle; 1: fp32, no swizzle (L2 prefetch only); 2: bf16, 64-byte swizzle
+  const bool fp32 = mode == 1;
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) { set_error("cuTensorMapEncodeTiled is not available"); return false; }
   const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  const cuuint64_t gstr[1] = {(cuuint64_t)ld * 2};
+  const cuuint64_t gstr[1] = {(cuuint64_t)ld * (fp32 ? 4 : 2)};
   const cuuint32_t box[2] = {(cuuint32_t)box_c, (cuuint32_t)box_r};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+  // fp32 maps are only used for L2 prefetches (no shared-memory image, so no swizzle)
+  const CUresult r = fn(out, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                        const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        mode == 1 ? CU_TENSOR_MAP_SWIZZLE_NONE
+                                  : (mode == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B),
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with code " + std::to_string((int)r)); return false; }
   return true;
@@ -557,6 +467,8 @@ struct TcPlan {
   const int* col_start = nullptr; int col_blocks = 0;
   const int* row_start = nullptr; int rows_total = 0;
   const int* npart = nullptr;
+  BackTileDesc* td2_dev = nullptr;   // per-tile records of the back-projection
+  float* fast_dev = nullptr;         // per matrix of the list: {bias factor, lambda}
   int num_sms = 148;
   bool attrs_set = false;
 };
@@ -578,12 +490,28 @@ size_t tc_gsq_floats(const fira_matrix_desc& d) {
 
 size_t tc_part_floats(const fira_matrix_desc& d) { return ((size_t)std::max(d.m, d.n) + 255) / 256; }
 
-size_t tc_maps_bytes(int count) { return align_up(sizeof(TcMaps) * (size_t)count); }
+static size_t back_tiles(const fira_matrix_desc& d) {
+  return (size_t)((d.m + BM - 1) / BM) * ((d.n + BN_MAX - 1) / BN_MAX);
+}
+
+// Device tables of this engine: tensor maps, fast scalars, back-projection tile records.
+size_t tc_tables_bytes(const fira_hparams& hp, const fira_matrix_desc* descs, int count) {
+  size_t ntc = 0, tiles = 0;
+  for (int i = 0; i < count; ++i)
+    if (engine_for(hp, descs[i]) == 1) { ++ntc; tiles += back_tiles(descs[i]); }
+  return align_up(sizeof(TcMaps) * ntc) + align_up(2 * sizeof(float) * ntc) + align_up(sizeof(BackTileDesc) * tiles);
+}
 
 static bool encode_matrix_maps(const MatDev& mt, TcMaps& mp, bool only_g) {
   // G is [m][n]: left -> boxes of 64 l x 64 d rows; right -> box of 64 d x 128 l rows
   if (!encode_map(&mp.g1a, mt.G, mt.m, mt.n, mt.ld, 64, mt.left ? 64 : 128)) return false;
+  if (!encode_map(&mp.pg, mt.G, mt.m, mt.n, mt.ld, 64, 128)) return false;
+  if (!encode_map(&mp.pw, mt.W, mt.m, mt.n, mt.ld, 64, 128)) return false;
+  if (!encode_map(&mp.eg, mt.G, mt.m, mt.n, mt.ld, K2_ECOLS, 128, 2)) return false;
+  if (!encode_map(&mp.ew, mt.W, mt.m, mt.n, mt.ld, K2_ECOLS, 128, 2)) return false;
   if (only_g) return true;
+  if (!encode_map(&mp.pm, mt.M, mt.l, mt.r, mt.r, 64, 128, 1)) return false;
+  if (!encode_map(&mp.pv, mt.V, mt.l, mt.r, mt.r, 64, 128, 1)) return false;
   if (!encode_map(&mp.g1b, mt.P, mt.d, mt.r, mt.r, 64, 64)) return false;
   const void* a2 = mt.left ? (const void*)mt.P : (const void*)mt.Xb;
   const void* b2 = mt.left ? (const void*)mt.Xb : (const void*)mt.P;
@@ -627,11 +555,35 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
   pl->row_start = c->ints_dev + o_rs; pl->rows_total = rs.back();
   pl->npart = c->ints_dev + o_np;
   pl->maps.resize(lst.size());
-  pl->maps_dev = reinterpret_cast<TcMaps*>(c->tc_maps_dev);
+  char* tab = c->tc_maps_dev;
+  pl->maps_dev = reinterpret_cast<TcMaps*>(tab); tab += align_up(sizeof(TcMaps) * lst.size());
+  pl->fast_dev = reinterpret_cast<float*>(tab); tab += align_up(2 * sizeof(float) * lst.size());
+  pl->td2_dev = reinterpret_cast<BackTileDesc*>(tab);
+  {
+    std::vector<BackTileDesc> td;
+    td.reserve(pl->k2_tiles);
+    for (size_t q = 0; q < lst.size(); ++q) {
+      const MatDev& mt = c->mats[lst[q]];
+      const int nrt = (mt.m + BM - 1) / BM, nct = (mt.n + BN_MAX - 1) / BN_MAX;
+      for (int a = 0; a < nrt; ++a)
+        for (int b = 0; b < nct; ++b) {
+          BackTileDesc d;
+          d.kvec = mt.kvec; d.slot = (int)q; d.i0 = a * BM; d.j0 = b * BN_MAX; d.nkb = mt.r / BK;
+          d.n = mt.n; d.m_left = mt.m | (mt.left ? (int)0x80000000 : 0);
+          td.push_back(d);
+        }
+    }
+    if ((int)td.size() != pl->k2_tiles) { set_error("internal: tile count mismatch"); return FIRA_ERR_INVALID_ARG; }
+    cudaError_t e = cudaMemcpyAsync(pl->td2_dev, td.data(), sizeof(BackTileDesc) * td.size(),
+                                    cudaMemcpyHostToDevice, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // td dies at the end of this block
+    if (e != cudaSuccess) { set_error(std::string("tile table upload: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
+  }
   // maps that do not depend on W / G; the G map is encoded when the pointers are known
   for (size_t q = 0; q < lst.size(); ++q) {
     MatDev mt = c->mats[lst[q]];
-    mt.G = mt.P;   // placeholder address with valid alignment; replaced in tc_update_pointers
+    mt.G = mt.P;   // placeholder addresses with valid alignment; replaced in tc_update_pointers
+    mt.W = mt.P;
     if (!encode_matrix_maps(mt, pl->maps[q], false)) return FIRA_ERR_CUDA;
   }
   return FIRA_OK;
@@ -666,7 +618,7 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   cudaStream_t st = c->stream;
   if (!pl->attrs_set) {
     cudaError_t e1 = cudaFuncSetAttribute(k_tc_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES);
-    cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES);
+    cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES);
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
       set_error(std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
       return -1;
@@ -687,10 +639,10 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   k_finalize<<<pl->nlist, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->npart, hp, c->status_dev);
   tm->mark(st);
   k_tc_form_x<<<(pl->rows_total + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start,
-                                                        pl->rows_total, hp.a_low, hp.a_res);
+                                                        pl->rows_total, hp.a_low, hp.a_res, pl->fast_dev);
   tm->mark(st);
-  k_tc_back_project<<<std::min(pl->k2_tiles, pl->num_sms), TC_THREADS, TC_SMEM_BYTES, st>>>(
-      mats, pl->maps_dev, pl->list, pl->nlist, pl->k2_start, pl->k2_tiles, hp, c->status_dev);
+  k_tc_back_project<<<std::min(pl->k2_tiles, pl->num_sms), K2_THREADS, K2_SMEM_BYTES, st>>>(
+      pl->maps_dev, pl->td2_dev, pl->k2_tiles, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);
   return 7;
 }

@@ -16,8 +16,8 @@ bool tc_supported(const fira_matrix_desc& d);
 size_t tc_colpart_floats(const fira_matrix_desc& d);
 size_t tc_part_floats(const fira_matrix_desc& d);
 size_t tc_gsq_floats(const fira_matrix_desc& d);
-// Bytes of the device-resident tensor-map table for `count` matrices.
-size_t tc_maps_bytes(int count);
+// Bytes of this engine's device-resident tables (tensor maps, tile records) for a matrix list.
+size_t tc_tables_bytes(const fira_hparams& hp, const fira_matrix_desc* descs, int count);
 // Appends this engine's schedule arrays to `ints` (host image of the device int
 // block) and records where they are.
 fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints);

@@ -119,90 +119,3 @@ __device__ __forceinline__ void adam_half(const MVHalf& b, const ProjTile& pt, i
     }
   }
 }
-
-// ---------------------------------------------------------------------------- back-projection epilogue
-// Coalesced layout of a 32-column bf16 chunk: lane -> row 8 i + lane / 4 (i = 0..3),
-// columns 8 (lane % 4) .. + 7: four lanes cover one 64-byte row segment of G or W.
-struct BackTile {
-  const __nv_bfloat16* G;   // at (row of i = 0, first column of this lane in chunk 0)
-  __nv_bfloat16* W;
-  const float* kvec;
-  long long ld;
-  float cres;               // a_res * lambda
-  float krow[4];            // k of the four rows when the factors are per row
-  int row0;                 // row of W of i = 0
-  int m, n, j0, left;       // j0: this lane's first column in chunk 0
-  bool valid;
-};
-
-__device__ __forceinline__ BackTile back_tile_info(const MatDev* __restrict__ mats, const int* __restrict__ list,
-                                                   int nlist, const int* __restrict__ tile_start, int t,
-                                                   int total_tiles, int quarter, int half, int lane,
-                                                   const Hyper& hp) {
-  BackTile bt;
-  bt.valid = t < total_tiles;
-  if (!bt.valid) { bt.m = 0; bt.n = 0; bt.row0 = 0; bt.j0 = 0; return bt; }
-  const int p = find_matrix(tile_start, nlist, t);
-  const MatDev& mt = mats[list[p]];
-  const int nct = (mt.n + BN_MAX - 1) / BN_MAX;
-  const int local = t - tile_start[p];
-  bt.m = mt.m; bt.n = mt.n; bt.left = mt.left; bt.ld = mt.ld;
-  bt.row0 = (local / nct) * BM + quarter * 32 + (lane >> 2);
-  bt.j0 = (local % nct) * BN_MAX + half * (BN_MAX / 2) + 8 * (lane & 3);
-  bt.cres = hp.a_res * mt.sc->lambda;
-  bt.kvec = mt.kvec;
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-    bt.krow[i] = (!mt.left && bt.row0 + 8 * i < mt.m) ? mt.kvec[bt.row0 + 8 * i] : 0.f;
-  const long long off = (long long)bt.row0 * mt.ld + bt.j0;
-  bt.G = static_cast<const __nv_bfloat16*>(mt.G) + off;
-  bt.W = static_cast<__nv_bfloat16*>(mt.W) + off;
-  return bt;
-}
-
-struct GWChunk { uint4 g[4]; uint4 w[4]; float4 k0, k1; };
-
-// n is a multiple of 8, so a group of 8 columns is inside or outside as a whole.
-__device__ __forceinline__ void load_gw(GWChunk& b, const BackTile& bt, int chunk) {
-  if (!bt.valid || bt.j0 + 32 * chunk >= bt.n) return;
-  if (bt.left) {
-    b.k0 = *reinterpret_cast<const float4*>(bt.kvec + bt.j0 + 32 * chunk);
-    b.k1 = *reinterpret_cast<const float4*>(bt.kvec + bt.j0 + 32 * chunk + 4);
-  }
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    if (bt.row0 + 8 * i < bt.m) {
-      const long long off = (long long)(8 * i) * bt.ld + 32 * chunk;
-      b.g[i] = *reinterpret_cast<const uint4*>(bt.G + off);
-      b.w[i] = *reinterpret_cast<const uint4*>(bt.W + off);
-    }
-  }
-}
-
-// W[i][j] -= lr (D[i][j] + a_res lambda k G[i][j]) on one 32-column chunk of the warp's
-// 32 rows; D comes from the staging tile.
-__device__ __forceinline__ void update_chunk(const GWChunk& b, const BackTile& bt, int chunk, const float* stg,
-                                             int lane, float lr) {
-  const int j = bt.j0 + 32 * chunk;
-  if (j >= bt.n) return;
-  const float kcol[8] = {b.k0.x, b.k0.y, b.k0.z, b.k0.w, b.k1.x, b.k1.y, b.k1.z, b.k1.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    if (bt.row0 + 8 * i < bt.m) {
-      const int srow = 8 * i + (lane >> 2);
-      const float* drow = stg + srow * STG_PITCH;
-      const float4 d0 = *reinterpret_cast<const float4*>(drow + 4 * ((2 * (lane & 3)) ^ (srow & 7)));
-      const float4 d1 = *reinterpret_cast<const float4*>(drow + 4 * ((2 * (lane & 3) + 1) ^ (srow & 7)));
-      const float d[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-      float g[8], w[8];
-      unpack8_bf16(b.g[i], g);
-      unpack8_bf16(b.w[i], w);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const float kf = bt.left ? kcol[e] : bt.krow[i];
-        w[e] = w[e] - lr * (d[e] + bt.cres * kf * g[e]);
-      }
-      *reinterpret_cast<uint4*>(bt.W + (long long)(8 * i) * bt.ld + 32 * chunk) = pack8_bf16(w);
-    }
-  }
-}
