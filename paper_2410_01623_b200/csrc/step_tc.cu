@@ -53,7 +53,7 @@ struct TcMaps {
   CUtensorMap g1a;   // G, box for the projection product
   CUtensorMap g1b;   // Pi [d][r], boxes of 64 r x 64 d
   CUtensorMap g2a;   // back-projection A operand (Pi when left, X when right), box 64 x 128
-  CUtensorMap g2b;   // back-projection B operand (X when left, Pi when right), box 64 x 256
+  CUtensorMap g2b;   // back-projection B operand (X when left, Pi when right), box 64 x 128
   // maps used only to prefetch epilogue operands into L2 ahead of the epilogue
   CUtensorMap pg;    // G [m][n] bf16, box 64 x 128
   CUtensorMap pw;    // W [m][n] bf16, box 64 x 128
@@ -491,7 +491,7 @@ size_t tc_gsq_floats(const fira_matrix_desc& d) {
 size_t tc_part_floats(const fira_matrix_desc& d) { return ((size_t)std::max(d.m, d.n) + 255) / 256; }
 
 static size_t back_tiles(const fira_matrix_desc& d) {
-  return (size_t)((d.m + BM - 1) / BM) * ((d.n + BN_MAX - 1) / BN_MAX);
+  return (size_t)((d.m + 2 * BM - 1) / (2 * BM)) * ((d.n + BN_MAX - 1) / BN_MAX);   // 256 x 256, one per CTA pair
 }
 
 // Device tables of this engine: tensor maps, fast scalars, back-projection tile records.
@@ -517,7 +517,7 @@ static bool encode_matrix_maps(const MatDev& mt, TcMaps& mp, bool only_g) {
   const void* b2 = mt.left ? (const void*)mt.Xb : (const void*)mt.P;
   const long long a2rows = mt.left ? mt.d : mt.l, b2rows = mt.left ? mt.l : mt.d;
   if (!encode_map(&mp.g2a, a2, a2rows, mt.r, mt.r, 64, 128)) return false;
-  if (!encode_map(&mp.g2b, b2, b2rows, mt.r, mt.r, 64, 256)) return false;
+  if (!encode_map(&mp.g2b, b2, b2rows, mt.r, mt.r, 64, 128)) return false;
   return true;
 }
 
@@ -532,7 +532,7 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
     const MatDev& mt = c->mats[i];
     const int bn = host_tile_bn(mt.r);
     k1.push_back(k1.back() + ((mt.l + BM - 1) / BM) * (mt.r / bn));
-    k2.push_back(k2.back() + ((mt.m + BM - 1) / BM) * ((mt.n + BN_MAX - 1) / BN_MAX));
+    k2.push_back(k2.back() + ((mt.m + 2 * BM - 1) / (2 * BM)) * ((mt.n + BN_MAX - 1) / BN_MAX));
     const int gblocks = mt.left ? ((mt.d + GSQ_ROWS - 1) / GSQ_ROWS) * ((mt.n + 2047) / 2048) : (mt.m + 7) / 8;
     gs.push_back(gs.back() + gblocks);
     const int cb = (mt.l + 255) / 256;
@@ -564,11 +564,11 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
     td.reserve(pl->k2_tiles);
     for (size_t q = 0; q < lst.size(); ++q) {
       const MatDev& mt = c->mats[lst[q]];
-      const int nrt = (mt.m + BM - 1) / BM, nct = (mt.n + BN_MAX - 1) / BN_MAX;
+      const int nrt = (mt.m + 2 * BM - 1) / (2 * BM), nct = (mt.n + BN_MAX - 1) / BN_MAX;
       for (int a = 0; a < nrt; ++a)
         for (int b = 0; b < nct; ++b) {
           BackTileDesc d;
-          d.kvec = mt.kvec; d.slot = (int)q; d.i0 = a * BM; d.j0 = b * BN_MAX; d.nkb = mt.r / BK;
+          d.kvec = mt.kvec; d.slot = (int)q; d.i0 = a * 2 * BM; d.j0 = b * BN_MAX; d.nkb = mt.r / BK;
           d.n = mt.n; d.m_left = mt.m | (mt.left ? (int)0x80000000 : 0);
           td.push_back(d);
         }
@@ -641,7 +641,8 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   k_tc_form_x<<<(pl->rows_total + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start,
                                                         pl->rows_total, hp.a_low, hp.a_res, pl->fast_dev);
   tm->mark(st);
-  k_tc_back_project<<<std::min(pl->k2_tiles, pl->num_sms), K2_THREADS, K2_SMEM_BYTES, st>>>(
+  // clusters of two CTAs, at most one CTA per SM
+  k_tc_back_project<<<2 * std::min(pl->k2_tiles, pl->num_sms / 2), K2_THREADS, K2_SMEM_BYTES, st>>>(
       pl->maps_dev, pl->td2_dev, pl->k2_tiles, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);
   return 7;
