@@ -206,6 +206,18 @@ def workload_config(wl, args):
                   else "L2 flushed between steps"}
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The job's time is the slowest rank's: every rank steps its own replica (the path
+    has no exchange step), so the only collective is this MAX over the ranks' times."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 # ----------------------------------------------------------------------------- our arm
 def main():
     args = parse_args()
@@ -281,10 +293,7 @@ def main():
     f.enable_phase_timing(False)
     launches = f.last_step_launches() * args.steps
     status = f.poll()
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    ms_step = max_over_ranks(ms_total, world, dev) / args.steps
 
     # ---- refresh, timed separately (one layer, scaled, unless --refresh full)
     refresh = None
@@ -370,10 +379,7 @@ def run_e2e(f, wl, W, G, dev, world, steps):
         f.step_host(Wh, Gh, staging)
     b.record()
     torch.cuda.synchronize()
-    t = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return {"value": float(t.item()) / steps, "unit": UNIT, "h2d_bytes_per_step": h2d,
+    return {"value": max_over_ranks(a.elapsed_time(b), world, dev) / steps, "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "steps": steps}
 
 
