@@ -17,9 +17,11 @@
 // with a bf16-rounded projection it is exact to about 2^-8 ||R_l||^2.  It only enters
 // the limiter factor lambda and the remembered norm.
 //
-// Tile shapes: 128 (TMEM lanes) x BN <= 256 (TMEM columns) x 64 (one 128-byte swizzle
-// row of bf16) per pipeline stage; two accumulators of 256 columns alternate so that
-// the epilogue of one tile overlaps the products of the next.
+// Both tensor-core kernels run on CTA pairs (clusters of two, tcgen05 cta_group::2):
+// tiles of 256 x BN <= 256 accumulator elements per pair, 64 (one 128-byte swizzle row of
+// bf16) deep per pipeline stage; two accumulators of 256 tensor-memory columns alternate so
+// that the epilogue of one tile overlaps the products of the next; all epilogue traffic
+// moves through TMA boxes in shared memory.
 #include <cuda.h>
 
 #include <algorithm>
@@ -35,18 +37,9 @@ namespace {
 constexpr int BM = 128;           // tile rows = TMEM lanes
 constexpr int BN_MAX = 256;       // tile columns = TMEM columns per accumulator
 constexpr int BK = 64;            // k-block: 64 bf16 = 128 bytes
-constexpr int STAGES = 4;
-constexpr int A_STAGE_BYTES = BM * BK * 2;       // 16 KiB
-constexpr int B_STAGE_BYTES = BN_MAX * BK * 2;   // 32 KiB
-constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int A_STAGE_BYTES = BM * BK * 2;       // 16 KiB: 128 rows x 64 bf16
 constexpr int CHUNK_BYTES = 64 * BK * 2;         // one 64 x 64 box: 8 KiB
-constexpr int EPI_WARPS = 8;
-constexpr int TC_THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
-constexpr int STG_PITCH = 32;                    // floats per staged row (16-byte slots XOR-swizzled)
-constexpr int STG_WARP_FLOATS = 32 * STG_PITCH;  // one warp's 32 x 32 fp32 staging tile
-constexpr size_t TC_SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 256 + (size_t)EPI_WARPS * STG_WARP_FLOATS * 4;
-static_assert(TC_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr int GSQ_ROWS = 128;     // rows per partial sum of G^2 (left orientation)
 
 struct TcMaps {
@@ -57,75 +50,19 @@ struct TcMaps {
   // maps used only to prefetch epilogue operands into L2 ahead of the epilogue
   CUtensorMap pg;    // G [m][n] bf16, box 64 x 128
   CUtensorMap pw;    // W [m][n] bf16, box 64 x 128
-  CUtensorMap pm;    // M [l][r] fp32, box 64 x 128
-  CUtensorMap pv;    // V [l][r] fp32, box 64 x 128
   // boxes of the back-projection epilogue (64-byte swizzle)
   CUtensorMap eg;    // G [m][n] bf16, box 32 x 128
   CUtensorMap ew;    // W [m][n] bf16, box 32 x 128 (loaded and stored)
+  // boxes of the projection epilogue
+  CUtensorMap em;    // M [l][r] fp32, box 32 x 128, 128-byte swizzle (loaded and stored)
+  CUtensorMap ev;    // V [l][r] fp32, same
+  CUtensorMap en;    // N [l][r] bf16, box 32 x 128, 64-byte swizzle (stored)
+  CUtensorMap er;    // R [l][r] bf16, same
 };
 static_assert(sizeof(TcMaps) % 64 == 0, "tensor maps must stay 64-byte aligned");
 
-__device__ __forceinline__ int tile_bn(int r) {
-  return (r % 256 == 0) ? 256 : (r % 192 == 0) ? 192 : (r % 128 == 0) ? 128 : 64;
-}
-
-struct SharedCtl {
-  uint64_t full[STAGES];
-  uint64_t empty[STAGES];
-  uint64_t tmem_full[2];
-  uint64_t tmem_empty[2];
-  uint32_t tmem_base;
-  int abort_flag;
-};
-
-// Common prologue: carve shared memory, init barriers, allocate TMEM.
-// Returns false (all threads alike) if the dynamic shared memory does not start on a
-// 1024-byte boundary, which the 128-byte swizzle of the TMA tiles needs.
-__device__ __forceinline__ bool tc_prologue(unsigned char* smem_raw, unsigned char*& tiles, SharedCtl*& ctl) {
-  tiles = smem_raw;
-  if (ptx::smem_u32(smem_raw) & 1023u) return false;
-  ctl = reinterpret_cast<SharedCtl*>(tiles + (size_t)STAGES * STAGE_BYTES);
-  const int warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      ptx::mbar_init(ptx::smem_u32(&ctl->full[s]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl->empty[s]), 1);
-    }
-    for (int b = 0; b < 2; ++b) {
-      ptx::mbar_init(ptx::smem_u32(&ctl->tmem_full[b]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[b]), EPI_WARPS);
-    }
-    ctl->abort_flag = 0;
-    ptx::fence_barrier_init();
-  }
-  if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_u32(&ctl->tmem_base), TMEM_COLS);
-    ptx::tmem_relinquish();
-  }
-  ptx::tc_fence_before();
-  __syncthreads();
-  ptx::tc_fence_after();
-  return true;
-}
-
-__device__ __forceinline__ void tc_epilogue_teardown(SharedCtl* ctl, unsigned* status) {
-  ptx::tc_fence_before();
-  __syncthreads();
-  if ((threadIdx.x >> 5) == 1) {
-    __syncwarp();
-    ptx::tc_fence_after();
-    ptx::tmem_dealloc(ctl->tmem_base, TMEM_COLS);
-  }
-  if (threadIdx.x == 0 && ctl->abort_flag) atomicOr(status, DEV_STATUS_TIMEOUT);
-}
-
-// After an aborted run the producer gives its copies in flight a bounded time to land.
-__device__ __forceinline__ void drain_stage_waits(SharedCtl* ctl, int stage, uint32_t phase, int issued_any) {
-  if (!issued_any) return;
-  for (int s = 0; s < STAGES; ++s)
-    for (uint32_t it = 0; it < (1u << 16); ++it)
-      if (ptx::mbar_try_wait(ptx::smem_u32(&ctl->full[s]), (s < stage) ? phase : (phase ^ 1u))) break;
-}
+// r-extent of a projection tile; r is a multiple of 128 on this path
+__device__ __forceinline__ int tile_bn(int r) { return (r % 256 == 0) ? 256 : 128; }
 
 __device__ __forceinline__ uint4 pack8_bf16(const float (&v)[8]) {
   __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
@@ -146,165 +83,19 @@ __device__ __forceinline__ void unpack8_bf16(const uint4& u, float (&v)[8]) {
   }
 }
 
-#include "tc_epilogue.cuh"
-
-// ============================================================================ projection product
-// Rt[l][j] = sum_d G(d,l) Pi[d][j].  Tile: 128 l x BN r.  A = G: left orientation
-// MN-major (G is [d][l], l contiguous: two 64 x 64 boxes), right orientation K-major
-// (G is [l][d]: one box of 64 d x 128 l).  B = Pi [d][r]: MN-major, BN/64 boxes.
-__global__ void __launch_bounds__(TC_THREADS, 1)
-k_tc_project(const MatDev* __restrict__ mats, const TcMaps* __restrict__ maps, const int* __restrict__ list,
-             int nlist, const int* __restrict__ tile_start, int total_tiles, Hyper hp,
-             unsigned* __restrict__ status) {
-  extern __shared__ __align__(1024) unsigned char smem_raw[];
-  unsigned char* tiles;
-  SharedCtl* ctl;
-  if (!tc_prologue(smem_raw, tiles, ctl)) {
-    if (threadIdx.x == 0) atomicOr(status, DEV_STATUS_TIMEOUT);
-    return;
-  }
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  volatile int* abort_flag = &ctl->abort_flag;
-  const uint32_t tiles_u32 = ptx::smem_u32(tiles);
-
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      int stage = 0; uint32_t phase = 0; int issued = 0; bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const int p = find_matrix(tile_start, nlist, t);
-        const MatDev& mt = mats[list[p]];
-        const TcMaps* mp = &maps[p];
-        const int r = mt.r, d = mt.d, left = mt.left;
-        const int bn = tile_bn(r), nrt = r / bn;
-        const int local = t - tile_start[p];
-        const int l0 = (local / nrt) * BM, r0 = (local % nrt) * bn;
-        const int nkb = (d + BK - 1) / BK;
-        const uint32_t bytes = A_STAGE_BYTES + bn * BK * 2;
-        // the epilogue of this tile reads M and V; start moving them from HBM to L2 now
-        for (int c = 0; c < bn / 64; ++c) {
-          ptx::tma_prefetch_l2_2d(&mp->pm, r0 + 64 * c, l0);
-          ptx::tma_prefetch_l2_2d(&mp->pv, r0 + 64 * c, l0);
-        }
-        for (int kb = 0; kb < nkb; ++kb) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
-          const uint32_t sa = tiles_u32 + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
-          ptx::mbar_expect_tx(fb, bytes);
-          const int k0 = kb * BK;
-          if (left) {
-            ptx::tma_load_2d(sa, &mp->g1a, fb, l0, k0);
-            ptx::tma_load_2d(sa + CHUNK_BYTES, &mp->g1a, fb, l0 + 64, k0);
-          } else {
-            ptx::tma_load_2d(sa, &mp->g1a, fb, k0, l0);
-          }
-          for (int c = 0; c < bn / 64; ++c) ptx::tma_load_2d(sb + c * CHUNK_BYTES, &mp->g1b, fb, r0 + 64 * c, k0);
-          issued = 1;
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-        }
-      }
-      if (!ok) drain_stage_waits(ctl, stage, phase, issued);
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      int stage = 0; uint32_t phase = 0; int buf = 0; uint32_t bphase = 0; bool ok = true;
-      const uint32_t tmem = ctl->tmem_base;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const int p = find_matrix(tile_start, nlist, t);
-        const MatDev& mt = mats[list[p]];
-        const int left = mt.left, bn = tile_bn(mt.r);
-        const int nkb = (mt.d + BK - 1) / BK;
-        const uint32_t idesc = ptx::make_idesc_bf16(BM, bn, left, 1);
-        if (!ptx::mbar_wait(ptx::smem_u32(&ctl->tmem_empty[buf]), bphase ^ 1u, abort_flag)) { ok = false; break; }
-        ptx::tc_fence_after();
-        const uint32_t dcol = tmem + buf * BN_MAX;
-        for (int kb = 0; kb < nkb; ++kb) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
-          ptx::tc_fence_after();
-          const uint32_t sa = tiles_u32 + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
-#pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            // MN-major: 16 k-rows of 128 bytes per step; K-major: 32 bytes along the row
-            const uint64_t ad = left ? ptx::make_smem_desc(sa + k * 2048, CHUNK_BYTES, 1024)
-                                     : ptx::make_smem_desc(sa + k * 32, 0, 1024);
-            const uint64_t bd = ptx::make_smem_desc(sb + k * 2048, CHUNK_BYTES, 1024);
-            ptx::umma_bf16(dcol, ad, bd, idesc, (kb | k) ? 1u : 0u);
-          }
-          ptx::umma_commit(ptx::smem_u32(&ctl->empty[stage]));
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-        }
-        if (!ok) break;
-        ptx::umma_commit(ptx::smem_u32(&ctl->tmem_full[buf]));
-        if (++buf == 2) { buf = 0; bphase ^= 1u; }
-      }
-    }
-  } else {
-    // ------------------------------------------------------------ epilogue: Adam on R
-    const int ew = warp - 2;
-    const int quarter = warp & 3;       // TMEM lanes 32*quarter .. +31 are this warp's
-    const int half = ew >> 2;           // which half of the tile's columns
-    float* stg = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(ctl) + 256) + ew * STG_WARP_FLOATS;
-    int buf = 0; uint32_t bphase = 0;
-    const uint32_t tmem = ctl->tmem_base;
-    ProjTile cur = proj_tile(mats, list, nlist, tile_start, blockIdx.x, total_tiles, quarter, half, lane);
-    MVHalf bufA, bufB;
-    if (cur.valid) load_mv(bufA, cur, 0);
-    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-      const ProjTile nxt = proj_tile(mats, list, nlist, tile_start, t + gridDim.x, total_tiles, quarter, half, lane);
-      if (!ptx::mbar_wait(ptx::smem_u32(&ctl->tmem_full[buf]), bphase, abort_flag)) break;
-      ptx::tc_fence_after();
-      float nn[8] = {}, rn[8] = {};
-      const uint32_t tcol = tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX + half * cur.nch * 32;
-      for (int c = 0; c < cur.nch; ++c) {
-        stage_rows(stg, lane, tcol + 32 * c);
-        if (c == cur.nch - 1) {           // the accumulator has been read out completely
-          ptx::tc_fence_before();
-          if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[buf]));
-        }
-        load_mv(bufB, cur, 2 * c + 1);
-        adam_half(bufA, cur, 2 * c, stg, lane, hp, nn, rn);
-        if (c + 1 < cur.nch) load_mv(bufA, cur, 2 * c + 2);
-        else if (nxt.valid) load_mv(bufA, nxt, 0);
-        adam_half(bufB, cur, 2 * c + 1, stg, lane, hp, nn, rn);
-        __syncwarp();                     // the staging tile is free again
-      }
-      // row sums: the eight lanes of a row hold its partial sums
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-#pragma unroll
-        for (int o = 1; o < 8; o <<= 1) {
-          nn[i] += __shfl_xor_sync(0xffffffffu, nn[i], o);
-          rn[i] += __shfl_xor_sync(0xffffffffu, rn[i], o);
-        }
-      }
-      if ((lane & 7) == 0) {
-        // colpart[part][l] = partial ||N_l||^2, colpart[nparts + part][l] = partial ||R_l||^2
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int l = cur.l0 + 4 * i;
-          if (l < cur.L) {
-            cur.colpart[(long long)cur.part * cur.L + l] = nn[i];
-            cur.colpart[(long long)(cur.nparts + cur.part) * cur.L + l] = rn[i];
-          }
-        }
-      }
-      cur = nxt;
-      if (++buf == 2) { buf = 0; bphase ^= 1u; }
-    }
-  }
-  tc_epilogue_teardown(ctl, status);
-}
-
+#include "tc_project.cuh"
 #include "tc_back_project.cuh"
 
 // ============================================================================ small kernels
-__global__ void k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist, Hyper hp) {
+__global__ void k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist, Hyper hp,
+                          float* __restrict__ fast) {
   const int p = blockIdx.x * blockDim.x + threadIdx.x;
   if (p >= nlist) return;
   const MatDev& mt = mats[list[p]];
   const double s = (double)(mt.sc->t + 1);
-  mt.sc->pad = (float)(sqrt(1.0 - pow((double)hp.beta2, s)) / (1.0 - pow((double)hp.beta1, s)));
+  const float bias = (float)(sqrt(1.0 - pow((double)hp.beta2, s)) / (1.0 - pow((double)hp.beta1, s)));
+  mt.sc->pad = bias;
+  fast[2 * p] = bias;          // read by the projection epilogue
 }
 
 // Sums of G^2 per unprojected index.  Left: gsq[rb][col] over blocks of GSQ_ROWS rows
@@ -363,11 +154,11 @@ k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, i
   const int l = b * 256 + threadIdx.x;
   float contrib = 0.f;
   if (l < mt.l) {
-    const int nparts = 2 * (mt.r / tile_bn(mt.r));
+    const int nparts = mt.r / tile_bn(mt.r);
     float nn = 0.f, rn = 0.f, gs = 0.f;
     for (int q = 0; q < nparts; ++q) {
-      nn += mt.colpart[(long long)q * mt.l + l];
-      rn += mt.colpart[(long long)(nparts + q) * mt.l + l];
+      nn += mt.colpart[(long long)(2 * q) * mt.l + l];
+      rn += mt.colpart[(long long)(2 * q + 1) * mt.l + l];
     }
     const int ngs = mt.left ? (mt.d + GSQ_ROWS - 1) / GSQ_ROWS : 1;
     for (int q = 0; q < ngs; ++q) gs += mt.gsq[(long long)q * mt.l + l];
@@ -434,7 +225,7 @@ EncodeTiledFn get_encode_fn() {
 // bf16 row-major matrix [rows][cols] with leading dimension ld; box = box_c x box_r.
 bool encode_map(CUtensorMap* out, const void* base, long long rows, long long cols, long long ld,
                 int box_c, int box_r, int mode = 0) {
-  // mode 0: bf16, 128-byte swizzle; 1: fp32, no swizzle (L2 prefetch only); 2: bf16, 64-byte swizzle
+  // mode 0: bf16, 128-byte swizzle; 1: fp32, 128-byte swizzle; 2: bf16, 64-byte swizzle
   const bool fp32 = mode == 1;
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) { set_error("cuTensorMapEncodeTiled is not available"); return false; }
@@ -442,17 +233,15 @@ bool encode_map(CUtensorMap* out, const void* base, long long rows, long long co
   const cuuint64_t gstr[1] = {(cuuint64_t)ld * (fp32 ? 4 : 2)};
   const cuuint32_t box[2] = {(cuuint32_t)box_c, (cuuint32_t)box_r};
   const cuuint32_t estr[2] = {1, 1};
-  // fp32 maps are only used for L2 prefetches (no shared-memory image, so no swizzle)
   const CUresult r = fn(out, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
                         const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        mode == 1 ? CU_TENSOR_MAP_SWIZZLE_NONE
-                                  : (mode == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B),
+                        mode == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with code " + std::to_string((int)r)); return false; }
   return true;
 }
 
-int host_tile_bn(int r) { return (r % 256 == 0) ? 256 : (r % 192 == 0) ? 192 : (r % 128 == 0) ? 128 : 64; }
+int host_tile_bn(int r) { return (r % 256 == 0) ? 256 : 128; }
 
 }  // namespace
 
@@ -467,6 +256,7 @@ struct TcPlan {
   const int* col_start = nullptr; int col_blocks = 0;
   const int* row_start = nullptr; int rows_total = 0;
   const int* npart = nullptr;
+  ProjTileDesc* td1_dev = nullptr;   // per-tile records of the projection
   BackTileDesc* td2_dev = nullptr;   // per-tile records of the back-projection
   float* fast_dev = nullptr;         // per matrix of the list: {bias factor, lambda}
   int num_sms = 148;
@@ -475,12 +265,12 @@ struct TcPlan {
 
 bool tc_supported(const fira_matrix_desc& d) {
   const long long ld = d.ld ? d.ld : d.n;
-  return d.dtype == FIRA_BF16 && d.r % 64 == 0 && d.m >= 256 && d.n >= 256 && d.n % 8 == 0 && ld % 8 == 0;
+  return d.dtype == FIRA_BF16 && d.r % 128 == 0 && d.m >= 256 && d.n >= 256 && d.n % 8 == 0 && ld % 8 == 0;
 }
 
 size_t tc_colpart_floats(const fira_matrix_desc& d) {
   const size_t l = std::max(d.m, d.n);
-  return 2 * (size_t)(2 * (d.r / host_tile_bn(d.r))) * l;
+  return 2 * (size_t)(d.r / host_tile_bn(d.r)) * l;
 }
 
 size_t tc_gsq_floats(const fira_matrix_desc& d) {
@@ -490,16 +280,22 @@ size_t tc_gsq_floats(const fira_matrix_desc& d) {
 
 size_t tc_part_floats(const fira_matrix_desc& d) { return ((size_t)std::max(d.m, d.n) + 255) / 256; }
 
+static size_t proj_tiles(const fira_matrix_desc& d) {
+  const int l = std::max(d.m, d.n);
+  return (size_t)((l + 2 * BM - 1) / (2 * BM)) * (d.r / host_tile_bn(d.r));   // 256 l x BN r, one per CTA pair
+}
+
 static size_t back_tiles(const fira_matrix_desc& d) {
   return (size_t)((d.m + 2 * BM - 1) / (2 * BM)) * ((d.n + BN_MAX - 1) / BN_MAX);   // 256 x 256, one per CTA pair
 }
 
 // Device tables of this engine: tensor maps, fast scalars, back-projection tile records.
 size_t tc_tables_bytes(const fira_hparams& hp, const fira_matrix_desc* descs, int count) {
-  size_t ntc = 0, tiles = 0;
+  size_t ntc = 0, tiles2 = 0, tiles1 = 0;
   for (int i = 0; i < count; ++i)
-    if (engine_for(hp, descs[i]) == 1) { ++ntc; tiles += back_tiles(descs[i]); }
-  return align_up(sizeof(TcMaps) * ntc) + align_up(2 * sizeof(float) * ntc) + align_up(sizeof(BackTileDesc) * tiles);
+    if (engine_for(hp, descs[i]) == 1) { ++ntc; tiles2 += back_tiles(descs[i]); tiles1 += proj_tiles(descs[i]); }
+  return align_up(sizeof(TcMaps) * ntc) + align_up(2 * sizeof(float) * ntc) +
+         align_up(sizeof(BackTileDesc) * tiles2) + align_up(sizeof(ProjTileDesc) * tiles1);
 }
 
 static bool encode_matrix_maps(const MatDev& mt, TcMaps& mp, bool only_g) {
@@ -510,8 +306,10 @@ static bool encode_matrix_maps(const MatDev& mt, TcMaps& mp, bool only_g) {
   if (!encode_map(&mp.eg, mt.G, mt.m, mt.n, mt.ld, K2_ECOLS, 128, 2)) return false;
   if (!encode_map(&mp.ew, mt.W, mt.m, mt.n, mt.ld, K2_ECOLS, 128, 2)) return false;
   if (only_g) return true;
-  if (!encode_map(&mp.pm, mt.M, mt.l, mt.r, mt.r, 64, 128, 1)) return false;
-  if (!encode_map(&mp.pv, mt.V, mt.l, mt.r, mt.r, 64, 128, 1)) return false;
+  if (!encode_map(&mp.em, mt.M, mt.l, mt.r, mt.r, K1_ECOLS, 128, 1)) return false;
+  if (!encode_map(&mp.ev, mt.V, mt.l, mt.r, mt.r, K1_ECOLS, 128, 1)) return false;
+  if (!encode_map(&mp.en, mt.Nb, mt.l, mt.r, mt.r, K1_ECOLS, 128, 2)) return false;
+  if (!encode_map(&mp.er, mt.Rb, mt.l, mt.r, mt.r, K1_ECOLS, 128, 2)) return false;
   if (!encode_map(&mp.g1b, mt.P, mt.d, mt.r, mt.r, 64, 64)) return false;
   const void* a2 = mt.left ? (const void*)mt.P : (const void*)mt.Xb;
   const void* b2 = mt.left ? (const void*)mt.Xb : (const void*)mt.P;
@@ -531,7 +329,7 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
   for (int i : lst) {
     const MatDev& mt = c->mats[i];
     const int bn = host_tile_bn(mt.r);
-    k1.push_back(k1.back() + ((mt.l + BM - 1) / BM) * (mt.r / bn));
+    k1.push_back(k1.back() + ((mt.l + 2 * BM - 1) / (2 * BM)) * (mt.r / bn));
     k2.push_back(k2.back() + ((mt.m + 2 * BM - 1) / (2 * BM)) * ((mt.n + BN_MAX - 1) / BN_MAX));
     const int gblocks = mt.left ? ((mt.d + GSQ_ROWS - 1) / GSQ_ROWS) * ((mt.n + 2047) / 2048) : (mt.m + 7) / 8;
     gs.push_back(gs.back() + gblocks);
@@ -558,7 +356,8 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
   char* tab = c->tc_maps_dev;
   pl->maps_dev = reinterpret_cast<TcMaps*>(tab); tab += align_up(sizeof(TcMaps) * lst.size());
   pl->fast_dev = reinterpret_cast<float*>(tab); tab += align_up(2 * sizeof(float) * lst.size());
-  pl->td2_dev = reinterpret_cast<BackTileDesc*>(tab);
+  pl->td2_dev = reinterpret_cast<BackTileDesc*>(tab); tab += align_up(sizeof(BackTileDesc) * (size_t)pl->k2_tiles);
+  pl->td1_dev = reinterpret_cast<ProjTileDesc*>(tab);
   {
     std::vector<BackTileDesc> td;
     td.reserve(pl->k2_tiles);
@@ -574,8 +373,27 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
         }
     }
     if ((int)td.size() != pl->k2_tiles) { set_error("internal: tile count mismatch"); return FIRA_ERR_INVALID_ARG; }
-    cudaError_t e = cudaMemcpyAsync(pl->td2_dev, td.data(), sizeof(BackTileDesc) * td.size(),
+    // projection tiles: the r-tiles of one l-range are neighbours, so that the CTA pairs
+    // working on them share the G panel in L2
+    std::vector<ProjTileDesc> tp;
+    tp.reserve(pl->k1_tiles);
+    for (size_t q = 0; q < lst.size(); ++q) {
+      const MatDev& mt = c->mats[lst[q]];
+      const int bn = host_tile_bn(mt.r), nrt = mt.r / bn, nlt = (mt.l + 2 * BM - 1) / (2 * BM);
+      for (int a = 0; a < nlt; ++a)
+        for (int b = 0; b < nrt; ++b) {
+          ProjTileDesc d;
+          d.colpart = mt.colpart; d.slot = (int)q; d.l0 = a * 2 * BM; d.r0 = b * bn;
+          d.nkb = (mt.d + BK - 1) / BK; d.bn_left = bn | (mt.left ? (int)0x80000000 : 0); d.L = mt.l;
+          tp.push_back(d);
+        }
+    }
+    if ((int)tp.size() != pl->k1_tiles) { set_error("internal: tile count mismatch"); return FIRA_ERR_INVALID_ARG; }
+    cudaError_t e = cudaMemcpyAsync(pl->td1_dev, tp.data(), sizeof(ProjTileDesc) * tp.size(),
                                     cudaMemcpyHostToDevice, c->stream);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(pl->td2_dev, td.data(), sizeof(BackTileDesc) * td.size(),
+                          cudaMemcpyHostToDevice, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // td dies at the end of this block
     if (e != cudaSuccess) { set_error(std::string("tile table upload: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
   }
@@ -617,7 +435,7 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   if (!pl || pl->nlist == 0) return 0;
   cudaStream_t st = c->stream;
   if (!pl->attrs_set) {
-    cudaError_t e1 = cudaFuncSetAttribute(k_tc_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES);
+    cudaError_t e1 = cudaFuncSetAttribute(k_tc_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
     cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES);
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
       set_error(std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
@@ -627,12 +445,13 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   }
   PhaseTimer* tm = &c->timer;
   const MatDev* mats = c->mats_dev;
-  k_tc_prep<<<(pl->nlist + 127) / 128, 128, 0, st>>>(mats, pl->list, pl->nlist, hp);
+  k_tc_prep<<<(pl->nlist + 127) / 128, 128, 0, st>>>(mats, pl->list, pl->nlist, hp, pl->fast_dev);
   tm->mark(st);
   k_tc_gsq<<<pl->gsq_blocks, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->gsq_start);
   tm->mark(st);
-  k_tc_project<<<std::min(pl->k1_tiles, pl->num_sms), TC_THREADS, TC_SMEM_BYTES, st>>>(
-      mats, pl->maps_dev, pl->list, pl->nlist, pl->k1_start, pl->k1_tiles, hp, c->status_dev);
+  // both tensor kernels: clusters of two CTAs, at most one CTA per SM
+  k_tc_project<<<2 * std::min(pl->k1_tiles, pl->num_sms / 2), K1_THREADS, K1_SMEM_BYTES, st>>>(
+      pl->maps_dev, pl->td1_dev, pl->k1_tiles, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);
   k_tc_colfactors<<<pl->col_blocks, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->col_start, hp);
   tm->mark(st);
@@ -641,7 +460,6 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   k_tc_form_x<<<(pl->rows_total + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start,
                                                         pl->rows_total, hp.a_low, hp.a_res, pl->fast_dev);
   tm->mark(st);
-  // clusters of two CTAs, at most one CTA per SM
   k_tc_back_project<<<2 * std::min(pl->k2_tiles, pl->num_sms / 2), K2_THREADS, K2_SMEM_BYTES, st>>>(
       pl->maps_dev, pl->td2_dev, pl->k2_tiles, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);

@@ -1,0 +1,328 @@
+// Projection product with Adam fused into its epilogue.  Included by step_tc.cu inside
+// its namespace.
+//
+//   Rt[l][j] = sum_d G(d,l) Pi[d][j]          (R = P^T G, stored with the rank index contiguous)
+//   M <- b1 M + (1-b1) R,  V <- b2 V + (1-b2) R^2,  N = bias M / (sqrt V + eps)     (Eq. 2-4)
+//   writes M, V (fp32), N, R (bf16) and the per-l partial sums ||N_l||^2, ||R_l||^2
+//
+// CTA pairs (clusters of two, one CTA per SM) walk tiles of 256 l x BN r with
+// tcgen05.mma.cta_group::2.  A = G: for m <= n an MN-major operand (G is [d][l], l
+// contiguous: two 64 x 64 boxes per CTA and stage), for m > n a K-major operand (one box
+// of 64 d x 128 l).  B = Pi [d][r], MN-major; each CTA loads half of the tile's r range.
+// No transposed copy of G or Pi is ever made, and no TMA multicast is used.
+//
+// The epilogue moves M and V through shared memory with TMA in both directions (boxes of
+// 128 rows x 32 columns, updated in place by one thread per row) and stores N and R the
+// same way: ordinary global loads would be throttled by the few L1 lines that remain when
+// nearly the whole L1/shared array is configured as shared memory.
+//
+// Warp roles: 0 operand producer (TMA); 1 MMA issuer (even CTA only) and TMEM owner;
+// 2 epilogue loader (TMA); 3-6 epilogue; 7 one thread that stores the finished boxes.
+constexpr int K1_STAGES = 4;
+constexpr int K1_STAGE_BYTES = 2 * A_STAGE_BYTES;       // A: 128 l x 64 d, B half: 128 r x 64 d
+constexpr int K1_EBUFS = 2;
+constexpr int K1_ECOLS = 32;                            // columns per epilogue box
+constexpr int K1_FBOX_BYTES = BM * K1_ECOLS * 4;        // fp32 box: 16 KiB
+constexpr int K1_HBOX_BYTES = BM * K1_ECOLS * 2;        // bf16 box: 8 KiB
+constexpr int K1_EBUF_BYTES = 2 * K1_FBOX_BYTES + 2 * K1_HBOX_BYTES;   // M, V, N, R
+constexpr int K1_EPI_THREADS = 128;
+constexpr int K1_THREADS = 32 * 8;
+constexpr size_t K1_SMEM_BYTES = (size_t)K1_STAGES * K1_STAGE_BYTES + (size_t)K1_EBUFS * K1_EBUF_BYTES + 512;
+static_assert(K1_SMEM_BYTES <= 227 * 1024, "shared memory budget");
+
+// Per-tile record (256 l x BN r), built on the host once (32 bytes).
+struct ProjTileDesc {
+  float* colpart;      // partial sums of the tile's matrix: [2 part + which][l]
+  int slot;            // index into the tensor-map table and the fast-scalar table
+  int l0, r0;          // first unprojected index / first rank index of the tile
+  int nkb;             // k-blocks: ceil(d / 64)
+  int bn_left;         // BN (128 or 256), bit 31 set for the left orientation
+  int L;               // number of unprojected indices of the matrix
+};
+static_assert(sizeof(ProjTileDesc) == 32, "ProjTileDesc layout");
+
+struct ProjCtl {
+  uint64_t full[K1_STAGES];     // (even CTA) both CTAs' operands of a stage have landed
+  uint64_t empty[K1_STAGES];    // the MMAs reading a stage are done (both CTAs are told)
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];       // (even CTA) both CTAs' epilogues have drained an accumulator
+  uint64_t efull[K1_EBUFS];     // an M box and a V box have landed
+  uint64_t eready[K1_EBUFS];    // the epilogue has finished the four boxes in place
+  uint64_t eempty[K1_EBUFS];    // their stores have read them: the buffer is free
+  uint32_t tmem_base;
+  int abort_flag;
+};
+static_assert(sizeof(ProjCtl) <= 512, "ProjCtl must fit its slot");
+
+__device__ __forceinline__ ProjTileDesc load_desc(const ProjTileDesc* __restrict__ td, int t) {
+  const int4 a = __ldg(reinterpret_cast<const int4*>(td + t));
+  const int4 b = __ldg(reinterpret_cast<const int4*>(td + t) + 1);
+  ProjTileDesc d;
+  d.colpart = reinterpret_cast<float*>((static_cast<unsigned long long>(static_cast<unsigned>(a.y)) << 32) |
+                                       static_cast<unsigned>(a.x));
+  d.slot = a.z; d.l0 = a.w; d.r0 = b.x; d.nkb = b.y; d.bn_left = b.z; d.L = b.w;
+  return d;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(K1_THREADS, 1)
+k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ tdesc, int total_tiles,
+             const float* __restrict__ fast, Hyper hp, unsigned* __restrict__ status) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* tiles = smem_raw;
+  unsigned char* ebuf = tiles + (size_t)K1_STAGES * K1_STAGE_BYTES;
+  ProjCtl* ctl = reinterpret_cast<ProjCtl*>(ebuf + (size_t)K1_EBUFS * K1_EBUF_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();          // 0: issues the MMAs; 1: its partner
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  // the swizzled TMA tiles need a 1024-byte aligned base (same in both CTAs)
+  const bool smem_ok = (ptx::smem_u32(smem_raw) & 1023u) == 0;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < K1_STAGES; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&ctl->full[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(ptx::smem_u32(&ctl->tmem_full[b]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[b]), 2 * 4);   // every epilogue warp of the pair
+    }
+    for (int b = 0; b < K1_EBUFS; ++b) {
+      ptx::mbar_init(ptx::smem_u32(&ctl->efull[b]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl->eready[b]), K1_EPI_THREADS);
+      ptx::mbar_init(ptx::smem_u32(&ctl->eempty[b]), 1);
+    }
+    ctl->abort_flag = smem_ok ? 0 : 1;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(ptx::smem_u32(&ctl->tmem_base), TMEM_COLS);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync_all();      // the partner's barriers exist before anything arrives on them
+  ptx::tc_fence_after();
+  volatile int* abort_flag = &ctl->abort_flag;
+  const uint32_t tiles_u32 = ptx::smem_u32(tiles);
+  const uint32_t ebuf_u32 = ptx::smem_u32(ebuf);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ operand producer
+    if (lane == 0 && smem_ok) {
+      int stage = 0; uint32_t phase = 0; bool ok = true;
+      ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
+      for (int t = pair; t < total_tiles && ok; t += npairs) {
+        const ProjTileDesc d = nd;
+        if (t + npairs < total_tiles) nd = load_desc(tdesc, t + npairs);
+        const TcMaps* mp = &maps[d.slot];
+        const int left = d.bn_left < 0;
+        const int bn = d.bn_left & 0xffff;
+        const int l0 = d.l0 + BM * (int)rank;             // this CTA's unprojected indices
+        const int rb0 = d.r0 + (bn / 2) * (int)rank;      // this CTA's half of the rank range
+        const uint32_t bytes = 2 * (A_STAGE_BYTES + (bn / 2) * BK * 2);   // both CTAs together
+        for (int kb = 0; kb < d.nkb; ++kb) {
+          if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+          // all boxes of the pair complete on the even CTA's barrier
+          const uint32_t fb = ptx::map_to_cta(ptx::smem_u32(&ctl->full[stage]), 0);
+          const uint32_t sa = tiles_u32 + stage * K1_STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+          if (rank == 0) ptx::mbar_expect_tx(ptx::smem_u32(&ctl->full[stage]), bytes);
+          const int k0 = kb * BK;
+          if (left) {
+            ptx::tma_load_2d_pair(sa, &mp->g1a, fb, l0, k0);
+            ptx::tma_load_2d_pair(sa + CHUNK_BYTES, &mp->g1a, fb, l0 + 64, k0);
+          } else {
+            ptx::tma_load_2d_pair(sa, &mp->g1a, fb, k0, l0);
+          }
+          for (int c = 0; c < bn / 128; ++c)
+            ptx::tma_load_2d_pair(sb + c * CHUNK_BYTES, &mp->g1b, fb, rb0 + 64 * c, k0);
+          if (++stage == K1_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok && rank == 0) {   // give copies in flight a bounded time to land
+        for (int s = 0; s < K1_STAGES; ++s)
+          for (uint32_t it = 0; it < (1u << 16); ++it)
+            if (ptx::mbar_try_wait_cluster(ptx::smem_u32(&ctl->full[s]), (s < stage) ? phase : (phase ^ 1u))) break;
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (even CTA)
+    if (lane == 0 && smem_ok && rank == 0) {
+      int stage = 0; uint32_t phase = 0; int buf = 0; uint32_t bphase = 0; bool ok = true;
+      ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
+      const uint32_t tmem = ctl->tmem_base;
+      for (int t = pair; t < total_tiles && ok; t += npairs) {
+        const ProjTileDesc d = nd;
+        if (t + npairs < total_tiles) nd = load_desc(tdesc, t + npairs);
+        const int left = d.bn_left < 0;
+        const int bn = d.bn_left & 0xffff;
+        const uint32_t idesc = ptx::make_idesc_bf16(2 * BM, bn, left, 1);
+        if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->tmem_empty[buf]), bphase ^ 1u, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t dcol = tmem + buf * BN_MAX;
+        for (int kb = 0; kb < d.nkb; ++kb) {
+          if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t sa = tiles_u32 + stage * K1_STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            // MN-major: 16 k-rows of 128 bytes per step; K-major: 32 bytes along the row
+            const uint64_t ad = left ? ptx::make_smem_desc(sa + k * 2048, CHUNK_BYTES, 1024)
+                                     : ptx::make_smem_desc(sa + k * 32, 0, 1024);
+            const uint64_t bd = ptx::make_smem_desc(sb + k * 2048, CHUNK_BYTES, 1024);
+            ptx::umma_bf16_pair(dcol, ad, bd, idesc, (kb | k) ? 1u : 0u);
+          }
+          ptx::umma_commit_pair(ptx::smem_u32(&ctl->empty[stage]), 3);
+          if (++stage == K1_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::umma_commit_pair(ptx::smem_u32(&ctl->tmem_full[buf]), 3);
+        if (++buf == 2) { buf = 0; bphase ^= 1u; }
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------ epilogue loader: M and V boxes
+    if (lane == 0 && smem_ok) {
+      int eb = 0; uint32_t ephase = 0; bool ok = true;
+      ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
+      for (int t = pair; t < total_tiles && ok; t += npairs) {
+        const ProjTileDesc d = nd;
+        if (t + npairs < total_tiles) nd = load_desc(tdesc, t + npairs);
+        const TcMaps* mp = &maps[d.slot];
+        const int bn = d.bn_left & 0xffff;
+        const int l0 = d.l0 + BM * (int)rank;
+        for (int c = 0; c < bn / K1_ECOLS; ++c) {
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->eempty[eb]), ephase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t fb = ptx::smem_u32(&ctl->efull[eb]);
+          const uint32_t dst = ebuf_u32 + eb * K1_EBUF_BYTES;
+          ptx::mbar_expect_tx(fb, 2 * K1_FBOX_BYTES);
+          ptx::tma_load_2d(dst, &mp->em, fb, d.r0 + K1_ECOLS * c, l0);
+          ptx::tma_load_2d(dst + K1_FBOX_BYTES, &mp->ev, fb, d.r0 + K1_ECOLS * c, l0);
+          if (++eb == K1_EBUFS) { eb = 0; ephase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 7) {
+    // ------------------------------------------------------------ box storer
+    if (lane == 0 && smem_ok) {
+      int eb = 0; uint32_t rphase = 0; bool ok = true;
+      ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
+      for (int t = pair; t < total_tiles && ok; t += npairs) {
+        const ProjTileDesc d = nd;
+        if (t + npairs < total_tiles) nd = load_desc(tdesc, t + npairs);
+        const TcMaps* mp = &maps[d.slot];
+        const int bn = d.bn_left & 0xffff;
+        const int l0 = d.l0 + BM * (int)rank;
+        for (int c = 0; c < bn / K1_ECOLS; ++c) {
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->eready[eb]), rphase, abort_flag)) { ok = false; break; }
+          if (l0 < d.L) {
+            const uint32_t src = ebuf_u32 + eb * K1_EBUF_BYTES;
+            const int j = d.r0 + K1_ECOLS * c;
+            ptx::tma_store_2d(&mp->em, src, j, l0);
+            ptx::tma_store_2d(&mp->ev, src + K1_FBOX_BYTES, j, l0);
+            ptx::tma_store_2d(&mp->en, src + 2 * K1_FBOX_BYTES, j, l0);
+            ptx::tma_store_2d(&mp->er, src + 2 * K1_FBOX_BYTES + K1_HBOX_BYTES, j, l0);
+            ptx::bulk_commit_group();
+            ptx::bulk_wait_group_read<0>();              // the boxes have been read: the buffer is free
+          }
+          ptx::mbar_arrive(ptx::smem_u32(&ctl->eempty[eb]));
+          if (++eb == K1_EBUFS) { eb = 0; rphase ^= 1u; }
+        }
+      }
+      ptx::bulk_wait_group_all();
+    }
+  } else if (smem_ok) {
+    // ------------------------------------------------------------ epilogue: Adam on R
+    const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31
+    const int row = quarter * 32 + lane;                // row of this CTA's half tile = TMEM lane
+    const uint32_t frow = (uint32_t)row * (K1_ECOLS * 4);   // fp32 boxes: 128-byte rows
+    const uint32_t fsw = (uint32_t)row & 7u;                //   128-byte swizzle: slot ^= row % 8
+    const uint32_t hrow = (uint32_t)row * (K1_ECOLS * 2);   // bf16 boxes: 64-byte rows
+    const uint32_t hsw = (uint32_t)(row >> 1) & 3u;         //   64-byte swizzle: slot ^= (row / 2) % 4
+    const uint32_t tmem_empty0 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[0]), 0);
+    const uint32_t tmem_empty1 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[1]), 0);
+    int buf = 0; uint32_t bphase = 0;
+    int eb = 0; uint32_t ephase = 0;
+    const uint32_t tmem = ctl->tmem_base;
+    bool ok = true;
+    ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
+    for (int t = pair; t < total_tiles && ok; t += npairs) {
+      const ProjTileDesc d = nd;
+      if (t + npairs < total_tiles) nd = load_desc(tdesc, t + npairs);
+      const int bn = d.bn_left & 0xffff;
+      const int l = d.l0 + BM * (int)rank + row;
+      const float bias = fast[2 * d.slot];
+      if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->tmem_full[buf]), bphase, abort_flag)) break;
+      ptx::tc_fence_after();
+      const uint32_t tcol = tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX;
+      const uint32_t te = buf ? tmem_empty1 : tmem_empty0;
+      const int nch = bn / K1_ECOLS;
+      float nn = 0.f, rn = 0.f;
+      for (int c = 0; c < nch; ++c) {
+        uint32_t rr[32];
+        __syncwarp();
+        ptx::tmem_ld_32x32b_x32(tcol + K1_ECOLS * c, rr);
+        ptx::tmem_ld_wait();
+        if (c == nch - 1) {                              // the accumulator has been read out
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_cluster(te);
+        }
+        if (!ptx::mbar_wait(ptx::smem_u32(&ctl->efull[eb]), ephase, abort_flag)) { ok = false; break; }
+        unsigned char* mb = ebuf + (size_t)eb * K1_EBUF_BYTES;
+        unsigned char* vb = mb + K1_FBOX_BYTES;
+        unsigned char* nb = vb + K1_FBOX_BYTES;
+        unsigned char* rb = nb + K1_HBOX_BYTES;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {                    // 8 columns at a time
+          const uint32_t f0 = frow + (((uint32_t)(2 * q) ^ fsw) << 4);
+          const uint32_t f1 = frow + (((uint32_t)(2 * q + 1) ^ fsw) << 4);
+          const float4 m0 = *reinterpret_cast<const float4*>(mb + f0);
+          const float4 m1 = *reinterpret_cast<const float4*>(mb + f1);
+          const float4 v0 = *reinterpret_cast<const float4*>(vb + f0);
+          const float4 v1 = *reinterpret_cast<const float4*>(vb + f1);
+          float mo[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+          float vo[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+          float rv[8], nv[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            rv[e] = __uint_as_float(rr[8 * q + e]);
+            mo[e] = hp.beta1 * mo[e] + (1.f - hp.beta1) * rv[e];
+            vo[e] = hp.beta2 * vo[e] + (1.f - hp.beta2) * rv[e] * rv[e];
+            nv[e] = bias * mo[e] / (sqrtf(vo[e]) + hp.eps);
+            nn = fmaf(nv[e], nv[e], nn);
+            rn = fmaf(rv[e], rv[e], rn);
+          }
+          *reinterpret_cast<float4*>(mb + f0) = make_float4(mo[0], mo[1], mo[2], mo[3]);
+          *reinterpret_cast<float4*>(mb + f1) = make_float4(mo[4], mo[5], mo[6], mo[7]);
+          *reinterpret_cast<float4*>(vb + f0) = make_float4(vo[0], vo[1], vo[2], vo[3]);
+          *reinterpret_cast<float4*>(vb + f1) = make_float4(vo[4], vo[5], vo[6], vo[7]);
+          const uint32_t h = hrow + (((uint32_t)q ^ hsw) << 4);
+          *reinterpret_cast<uint4*>(nb + h) = pack8_bf16(nv);
+          *reinterpret_cast<uint4*>(rb + h) = pack8_bf16(rv);
+        }
+        // hand the finished boxes to the storer: this thread's writes are visible to
+        // the async proxy (TMA) before it arrives
+        ptx::fence_proxy_async_smem();
+        ptx::mbar_arrive(ptx::smem_u32(&ctl->eready[eb]));
+        if (++eb == K1_EBUFS) { eb = 0; ephase ^= 1u; }
+      }
+      if (ok && l < d.L) {
+        // colpart[2 part][l] = partial ||N_l||^2, colpart[2 part + 1][l] = partial ||R_l||^2
+        const int part = d.r0 / bn;
+        d.colpart[(long long)(2 * part) * d.L + l] = nn;
+        d.colpart[(long long)(2 * part + 1) * d.L + l] = rn;
+      }
+      if (++buf == 2) { buf = 0; bphase ^= 1u; }
+    }
+  }
+  // Neither CTA may leave while its partner can still reach into its shared memory
+  // (operand reads by the MMAs, barrier arrivals).
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync_all();
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(ctl->tmem_base, TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && ctl->abort_flag) atomicOr(status, DEV_STATUS_TIMEOUT);
+}
