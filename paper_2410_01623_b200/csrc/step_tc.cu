@@ -43,8 +43,8 @@ constexpr int TMEM_COLS = 512;
 constexpr int GSQ_ROWS = 128;     // rows per partial sum of G^2 (left orientation)
 
 struct TcMaps {
-  CUtensorMap g1a;   // G, box for the projection product
-  CUtensorMap g1b;   // Pi [d][r], boxes of 64 r x 64 d
+  CUtensorMap g1a;   // G, box for the projection product (2-D, or chunked 3-D: see encode_matrix_maps)
+  CUtensorMap g1b;   // Pi [d][r] as chunks of 64 r: box of 64 r x 64 d x (BN / 128) chunks
   CUtensorMap g2a;   // back-projection A operand (Pi when left, X when right), box 64 x 128
   CUtensorMap g2b;   // back-projection B operand (X when left, Pi when right), box 64 x 128
   // maps used only to prefetch epilogue operands into L2 ahead of the epilogue
@@ -241,6 +241,24 @@ bool encode_map(CUtensorMap* out, const void* base, long long rows, long long co
   return true;
 }
 
+// The same matrix seen as [cols / 64 chunks][rows][64]: one box brings `nchunk` adjacent
+// 64-column chunks of box_r rows, each landing as its own swizzled 128-byte-row block (the
+// layout of an MN-major operand).  Needs cols % 64 == 0: the chunk dimension has no ragged edge.
+bool encode_map_chunked(CUtensorMap* out, const void* base, long long rows, long long cols, long long ld,
+                        int box_r, int nchunk) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) { set_error("cuTensorMapEncodeTiled is not available"); return false; }
+  const cuuint64_t gdim[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+  const cuuint64_t gstr[2] = {(cuuint64_t)ld * 2, 128};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_r, (cuuint32_t)nchunk};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstr, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled (chunked) failed with code " + std::to_string((int)r)); return false; }
+  return true;
+}
+
 int host_tile_bn(int r) { return (r % 256 == 0) ? 256 : 128; }
 
 }  // namespace
@@ -299,8 +317,11 @@ size_t tc_tables_bytes(const fira_hparams& hp, const fira_matrix_desc* descs, in
 }
 
 static bool encode_matrix_maps(const MatDev& mt, TcMaps& mp, bool only_g) {
-  // G is [m][n]: left -> boxes of 64 l x 64 d rows; right -> box of 64 d x 128 l rows
-  if (!encode_map(&mp.g1a, mt.G, mt.m, mt.n, mt.ld, 64, mt.left ? 64 : 128)) return false;
+  // G is [m][n]: left -> 64 d rows of two 64-wide chunks of l (one chunked box when n % 64 == 0,
+  // else two plain boxes); right -> box of 64 d x 128 l rows
+  if (mt.left && mt.n % 64 == 0) {
+    if (!encode_map_chunked(&mp.g1a, mt.G, mt.m, mt.n, mt.ld, 64, 2)) return false;
+  } else if (!encode_map(&mp.g1a, mt.G, mt.m, mt.n, mt.ld, 64, mt.left ? 64 : 128)) return false;
   if (!encode_map(&mp.pg, mt.G, mt.m, mt.n, mt.ld, 64, 128)) return false;
   if (!encode_map(&mp.pw, mt.W, mt.m, mt.n, mt.ld, 64, 128)) return false;
   if (!encode_map(&mp.eg, mt.G, mt.m, mt.n, mt.ld, K2_ECOLS, 128, 2)) return false;
@@ -310,7 +331,7 @@ static bool encode_matrix_maps(const MatDev& mt, TcMaps& mp, bool only_g) {
   if (!encode_map(&mp.ev, mt.V, mt.l, mt.r, mt.r, K1_ECOLS, 128, 1)) return false;
   if (!encode_map(&mp.en, mt.Nb, mt.l, mt.r, mt.r, K1_ECOLS, 128, 2)) return false;
   if (!encode_map(&mp.er, mt.Rb, mt.l, mt.r, mt.r, K1_ECOLS, 128, 2)) return false;
-  if (!encode_map(&mp.g1b, mt.P, mt.d, mt.r, mt.r, 64, 64)) return false;
+  if (!encode_map_chunked(&mp.g1b, mt.P, mt.d, mt.r, mt.r, 64, host_tile_bn(mt.r) / 128)) return false;
   const void* a2 = mt.left ? (const void*)mt.P : (const void*)mt.Xb;
   const void* b2 = mt.left ? (const void*)mt.Xb : (const void*)mt.P;
   const long long a2rows = mt.left ? mt.d : mt.l, b2rows = mt.left ? mt.l : mt.d;
@@ -384,7 +405,8 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
         for (int b = 0; b < nrt; ++b) {
           ProjTileDesc d;
           d.colpart = mt.colpart; d.slot = (int)q; d.l0 = a * 2 * BM; d.r0 = b * bn;
-          d.nkb = (mt.d + BK - 1) / BK; d.bn_left = bn | (mt.left ? (int)0x80000000 : 0); d.L = mt.l;
+          d.nkb = (mt.d + BK - 1) / BK; d.L = mt.l;
+          d.bn_left = bn | (mt.left ? (int)0x80000000 : 0) | ((mt.left && mt.n % 64 == 0) ? PROJ_A_CHUNKED : 0);
           tp.push_back(d);
         }
     }

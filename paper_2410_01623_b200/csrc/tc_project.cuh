@@ -7,9 +7,14 @@
 //
 // CTA pairs (clusters of two, one CTA per SM) walk tiles of 256 l x BN r with
 // tcgen05.mma.cta_group::2.  A = G: for m <= n an MN-major operand (G is [d][l], l
-// contiguous: two 64 x 64 boxes per CTA and stage), for m > n a K-major operand (one box
-// of 64 d x 128 l).  B = Pi [d][r], MN-major; each CTA loads half of the tile's r range.
+// contiguous: 64 d rows of two 64-wide chunks per CTA and stage), for m > n a K-major operand
+// (one box of 64 d x 128 l).  B = Pi [d][r], MN-major; each CTA loads half of the tile's r range.
 // No transposed copy of G or Pi is ever made, and no TMA multicast is used.
+//
+// One TMA instruction occupies the issuing thread for well over a hundred cycles, so a stage is
+// loaded with two instructions: the chunks of an MN-major operand come as one 3-D box (the matrix
+// seen as [chunk][row][64]).  Only a left-orientation G whose width is not a multiple of 64 falls
+// back to one 2-D box per chunk.
 //
 // The epilogue moves M and V through shared memory with TMA in both directions (boxes of
 // 128 rows x 32 columns, updated in place by one thread per row) and stores N and R the
@@ -36,10 +41,11 @@ struct ProjTileDesc {
   int slot;            // index into the tensor-map table and the fast-scalar table
   int l0, r0;          // first unprojected index / first rank index of the tile
   int nkb;             // k-blocks: ceil(d / 64)
-  int bn_left;         // BN (128 or 256), bit 31 set for the left orientation
+  int bn_left;         // BN (128 or 256); bit 31: left orientation; bit 30: G comes as one chunked box
   int L;               // number of unprojected indices of the matrix
 };
 static_assert(sizeof(ProjTileDesc) == 32, "ProjTileDesc layout");
+constexpr int PROJ_A_CHUNKED = 1 << 30;
 
 struct ProjCtl {
   uint64_t full[K1_STAGES];     // (even CTA) both CTAs' operands of a stage have landed
@@ -53,6 +59,13 @@ struct ProjCtl {
   int abort_flag;
 };
 static_assert(sizeof(ProjCtl) <= 512, "ProjCtl must fit its slot");
+
+// sqrt.approx and the fast division are good to about 2 ulp each; N is rounded to bf16 next.
+__device__ __forceinline__ float fast_sqrt(float x) {
+  float y;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 __device__ __forceinline__ ProjTileDesc load_desc(const ProjTileDesc* __restrict__ td, int t) {
   const int4 a = __ldg(reinterpret_cast<const int4*>(td + t));
@@ -126,14 +139,15 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           const uint32_t sa = tiles_u32 + stage * K1_STAGE_BYTES, sb = sa + A_STAGE_BYTES;
           if (rank == 0) ptx::mbar_expect_tx(ptx::smem_u32(&ctl->full[stage]), bytes);
           const int k0 = kb * BK;
-          if (left) {
+          if (d.bn_left & PROJ_A_CHUNKED) {
+            ptx::tma_load_3d_pair(sa, &mp->g1a, fb, 0, k0, l0 >> 6);
+          } else if (left) {
             ptx::tma_load_2d_pair(sa, &mp->g1a, fb, l0, k0);
             ptx::tma_load_2d_pair(sa + CHUNK_BYTES, &mp->g1a, fb, l0 + 64, k0);
           } else {
             ptx::tma_load_2d_pair(sa, &mp->g1a, fb, k0, l0);
           }
-          for (int c = 0; c < bn / 128; ++c)
-            ptx::tma_load_2d_pair(sb + c * CHUNK_BYTES, &mp->g1b, fb, rb0 + 64 * c, k0);
+          ptx::tma_load_3d_pair(sb, &mp->g1b, fb, 0, k0, rb0 >> 6);
           if (++stage == K1_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -287,7 +301,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
             rv[e] = __uint_as_float(rr[8 * q + e]);
             mo[e] = hp.beta1 * mo[e] + (1.f - hp.beta1) * rv[e];
             vo[e] = hp.beta2 * vo[e] + (1.f - hp.beta2) * rv[e] * rv[e];
-            nv[e] = bias * mo[e] / (sqrtf(vo[e]) + hp.eps);
+            nv[e] = __fdividef(bias * mo[e], fast_sqrt(vo[e]) + hp.eps);
             nn = fmaf(nv[e], nv[e], nn);
             rn = fmaf(rv[e], rv[e], rn);
           }
