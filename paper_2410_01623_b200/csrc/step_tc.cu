@@ -47,16 +47,13 @@ struct TcMaps {
   CUtensorMap g1b;   // Pi [d][r] as chunks of 64 r: box of 64 r x 64 d x (BN / 128) chunks
   CUtensorMap g2a;   // back-projection A operand (Pi when left, X when right), box 64 x 128
   CUtensorMap g2b;   // back-projection B operand (X when left, Pi when right), box 64 x 128
-  // maps used only to prefetch epilogue operands into L2 ahead of the epilogue
-  CUtensorMap pg;    // G [m][n] bf16, box 64 x 128
-  CUtensorMap pw;    // W [m][n] bf16, box 64 x 128
   // boxes of the back-projection epilogue (64-byte swizzle)
   CUtensorMap eg;    // G [m][n] bf16, box 32 x 128
   CUtensorMap ew;    // W [m][n] bf16, box 32 x 128 (loaded and stored)
   // boxes of the projection epilogue
-  CUtensorMap em;    // M [l][r] fp32, box 32 x 128, 128-byte swizzle (loaded and stored)
+  CUtensorMap em;    // M [l][r] fp32, box 32 x 64, 128-byte swizzle (loaded and stored)
   CUtensorMap ev;    // V [l][r] fp32, same
-  CUtensorMap en;    // N [l][r] bf16, box 32 x 128, 64-byte swizzle (stored)
+  CUtensorMap en;    // N [l][r] bf16, box 32 x 64, 64-byte swizzle (stored)
   CUtensorMap er;    // R [l][r] bf16, same
 };
 static_assert(sizeof(TcMaps) % 64 == 0, "tensor maps must stay 64-byte aligned");
@@ -322,15 +319,13 @@ static bool encode_matrix_maps(const MatDev& mt, TcMaps& mp, bool only_g) {
   if (mt.left && mt.n % 64 == 0) {
     if (!encode_map_chunked(&mp.g1a, mt.G, mt.m, mt.n, mt.ld, 64, 2)) return false;
   } else if (!encode_map(&mp.g1a, mt.G, mt.m, mt.n, mt.ld, 64, mt.left ? 64 : 128)) return false;
-  if (!encode_map(&mp.pg, mt.G, mt.m, mt.n, mt.ld, 64, 128)) return false;
-  if (!encode_map(&mp.pw, mt.W, mt.m, mt.n, mt.ld, 64, 128)) return false;
   if (!encode_map(&mp.eg, mt.G, mt.m, mt.n, mt.ld, K2_ECOLS, 128, 2)) return false;
   if (!encode_map(&mp.ew, mt.W, mt.m, mt.n, mt.ld, K2_ECOLS, 128, 2)) return false;
   if (only_g) return true;
-  if (!encode_map(&mp.em, mt.M, mt.l, mt.r, mt.r, K1_ECOLS, 128, 1)) return false;
-  if (!encode_map(&mp.ev, mt.V, mt.l, mt.r, mt.r, K1_ECOLS, 128, 1)) return false;
-  if (!encode_map(&mp.en, mt.Nb, mt.l, mt.r, mt.r, K1_ECOLS, 128, 2)) return false;
-  if (!encode_map(&mp.er, mt.Rb, mt.l, mt.r, mt.r, K1_ECOLS, 128, 2)) return false;
+  if (!encode_map(&mp.em, mt.M, mt.l, mt.r, mt.r, K1_ECOLS, K1_EROWS, 1)) return false;
+  if (!encode_map(&mp.ev, mt.V, mt.l, mt.r, mt.r, K1_ECOLS, K1_EROWS, 1)) return false;
+  if (!encode_map(&mp.en, mt.Nb, mt.l, mt.r, mt.r, K1_ECOLS, K1_EROWS, 2)) return false;
+  if (!encode_map(&mp.er, mt.Rb, mt.l, mt.r, mt.r, K1_ECOLS, K1_EROWS, 2)) return false;
   if (!encode_map_chunked(&mp.g1b, mt.P, mt.d, mt.r, mt.r, 64, host_tile_bn(mt.r) / 128)) return false;
   const void* a2 = mt.left ? (const void*)mt.P : (const void*)mt.Xb;
   const void* b2 = mt.left ? (const void*)mt.Xb : (const void*)mt.P;

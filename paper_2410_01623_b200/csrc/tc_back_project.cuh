@@ -131,13 +131,6 @@ k_tc_back_project(const TcMaps* __restrict__ maps, const BackTileDesc* __restric
         const TcMaps* mp = &maps[d.slot];
         const int i0 = d.i0 + BM * (int)rank;            // this CTA's rows of W and of A
         const int jb0 = d.j0 + (BN_MAX / 2) * (int)rank; // this CTA's half of the B rows
-        // the epilogue of this tile reads G and W; start moving them from HBM to L2 now
-        for (int c = 0; c < BN_MAX / 64; ++c) {
-          if (d.j0 + 64 * c < d.n) {
-            ptx::tma_prefetch_l2_2d(&mp->pg, d.j0 + 64 * c, i0);
-            ptx::tma_prefetch_l2_2d(&mp->pw, d.j0 + 64 * c, i0);
-          }
-        }
         for (int kb = 0; kb < d.nkb; ++kb) {
           if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
           // all four boxes of the pair complete on the even CTA's barrier

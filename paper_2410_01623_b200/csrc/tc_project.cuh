@@ -17,22 +17,31 @@
 // back to one 2-D box per chunk.
 //
 // The epilogue moves M and V through shared memory with TMA in both directions (boxes of
-// 128 rows x 32 columns, updated in place by one thread per row) and stores N and R the
+// 64 rows x 32 columns, updated in place by one thread per row) and stores N and R the
 // same way: ordinary global loads would be throttled by the few L1 lines that remain when
-// nearly the whole L1/shared array is configured as shared memory.
+// nearly the whole L1/shared array is configured as shared memory.  The boxes of a tile come
+// in the order (columns 0-31, rows 0-63), (columns 0-31, rows 64-127), (columns 32-63, ...):
+// epilogue warps 0-1 take the even boxes, warps 2-3 the odd ones.  Three M/V buffers rotate
+// over all boxes, so that loads run ahead; the N/R buffer of a box is the one of its row half.
+// Small boxes leave room for five operand stages: the time from a stage's release to its next
+// MMA is several thousand cycles, which four stages do not cover.
 //
 // Warp roles: 0 operand producer (TMA); 1 MMA issuer (even CTA only) and TMEM owner;
 // 2 epilogue loader (TMA); 3-6 epilogue; 7 one thread that stores the finished boxes.
-constexpr int K1_STAGES = 4;
+constexpr int K1_STAGES = 5;
 constexpr int K1_STAGE_BYTES = 2 * A_STAGE_BYTES;       // A: 128 l x 64 d, B half: 128 r x 64 d
-constexpr int K1_EBUFS = 2;
 constexpr int K1_ECOLS = 32;                            // columns per epilogue box
-constexpr int K1_FBOX_BYTES = BM * K1_ECOLS * 4;        // fp32 box: 16 KiB
-constexpr int K1_HBOX_BYTES = BM * K1_ECOLS * 2;        // bf16 box: 8 KiB
-constexpr int K1_EBUF_BYTES = 2 * K1_FBOX_BYTES + 2 * K1_HBOX_BYTES;   // M, V, N, R
-constexpr int K1_EPI_THREADS = 128;
+constexpr int K1_EROWS = 64;                            // rows per epilogue box
+constexpr int K1_FBOX_BYTES = K1_EROWS * K1_ECOLS * 4;  // fp32 box: 8 KiB
+constexpr int K1_HBOX_BYTES = K1_EROWS * K1_ECOLS * 2;  // bf16 box: 4 KiB
+constexpr int K1_MVBUFS = 3;                            // {M box, V box}
+constexpr int K1_NRBUFS = 2;                            // {N box, R box}, one per row half
+constexpr int K1_MVBUF_BYTES = 2 * K1_FBOX_BYTES;
+constexpr int K1_NRBUF_BYTES = 2 * K1_HBOX_BYTES;
+constexpr int K1_BOX_THREADS = 64;                      // two warps work on a box
 constexpr int K1_THREADS = 32 * 8;
-constexpr size_t K1_SMEM_BYTES = (size_t)K1_STAGES * K1_STAGE_BYTES + (size_t)K1_EBUFS * K1_EBUF_BYTES + 512;
+constexpr size_t K1_SMEM_BYTES = (size_t)K1_STAGES * K1_STAGE_BYTES + (size_t)K1_MVBUFS * K1_MVBUF_BYTES +
+                                 (size_t)K1_NRBUFS * K1_NRBUF_BYTES + 512;
 static_assert(K1_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 // Per-tile record (256 l x BN r), built on the host once (32 bytes).
@@ -52,9 +61,11 @@ struct ProjCtl {
   uint64_t empty[K1_STAGES];    // the MMAs reading a stage are done (both CTAs are told)
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];       // (even CTA) both CTAs' epilogues have drained an accumulator
-  uint64_t efull[K1_EBUFS];     // an M box and a V box have landed
-  uint64_t eready[K1_EBUFS];    // the epilogue has finished the four boxes in place
-  uint64_t eempty[K1_EBUFS];    // their stores have read them: the buffer is free
+  uint64_t efull[K1_MVBUFS][2]; // an M box and a V box have landed; one barrier per row half, so that
+                                // its waiters (that half's warps) see every one of its phases
+  uint64_t eready[K1_MVBUFS];   // the epilogue has finished M, V (in place) and N, R of a box
+  uint64_t eempty[K1_MVBUFS];   // the stores have read M and V: the buffer is free
+  uint64_t nrempty[K1_NRBUFS];  // the stores have read N and R: the buffer is free
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -82,8 +93,9 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
              const float* __restrict__ fast, Hyper hp, unsigned* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* tiles = smem_raw;
-  unsigned char* ebuf = tiles + (size_t)K1_STAGES * K1_STAGE_BYTES;
-  ProjCtl* ctl = reinterpret_cast<ProjCtl*>(ebuf + (size_t)K1_EBUFS * K1_EBUF_BYTES);
+  unsigned char* mvbuf = tiles + (size_t)K1_STAGES * K1_STAGE_BYTES;
+  unsigned char* nrbuf = mvbuf + (size_t)K1_MVBUFS * K1_MVBUF_BYTES;
+  ProjCtl* ctl = reinterpret_cast<ProjCtl*>(nrbuf + (size_t)K1_NRBUFS * K1_NRBUF_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = ptx::cluster_ctarank();          // 0: issues the MMAs; 1: its partner
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
@@ -98,11 +110,13 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
       ptx::mbar_init(ptx::smem_u32(&ctl->tmem_full[b]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[b]), 2 * 4);   // every epilogue warp of the pair
     }
-    for (int b = 0; b < K1_EBUFS; ++b) {
-      ptx::mbar_init(ptx::smem_u32(&ctl->efull[b]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl->eready[b]), K1_EPI_THREADS);
+    for (int b = 0; b < K1_MVBUFS; ++b) {
+      ptx::mbar_init(ptx::smem_u32(&ctl->efull[b][0]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl->efull[b][1]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl->eready[b]), K1_BOX_THREADS);
       ptx::mbar_init(ptx::smem_u32(&ctl->eempty[b]), 1);
     }
+    for (int b = 0; b < K1_NRBUFS; ++b) ptx::mbar_init(ptx::smem_u32(&ctl->nrempty[b]), 1);
     ctl->abort_flag = smem_ok ? 0 : 1;
     ptx::fence_barrier_init();
   }
@@ -116,7 +130,8 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
   ptx::tc_fence_after();
   volatile int* abort_flag = &ctl->abort_flag;
   const uint32_t tiles_u32 = ptx::smem_u32(tiles);
-  const uint32_t ebuf_u32 = ptx::smem_u32(ebuf);
+  const uint32_t mvbuf_u32 = ptx::smem_u32(mvbuf);
+  const uint32_t nrbuf_u32 = ptx::smem_u32(nrbuf);
 
   if (warp == 0) {
     // ------------------------------------------------------------ operand producer
@@ -195,7 +210,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
   } else if (warp == 2) {
     // ------------------------------------------------------------ epilogue loader: M and V boxes
     if (lane == 0 && smem_ok) {
-      int eb = 0; uint32_t ephase = 0; bool ok = true;
+      int mv = 0; uint32_t mvphase = 0; bool ok = true;
       ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
       for (int t = pair; t < total_tiles && ok; t += npairs) {
         const ProjTileDesc d = nd;
@@ -203,21 +218,22 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         const TcMaps* mp = &maps[d.slot];
         const int bn = d.bn_left & 0xffff;
         const int l0 = d.l0 + BM * (int)rank;
-        for (int c = 0; c < bn / K1_ECOLS; ++c) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->eempty[eb]), ephase ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t fb = ptx::smem_u32(&ctl->efull[eb]);
-          const uint32_t dst = ebuf_u32 + eb * K1_EBUF_BYTES;
-          ptx::mbar_expect_tx(fb, 2 * K1_FBOX_BYTES);
-          ptx::tma_load_2d(dst, &mp->em, fb, d.r0 + K1_ECOLS * c, l0);
-          ptx::tma_load_2d(dst + K1_FBOX_BYTES, &mp->ev, fb, d.r0 + K1_ECOLS * c, l0);
-          if (++eb == K1_EBUFS) { eb = 0; ephase ^= 1u; }
+        for (int b = 0; b < 2 * (bn / K1_ECOLS); ++b) {
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->eempty[mv]), mvphase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t fb = ptx::smem_u32(&ctl->efull[mv][b & 1]);
+          const uint32_t dst = mvbuf_u32 + mv * K1_MVBUF_BYTES;
+          const int j = d.r0 + K1_ECOLS * (b >> 1), row = l0 + K1_EROWS * (b & 1);
+          ptx::mbar_expect_tx(fb, K1_MVBUF_BYTES);
+          ptx::tma_load_2d(dst, &mp->em, fb, j, row);
+          ptx::tma_load_2d(dst + K1_FBOX_BYTES, &mp->ev, fb, j, row);
+          if (++mv == K1_MVBUFS) { mv = 0; mvphase ^= 1u; }
         }
       }
     }
   } else if (warp == 7) {
     // ------------------------------------------------------------ box storer
     if (lane == 0 && smem_ok) {
-      int eb = 0; uint32_t rphase = 0; bool ok = true;
+      int mv = 0; uint32_t mvphase = 0; bool ok = true;
       ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
       for (int t = pair; t < total_tiles && ok; t += npairs) {
         const ProjTileDesc d = nd;
@@ -225,20 +241,22 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         const TcMaps* mp = &maps[d.slot];
         const int bn = d.bn_left & 0xffff;
         const int l0 = d.l0 + BM * (int)rank;
-        for (int c = 0; c < bn / K1_ECOLS; ++c) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->eready[eb]), rphase, abort_flag)) { ok = false; break; }
-          if (l0 < d.L) {
-            const uint32_t src = ebuf_u32 + eb * K1_EBUF_BYTES;
-            const int j = d.r0 + K1_ECOLS * c;
-            ptx::tma_store_2d(&mp->em, src, j, l0);
-            ptx::tma_store_2d(&mp->ev, src + K1_FBOX_BYTES, j, l0);
-            ptx::tma_store_2d(&mp->en, src + 2 * K1_FBOX_BYTES, j, l0);
-            ptx::tma_store_2d(&mp->er, src + 2 * K1_FBOX_BYTES + K1_HBOX_BYTES, j, l0);
+        for (int b = 0; b < 2 * (bn / K1_ECOLS); ++b) {
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->eready[mv]), mvphase, abort_flag)) { ok = false; break; }
+          const int nr = b & 1;
+          const int j = d.r0 + K1_ECOLS * (b >> 1), row = l0 + K1_EROWS * nr;
+          if (row < d.L) {
+            const uint32_t src = mvbuf_u32 + mv * K1_MVBUF_BYTES, srn = nrbuf_u32 + nr * K1_NRBUF_BYTES;
+            ptx::tma_store_2d(&mp->em, src, j, row);
+            ptx::tma_store_2d(&mp->ev, src + K1_FBOX_BYTES, j, row);
+            ptx::tma_store_2d(&mp->en, srn, j, row);
+            ptx::tma_store_2d(&mp->er, srn + K1_HBOX_BYTES, j, row);
             ptx::bulk_commit_group();
-            ptx::bulk_wait_group_read<0>();              // the boxes have been read: the buffer is free
+            ptx::bulk_wait_group_read<0>();              // the boxes have been read: the buffers are free
           }
-          ptx::mbar_arrive(ptx::smem_u32(&ctl->eempty[eb]));
-          if (++eb == K1_EBUFS) { eb = 0; rphase ^= 1u; }
+          ptx::mbar_arrive(ptx::smem_u32(&ctl->eempty[mv]));
+          ptx::mbar_arrive(ptx::smem_u32(&ctl->nrempty[nr]));
+          if (++mv == K1_MVBUFS) { mv = 0; mvphase ^= 1u; }
         }
       }
       ptx::bulk_wait_group_all();
@@ -247,14 +265,22 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     // ------------------------------------------------------------ epilogue: Adam on R
     const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31
     const int row = quarter * 32 + lane;                // row of this CTA's half tile = TMEM lane
-    const uint32_t frow = (uint32_t)row * (K1_ECOLS * 4);   // fp32 boxes: 128-byte rows
-    const uint32_t fsw = (uint32_t)row & 7u;                //   128-byte swizzle: slot ^= row % 8
-    const uint32_t hrow = (uint32_t)row * (K1_ECOLS * 2);   // bf16 boxes: 64-byte rows
-    const uint32_t hsw = (uint32_t)(row >> 1) & 3u;         //   64-byte swizzle: slot ^= (row / 2) % 4
+    const int half = quarter >> 1;                      // boxes with b % 2 == half are this warp's
+    const int brow = row & (K1_EROWS - 1);              // row within the box
+    const uint32_t frow = (uint32_t)brow * (K1_ECOLS * 4);  // fp32 boxes: 128-byte rows
+    const uint32_t fsw = (uint32_t)brow & 7u;               //   128-byte swizzle: slot ^= row % 8
+    const uint32_t hrow = (uint32_t)brow * (K1_ECOLS * 2);  // bf16 boxes: 64-byte rows
+    const uint32_t hsw = (uint32_t)(brow >> 1) & 3u;        //   64-byte swizzle: slot ^= (row / 2) % 4
     const uint32_t tmem_empty0 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[0]), 0);
     const uint32_t tmem_empty1 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[1]), 0);
     int buf = 0; uint32_t bphase = 0;
-    int eb = 0; uint32_t ephase = 0;
+    // This warp's boxes have the indices half, half + 2, ...: the M/V buffer is index % 3, and each
+    // (buffer, half) barrier is used by every third of them.
+    int mv = half; int mvuse = 0; uint32_t mvphase = 0;
+    uint32_t nrphase = 0;                               // parity of this half's N/R buffer use
+    const uint32_t nrempty = ptx::smem_u32(&ctl->nrempty[half]);
+    unsigned char* nb = nrbuf + (size_t)half * K1_NRBUF_BYTES;
+    unsigned char* rb = nb + K1_HBOX_BYTES;
     const uint32_t tmem = ctl->tmem_base;
     bool ok = true;
     ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
@@ -280,11 +306,10 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive_cluster(te);
         }
-        if (!ptx::mbar_wait(ptx::smem_u32(&ctl->efull[eb]), ephase, abort_flag)) { ok = false; break; }
-        unsigned char* mb = ebuf + (size_t)eb * K1_EBUF_BYTES;
+        if (!ptx::mbar_wait(ptx::smem_u32(&ctl->efull[mv][half]), mvphase, abort_flag)) { ok = false; break; }
+        if (!ptx::mbar_wait(nrempty, nrphase ^ 1u, abort_flag)) { ok = false; break; }
+        unsigned char* mb = mvbuf + (size_t)mv * K1_MVBUF_BYTES;
         unsigned char* vb = mb + K1_FBOX_BYTES;
-        unsigned char* nb = vb + K1_FBOX_BYTES;
-        unsigned char* rb = nb + K1_HBOX_BYTES;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {                    // 8 columns at a time
           const uint32_t f0 = frow + (((uint32_t)(2 * q) ^ fsw) << 4);
@@ -316,8 +341,11 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         // hand the finished boxes to the storer: this thread's writes are visible to
         // the async proxy (TMA) before it arrives
         ptx::fence_proxy_async_smem();
-        ptx::mbar_arrive(ptx::smem_u32(&ctl->eready[eb]));
-        if (++eb == K1_EBUFS) { eb = 0; ephase ^= 1u; }
+        ptx::mbar_arrive(ptx::smem_u32(&ctl->eready[mv]));
+        nrphase ^= 1u;
+        mv += 2;                                         // this warp's next box is two further on
+        if (mv >= K1_MVBUFS) mv -= K1_MVBUFS;
+        if (++mvuse == K1_MVBUFS) { mvuse = 0; mvphase ^= 1u; }
       }
       if (ok && l < d.L) {
         // colpart[2 part][l] = partial ||N_l||^2, colpart[2 part + 1][l] = partial ||R_l||^2
