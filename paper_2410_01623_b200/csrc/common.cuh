@@ -42,8 +42,7 @@ struct MatDev {
   __nv_bfloat16* Nb;  // scratch of the tensor-core path: l x r bf16 N
   __nv_bfloat16* Rb;  //   "      l x r bf16 R
   __nv_bfloat16* Xb;  //   "      l x r bf16 X
-  float* colpart;     //   "      per (r-tile, l) partial sums of N^2 and R^2
-  float* gsq;         //   "      per-l sums of G^2
+  float* colpart;     //   "      per (r-tile, l) partial sums of N^2 and R^2, then per-l sums of G^2
   long long ld;
   int m, n, r;
   int left;           // 1: m <= n (left projection), 0: right projection

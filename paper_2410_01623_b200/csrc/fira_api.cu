@@ -76,7 +76,7 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
   size_t refresh_max = 0;
   L.offRt.assign(count, 0); L.offXt.assign(count, 0); L.offK.assign(count, 0); L.offPart.assign(count, 0);
   L.offNb.assign(count, 0); L.offRb.assign(count, 0); L.offXb.assign(count, 0);
-  L.offColpart.assign(count, 0); L.offGsq.assign(count, 0);
+  L.offColpart.assign(count, 0);
   for (int i = 0; i < count; ++i) {
     fira_matrix_desc d = descs[i];
     if (d.ld == 0) d.ld = d.n;
@@ -92,7 +92,6 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
       L.offRb[i] = w; w += align_up(ll * r * 2);
       L.offXb[i] = w; w += align_up(ll * r * 2);
       L.offColpart[i] = w; w += align_up(tc_colpart_floats(d) * 4);
-      L.offGsq[i] = w; w += align_up(tc_gsq_floats(d) * 4);
       L.offPart[i] = w; w += align_up(tc_part_floats(d) * 4);
     }
     refresh_max = std::max(refresh_max, refresh_bytes_per_matrix(d));
@@ -201,7 +200,6 @@ fira_status fira_init(fira_ctx** out, const fira_hparams* hp, const fira_matrix_
       mt.Rb = (__nv_bfloat16*)(c->work_base + L.offRb[i]);
       mt.Xb = (__nv_bfloat16*)(c->work_base + L.offXb[i]);
       mt.colpart = (float*)(c->work_base + L.offColpart[i]);
-      mt.gsq = (float*)(c->work_base + L.offGsq[i]);
       c->tc_list.push_back(i);
     }
   }

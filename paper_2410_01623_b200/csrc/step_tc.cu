@@ -5,9 +5,9 @@
 // l = unprojected index (columns of G when m <= n, rows otherwise), d = projected
 // index, Pi = the d x r projection.  Launches per step:
 //   k_tc_prep          bias factor sqrt(1-b2^s)/(1-b1^s) per matrix
-//   k_tc_gsq           partial sums of G^2 per l                          (for ||S||)
 //   k_tc_project       Rt = G^T Pi on the tensor cores; epilogue: M, V update (Eq. 2-3),
-//                      N (Eq. 4), bf16 copies of N and R, per-l partial ||N_l||^2, ||R_l||^2
+//                      N (Eq. 4), bf16 copies of N and R, per-l partial ||N_l||^2, ||R_l||^2;
+//                      ||G_l||^2 from the A stages in shared memory             (for ||S||)
 //   k_tc_colfactors    k_l (Eq. 11) and partial sums of ||S||^2 = sum_l k_l^2 (||G_l||^2 - ||R_l||^2)
 //   k_finalize         lambda, ||S_prev||, t (Eq. 12)
 //   k_tc_form_x        X = a_low N - a_res lambda k_l R  (bf16)
@@ -40,7 +40,6 @@ constexpr int BK = 64;            // k-block: 64 bf16 = 128 bytes
 constexpr int A_STAGE_BYTES = BM * BK * 2;       // 16 KiB: 128 rows x 64 bf16
 constexpr int CHUNK_BYTES = 64 * BK * 2;         // one 64 x 64 box: 8 KiB
 constexpr int TMEM_COLS = 512;
-constexpr int GSQ_ROWS = 128;     // rows per partial sum of G^2 (left orientation)
 
 struct TcMaps {
   CUtensorMap g1a;   // G, box for the projection product (2-D, or chunked 3-D: see encode_matrix_maps)
@@ -95,51 +94,6 @@ __global__ void k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict
   fast[2 * p] = bias;          // read by the projection epilogue
 }
 
-// Sums of G^2 per unprojected index.  Left: gsq[rb][col] over blocks of GSQ_ROWS rows
-// (one block = GSQ_ROWS rows x 2048 columns, 8 columns per thread); right: gsq[0][row],
-// one warp per row.  `start` counts blocks.
-__global__ void __launch_bounds__(256)
-k_tc_gsq(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
-         const int* __restrict__ start) {
-  const int p = find_matrix(start, nlist, blockIdx.x);
-  const MatDev& mt = mats[list[p]];
-  const int b = blockIdx.x - start[p];
-  const __nv_bfloat16* G = static_cast<const __nv_bfloat16*>(mt.G);
-  if (mt.left) {
-    const int ncb = (mt.n + 2047) / 2048;
-    const int rb = b / ncb, cb = b % ncb;
-    const int col = cb * 2048 + threadIdx.x * 8;
-    if (col >= mt.n) return;
-    float acc[8] = {};
-    const int row_end = min(mt.m, (rb + 1) * GSQ_ROWS);
-    for (int row = rb * GSQ_ROWS; row < row_end; ++row) {
-      const uint4 u = *reinterpret_cast<const uint4*>(G + (long long)row * mt.ld + col);
-      float g[8];
-      unpack8_bf16(u, g);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] = fmaf(g[e], g[e], acc[e]);
-    }
-    float* out = mt.gsq + (long long)rb * mt.l + col;
-    *reinterpret_cast<float4*>(out) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-    *reinterpret_cast<float4*>(out + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
-  } else {
-    const int row = b * 8 + (threadIdx.x >> 5);
-    if (row >= mt.m) return;
-    const int lane = threadIdx.x & 31;
-    float acc = 0.f;
-    for (int col = lane * 8; col < mt.n; col += 256) {
-      const uint4 u = *reinterpret_cast<const uint4*>(G + (long long)row * mt.ld + col);
-      float g[8];
-      unpack8_bf16(u, g);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc = fmaf(g[e], g[e], acc);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) mt.gsq[row] = acc;
-  }
-}
-
 // k_l and the partial sums of ||S||^2, 256 values of l per block.
 __global__ void __launch_bounds__(256)
 k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
@@ -157,8 +111,7 @@ k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, i
       nn += mt.colpart[(long long)(2 * q) * mt.l + l];
       rn += mt.colpart[(long long)(2 * q + 1) * mt.l + l];
     }
-    const int ngs = mt.left ? (mt.d + GSQ_ROWS - 1) / GSQ_ROWS : 1;
-    for (int q = 0; q < ngs; ++q) gs += mt.gsq[(long long)q * mt.l + l];
+    for (int q = 2 * nparts; q < 4 * nparts; ++q) gs += mt.colpart[(long long)q * mt.l + l];   // ||G_l||^2 in parts
     const float k = sqrtf(nn) / (sqrtf(rn) + hp.eps);
     mt.kvec[l] = k;
     contrib = k * k * fmaxf(gs - rn, 0.f);
@@ -267,7 +220,6 @@ struct TcPlan {
   int nlist = 0;
   const int* k1_start = nullptr; int k1_tiles = 0;
   const int* k2_start = nullptr; int k2_tiles = 0;
-  const int* gsq_start = nullptr; int gsq_blocks = 0;
   const int* col_start = nullptr; int col_blocks = 0;
   const int* row_start = nullptr; int rows_total = 0;
   const int* npart = nullptr;
@@ -285,12 +237,7 @@ bool tc_supported(const fira_matrix_desc& d) {
 
 size_t tc_colpart_floats(const fira_matrix_desc& d) {
   const size_t l = std::max(d.m, d.n);
-  return 2 * (size_t)(d.r / host_tile_bn(d.r)) * l;
-}
-
-size_t tc_gsq_floats(const fira_matrix_desc& d) {
-  const size_t l = std::max(d.m, d.n), dd = std::min(d.m, d.n);
-  return (d.m <= d.n ? (dd + GSQ_ROWS - 1) / GSQ_ROWS : 1) * l;
+  return 4 * (size_t)(d.r / host_tile_bn(d.r)) * l;   // N^2 and R^2 per r-tile, then two partial G^2 per r-tile
 }
 
 size_t tc_part_floats(const fira_matrix_desc& d) { return ((size_t)std::max(d.m, d.n) + 255) / 256; }
@@ -341,14 +288,12 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
   c->tc = pl;
   cudaDeviceGetAttribute(&pl->num_sms, cudaDevAttrMultiProcessorCount, c->device);
   const std::vector<int>& lst = c->tc_list;
-  std::vector<int> k1{0}, k2{0}, gs{0}, cs{0}, rs{0}, np;
+  std::vector<int> k1{0}, k2{0}, cs{0}, rs{0}, np;
   for (int i : lst) {
     const MatDev& mt = c->mats[i];
     const int bn = host_tile_bn(mt.r);
     k1.push_back(k1.back() + ((mt.l + 2 * BM - 1) / (2 * BM)) * (mt.r / bn));
     k2.push_back(k2.back() + ((mt.m + 2 * BM - 1) / (2 * BM)) * ((mt.n + BN_MAX - 1) / BN_MAX));
-    const int gblocks = mt.left ? ((mt.d + GSQ_ROWS - 1) / GSQ_ROWS) * ((mt.n + 2047) / 2048) : (mt.m + 7) / 8;
-    gs.push_back(gs.back() + gblocks);
     const int cb = (mt.l + 255) / 256;
     cs.push_back(cs.back() + cb);
     rs.push_back(rs.back() + mt.l);
@@ -359,12 +304,11 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
     ints.insert(ints.end(), v.begin(), v.end());
     return o;
   };
-  const size_t o_list = push_block(lst), o_k1 = push_block(k1), o_k2 = push_block(k2), o_gs = push_block(gs),
+  const size_t o_list = push_block(lst), o_k1 = push_block(k1), o_k2 = push_block(k2),
                o_cs = push_block(cs), o_rs = push_block(rs), o_np = push_block(np);
   pl->list = c->ints_dev + o_list; pl->nlist = (int)lst.size();
   pl->k1_start = c->ints_dev + o_k1; pl->k1_tiles = k1.back();
   pl->k2_start = c->ints_dev + o_k2; pl->k2_tiles = k2.back();
-  pl->gsq_start = c->ints_dev + o_gs; pl->gsq_blocks = gs.back();
   pl->col_start = c->ints_dev + o_cs; pl->col_blocks = cs.back();
   pl->row_start = c->ints_dev + o_rs; pl->rows_total = rs.back();
   pl->npart = c->ints_dev + o_np;
@@ -401,7 +345,8 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
           ProjTileDesc d;
           d.colpart = mt.colpart; d.slot = (int)q; d.l0 = a * 2 * BM; d.r0 = b * bn;
           d.nkb = (mt.d + BK - 1) / BK; d.L = mt.l;
-          d.bn_left = bn | (mt.left ? (int)0x80000000 : 0) | ((mt.left && mt.n % 64 == 0) ? PROJ_A_CHUNKED : 0);
+          d.bn_left = bn | ((mt.r / bn) << 16) | (mt.left ? (int)0x80000000 : 0) |
+                      ((mt.left && mt.n % 64 == 0) ? PROJ_A_CHUNKED : 0);
           tp.push_back(d);
         }
     }
@@ -441,10 +386,10 @@ fira_status tc_update_pointers(fira_ctx* c) {
 }
 
 int tc_phase_names(const char** out) {
-  static const char* names[7] = {"k_tc_prep", "k_tc_gsq", "k_tc_project", "k_tc_colfactors",
+  static const char* names[6] = {"k_tc_prep", "k_tc_project", "k_tc_colfactors",
                                  "k_finalize(tc)", "k_tc_form_x", "k_tc_back_project"};
-  for (int i = 0; i < 7; ++i) out[i] = names[i];
-  return 7;
+  for (int i = 0; i < 6; ++i) out[i] = names[i];
+  return 6;
 }
 
 int launch_tc_step(fira_ctx* c, const Hyper& hp) {
@@ -464,8 +409,6 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   const MatDev* mats = c->mats_dev;
   k_tc_prep<<<(pl->nlist + 127) / 128, 128, 0, st>>>(mats, pl->list, pl->nlist, hp, pl->fast_dev);
   tm->mark(st);
-  k_tc_gsq<<<pl->gsq_blocks, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->gsq_start);
-  tm->mark(st);
   // both tensor kernels: clusters of two CTAs, at most one CTA per SM
   k_tc_project<<<2 * std::min(pl->k1_tiles, pl->num_sms / 2), K1_THREADS, K1_SMEM_BYTES, st>>>(
       pl->maps_dev, pl->td1_dev, pl->k1_tiles, pl->fast_dev, hp, c->status_dev);
@@ -480,7 +423,7 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   k_tc_back_project<<<2 * std::min(pl->k2_tiles, pl->num_sms / 2), K2_THREADS, K2_SMEM_BYTES, st>>>(
       pl->maps_dev, pl->td2_dev, pl->k2_tiles, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);
-  return 7;
+  return 6;
 }
 
 }  // namespace fira

@@ -15,7 +15,6 @@ bool tc_supported(const fira_matrix_desc& d);
 // partial sums of ||S||^2.
 size_t tc_colpart_floats(const fira_matrix_desc& d);
 size_t tc_part_floats(const fira_matrix_desc& d);
-size_t tc_gsq_floats(const fira_matrix_desc& d);
 // Bytes of this engine's device-resident tables (tensor maps, tile records) for a matrix list.
 size_t tc_tables_bytes(const fira_hparams& hp, const fira_matrix_desc* descs, int count);
 // Appends this engine's schedule arrays to `ints` (host image of the device int

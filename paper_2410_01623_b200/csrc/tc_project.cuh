@@ -3,7 +3,8 @@
 //
 //   Rt[l][j] = sum_d G(d,l) Pi[d][j]          (R = P^T G, stored with the rank index contiguous)
 //   M <- b1 M + (1-b1) R,  V <- b2 V + (1-b2) R^2,  N = bias M / (sqrt V + eps)     (Eq. 2-4)
-//   writes M, V (fp32), N, R (bf16) and the per-l partial sums ||N_l||^2, ||R_l||^2
+//   writes M, V (fp32), N, R (bf16), the per-l partial sums ||N_l||^2, ||R_l||^2 and, from the
+//   tiles of the first r range, the per-l sums ||G_l||^2 (needed for ||S||)
 //
 // CTA pairs (clusters of two, one CTA per SM) walk tiles of 256 l x BN r with
 // tcgen05.mma.cta_group::2.  A = G: for m <= n an MN-major operand (G is [d][l], l
@@ -26,8 +27,15 @@
 // Small boxes leave room for five operand stages: the time from a stage's release to its next
 // MMA is several thousand cycles, which four stages do not cover.
 //
+// ||G_l||^2: G passes through shared memory as the A operand anyway.  The r / BN tiles that share a
+// panel of G split its k-blocks between them (tile `part` takes k-blocks part, part + r / BN, ...):
+// four more warps square and sum such an A stage while its MMAs run (the MMA issuer tells both CTAs
+// when the stage has landed; the producer waits for the warps before it overwrites the stage, on
+// those k-blocks only).  This replaces a separate pass over G in HBM.
+//
 // Warp roles: 0 operand producer (TMA); 1 MMA issuer (even CTA only) and TMEM owner;
-// 2 epilogue loader (TMA); 3-6 epilogue; 7 one thread that stores the finished boxes.
+// 2 epilogue loader (TMA); 3-6 epilogue; 7 one thread that stores the finished boxes;
+// 8-11 sums of G^2.
 constexpr int K1_STAGES = 5;
 constexpr int K1_STAGE_BYTES = 2 * A_STAGE_BYTES;       // A: 128 l x 64 d, B half: 128 r x 64 d
 constexpr int K1_ECOLS = 32;                            // columns per epilogue box
@@ -39,7 +47,8 @@ constexpr int K1_NRBUFS = 2;                            // {N box, R box}, one p
 constexpr int K1_MVBUF_BYTES = 2 * K1_FBOX_BYTES;
 constexpr int K1_NRBUF_BYTES = 2 * K1_HBOX_BYTES;
 constexpr int K1_BOX_THREADS = 64;                      // two warps work on a box
-constexpr int K1_THREADS = 32 * 8;
+constexpr int K1_GSQ_WARPS = 4;
+constexpr int K1_THREADS = 32 * (8 + K1_GSQ_WARPS);
 constexpr size_t K1_SMEM_BYTES = (size_t)K1_STAGES * K1_STAGE_BYTES + (size_t)K1_MVBUFS * K1_MVBUF_BYTES +
                                  (size_t)K1_NRBUFS * K1_NRBUF_BYTES + 512;
 static_assert(K1_SMEM_BYTES <= 227 * 1024, "shared memory budget");
@@ -50,7 +59,7 @@ struct ProjTileDesc {
   int slot;            // index into the tensor-map table and the fast-scalar table
   int l0, r0;          // first unprojected index / first rank index of the tile
   int nkb;             // k-blocks: ceil(d / 64)
-  int bn_left;         // BN (128 or 256); bit 31: left orientation; bit 30: G comes as one chunked box
+  int bn_left;         // bits 0-15: BN (128 or 256); 16-23: r / BN; 30: G comes as one chunked box; 31: left
   int L;               // number of unprojected indices of the matrix
 };
 static_assert(sizeof(ProjTileDesc) == 32, "ProjTileDesc layout");
@@ -61,6 +70,8 @@ struct ProjCtl {
   uint64_t empty[K1_STAGES];    // the MMAs reading a stage are done (both CTAs are told)
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];       // (even CTA) both CTAs' epilogues have drained an accumulator
+  uint64_t afull[K1_STAGES];    // told by the MMA issuer to both CTAs: a stage that the G^2 warps read has landed
+  uint64_t gdone[K1_STAGES];    // the G^2 warps have read that stage
   uint64_t efull[K1_MVBUFS][2]; // an M box and a V box have landed; one barrier per row half, so that
                                 // its waiters (that half's warps) see every one of its phases
   uint64_t eready[K1_MVBUFS];   // the epilogue has finished M, V (in place) and N, R of a box
@@ -105,6 +116,8 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     for (int s = 0; s < K1_STAGES; ++s) {
       ptx::mbar_init(ptx::smem_u32(&ctl->full[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctl->empty[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl->afull[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl->gdone[s]), K1_GSQ_WARPS);
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(ptx::smem_u32(&ctl->tmem_full[b]), 1);
@@ -137,6 +150,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     // ------------------------------------------------------------ operand producer
     if (lane == 0 && smem_ok) {
       int stage = 0; uint32_t phase = 0; bool ok = true;
+      uint32_t gmask = 0, gphase = 0;   // per stage: its occupant is read by the G^2 warps / parity of that wait
       ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
       for (int t = pair; t < total_tiles && ok; t += npairs) {
         const ProjTileDesc d = nd;
@@ -146,9 +160,16 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         const int bn = d.bn_left & 0xffff;
         const int l0 = d.l0 + BM * (int)rank;             // this CTA's unprojected indices
         const int rb0 = d.r0 + (bn / 2) * (int)rank;      // this CTA's half of the rank range
+        const int nparts = (d.bn_left >> 16) & 0xff;
+        int gturn = d.r0 / bn;                            // next k-block that the G^2 warps read
         const uint32_t bytes = 2 * (A_STAGE_BYTES + (bn / 2) * BK * 2);   // both CTAs together
         for (int kb = 0; kb < d.nkb; ++kb) {
           if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+          if ((gmask >> stage) & 1u) {                     // the previous occupant is still being squared
+            if (!ptx::mbar_wait(ptx::smem_u32(&ctl->gdone[stage]), (gphase >> stage) & 1u, abort_flag)) { ok = false; break; }
+            gphase ^= 1u << stage;
+          }
+          if (kb == gturn) { gturn += nparts; gmask |= 1u << stage; } else { gmask &= ~(1u << stage); }
           // all boxes of the pair complete on the even CTA's barrier
           const uint32_t fb = ptx::map_to_cta(ptx::smem_u32(&ctl->full[stage]), 0);
           const uint32_t sa = tiles_u32 + stage * K1_STAGE_BYTES, sb = sa + A_STAGE_BYTES;
@@ -184,11 +205,17 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         const int left = d.bn_left < 0;
         const int bn = d.bn_left & 0xffff;
         const uint32_t idesc = ptx::make_idesc_bf16(2 * BM, bn, left, 1);
+        const int nparts = (d.bn_left >> 16) & 0xff;
+        int gturn = d.r0 / bn;                            // next k-block that the G^2 warps read
         if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->tmem_empty[buf]), bphase ^ 1u, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t dcol = tmem + buf * BN_MAX;
         for (int kb = 0; kb < d.nkb; ++kb) {
           if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+          if (kb == gturn) {                               // the G^2 warps may read this stage now
+            gturn += nparts;
+            ptx::mbar_arrive(ptx::smem_u32(&ctl->afull[stage]));     // (passed on to the odd CTA by a G^2 warp)
+          }
           ptx::tc_fence_after();
           const uint32_t sa = tiles_u32 + stage * K1_STAGE_BYTES, sb = sa + A_STAGE_BYTES;
 #pragma unroll
@@ -227,6 +254,84 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           ptx::tma_load_2d(dst, &mp->em, fb, j, row);
           ptx::tma_load_2d(dst + K1_FBOX_BYTES, &mp->ev, fb, j, row);
           if (++mv == K1_MVBUFS) { mv = 0; mvphase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp >= 8) {
+    // ------------------------------------------------------------ sums of G^2 over the A stages
+    if (smem_ok) {
+      const int w = warp - 8;
+      const int khalf = w >> 1;                          // left: d rows 32 khalf .. + 31 of a stage
+      int base = 0; uint32_t aphase = 0; bool ok = true;  // stage of the tile's first k-block; parities of afull
+      ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
+      for (int t = pair; t < total_tiles && ok; t += npairs) {
+        const ProjTileDesc d = nd;
+        if (t + npairs < total_tiles) nd = load_desc(tdesc, t + npairs);
+        const int left = d.bn_left < 0;
+        const int bn = d.bn_left & 0xffff;
+        const int nparts = (d.bn_left >> 16) & 0xff, part = d.r0 / bn;
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int kb = part; kb < d.nkb; kb += nparts) {  // this tile's share of the panel's k-blocks
+          const int stage = (base + kb) % K1_STAGES;
+          // afull is used for these k-blocks only and every use is awaited here: its parity cannot alias
+          if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->afull[stage]), (aphase >> stage) & 1u, abort_flag)) { ok = false; break; }
+          aphase ^= 1u << stage;
+          if (rank == 0 && w == 0 && lane == 0)            // a remote arrival would hold up the MMA issuer
+            ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&ctl->afull[stage]), 1));
+          {
+            const unsigned char* sa = tiles + (size_t)stage * K1_STAGE_BYTES;
+            if (left) {
+              // chunk w % 2: [64 d rows][64 l], 128-byte rows, 16-byte slot ^= row % 8.
+              // lane: slot lane % 8 (8 values of l), rows 32 khalf + lane / 8, + 4, ...
+              const unsigned char* ch = sa + (w & 1) * CHUNK_BYTES;
+              const int slot = lane & 7;
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int k = 32 * khalf + (lane >> 3) + 4 * i;
+                const uint4 u = *reinterpret_cast<const uint4*>(ch + k * 128 + ((slot ^ (k & 7)) << 4));
+                float g[8];
+                unpack8_bf16(u, g);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = fmaf(g[e], g[e], acc[e]);
+              }
+            } else {
+              // [128 l rows][64 d], 128-byte rows, slot ^= row % 8: one row per thread
+              const int row = 32 * w + lane;
+              const unsigned char* rp = sa + row * 128;
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                const uint4 u = *reinterpret_cast<const uint4*>(rp + ((q ^ (row & 7)) << 4));
+                float g[8];
+                unpack8_bf16(u, g);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[0] = fmaf(g[e], g[e], acc[0]);
+              }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->gdone[stage]));
+          }
+        }
+        base = (base + d.nkb) % K1_STAGES;
+        if (ok) {
+          // slots after the 2 nparts partial sums of N^2 and R^2: [2 part + khalf][l]
+          float* gs = d.colpart + (long long)(2 * nparts + 2 * part) * d.L;
+          const int lbase = d.l0 + BM * (int)rank;
+          if (left) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 8);
+              acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);
+            }
+            const int l = lbase + 64 * (w & 1) + 8 * lane;
+            if (lane < 8 && l < d.L) {                    // L is a multiple of 8
+              float* o = gs + (long long)khalf * d.L + l;
+              *reinterpret_cast<float4*>(o) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+              *reinterpret_cast<float4*>(o + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+            }
+          } else {
+            const int l = lbase + 32 * w + lane;
+            if (l < d.L) { gs[l] = acc[0]; gs[d.L + l] = 0.f; }
+          }
         }
       }
     }

@@ -50,6 +50,27 @@ def test_first_step_moments_expose_the_projection_product(shape, r):
     tr.assert_ok()
 
 
+@pytest.mark.parametrize("shape,r", [((512, 768), 128), ((768, 512), 128), ((1024, 1280), 512), ((1280, 1024), 512)])
+def test_axis_projection_pins_the_sums_of_g_squared(shape, r):
+    """With coordinate axes as the projection (orthonormal and exact in bf16) the column identity
+    ||S_l||^2 = ||G_l||^2 - ||R_l||^2 is exact, so the remembered norm checks the fused sums of G^2
+    (every k-block, both CTAs of a pair, every r-tile's share) far below the bf16 tolerance."""
+    m, n = shape
+    g = torch.Generator().manual_seed(m + r)
+    hp = fb.make_hparams(lr=1e-2, alpha=0.25, gamma=1.01)
+    W0 = [(torch.randn(m, n, generator=g) * 0.02).to(torch.bfloat16)]
+    tr = Trajectory([shape], r, torch.bfloat16, hp, W0)
+    d = min(m, n)
+    P = torch.zeros(d, r)
+    P[torch.randperm(d, generator=g)[:r], torch.arange(r)] = 1.0
+    tr.f.set_projection(0, P.to(torch.bfloat16).cuda())
+    for s in range(2):
+        tr.step([(torch.randn(m, n, generator=g) * torch.exp(torch.randn(n, generator=g))[None, :]).to(torch.bfloat16)])
+        assert tr.f.diagnostics(0)["norm_prev"] == pytest.approx(tr.st[0].prev_norm, rel=2e-4)
+    assert tr.f.diagnostics(0)["engine"] == 1
+    tr.assert_ok()
+
+
 def test_mixed_list_left_right_square_with_limiter():
     shapes = [(512, 1376), (1376, 512), (512, 512), (256, 2048), (640, 264)]
     tr = _case(shapes, [128, 128, 128, 256, 128], steps=6, seed=17, spike=(4,))
