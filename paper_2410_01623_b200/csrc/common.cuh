@@ -43,6 +43,9 @@ struct MatDev {
   __nv_bfloat16* Rb;  //   "      l x r bf16 R
   __nv_bfloat16* Xb;  //   "      l x r bf16 X
   float* colpart;     //   "      per (r-tile, l) partial sums of N^2 and R^2, then per-l sums of G^2
+  __nv_bfloat16* Gs;  //   "      copies of G and W with 16-byte aligned rows (pitch lds), only when the
+  __nv_bfloat16* Ws;  //          caller's rows are not (odd widths): TMA needs aligned rows
+  long long lds;
   long long ld;
   int m, n, r;
   int left;           // 1: m <= n (left projection), 0: right projection

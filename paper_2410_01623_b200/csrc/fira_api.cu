@@ -76,7 +76,7 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
   size_t refresh_max = 0;
   L.offRt.assign(count, 0); L.offXt.assign(count, 0); L.offK.assign(count, 0); L.offPart.assign(count, 0);
   L.offNb.assign(count, 0); L.offRb.assign(count, 0); L.offXb.assign(count, 0);
-  L.offColpart.assign(count, 0);
+  L.offColpart.assign(count, 0); L.offGs.assign(count, 0); L.offWs.assign(count, 0);
   for (int i = 0; i < count; ++i) {
     fira_matrix_desc d = descs[i];
     if (d.ld == 0) d.ld = d.n;
@@ -93,6 +93,11 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
       L.offXb[i] = w; w += align_up(ll * r * 2);
       L.offColpart[i] = w; w += align_up(tc_colpart_floats(d) * 4);
       L.offPart[i] = w; w += align_up(tc_part_floats(d) * 4);
+      const size_t lds = (size_t)tc_staging_pitch(d);
+      if (lds) {
+        L.offGs[i] = w; w += align_up((size_t)d.m * lds * 2);
+        L.offWs[i] = w; w += align_up((size_t)d.m * lds * 2);
+      }
     }
     refresh_max = std::max(refresh_max, refresh_bytes_per_matrix(d));
   }
@@ -200,6 +205,11 @@ fira_status fira_init(fira_ctx** out, const fira_hparams* hp, const fira_matrix_
       mt.Rb = (__nv_bfloat16*)(c->work_base + L.offRb[i]);
       mt.Xb = (__nv_bfloat16*)(c->work_base + L.offXb[i]);
       mt.colpart = (float*)(c->work_base + L.offColpart[i]);
+      mt.lds = tc_staging_pitch(c->descs[i]);
+      if (mt.lds) {
+        mt.Gs = (__nv_bfloat16*)(c->work_base + L.offGs[i]);
+        mt.Ws = (__nv_bfloat16*)(c->work_base + L.offWs[i]);
+      }
       c->tc_list.push_back(i);
     }
   }

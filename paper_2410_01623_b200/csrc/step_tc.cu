@@ -94,6 +94,26 @@ __global__ void k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict
   fast[2 * p] = bias;          // read by the projection epilogue
 }
 
+// Copies between the caller's G and W and the copies with aligned rows, one block per row of a
+// staged matrix.  dir 0: G -> Gs, W -> Ws; dir 1: Ws -> W.  The caller's rows start on 2-byte
+// boundaries only, so elements move one at a time.
+__global__ void __launch_bounds__(256)
+k_tc_stage(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+           const int* __restrict__ row_start, int dir) {
+  const int p = find_matrix(row_start, nlist, blockIdx.x);
+  const MatDev& mt = mats[list[p]];
+  const long long i = blockIdx.x - row_start[p];
+  const unsigned short* g = static_cast<const unsigned short*>(mt.G) + i * mt.ld;
+  unsigned short* w = static_cast<unsigned short*>(mt.W) + i * mt.ld;
+  unsigned short* gs = reinterpret_cast<unsigned short*>(mt.Gs) + i * mt.lds;
+  unsigned short* ws = reinterpret_cast<unsigned short*>(mt.Ws) + i * mt.lds;
+  if (dir == 0) {
+    for (int j = threadIdx.x; j < mt.n; j += 256) { gs[j] = g[j]; ws[j] = w[j]; }
+  } else {
+    for (int j = threadIdx.x; j < mt.n; j += 256) w[j] = ws[j];
+  }
+}
+
 // k_l and the partial sums of ||S||^2, 256 values of l per block.
 __global__ void __launch_bounds__(256)
 k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
@@ -222,6 +242,7 @@ struct TcPlan {
   const int* k2_start = nullptr; int k2_tiles = 0;
   const int* col_start = nullptr; int col_blocks = 0;
   const int* row_start = nullptr; int rows_total = 0;
+  const int* stage_list = nullptr; const int* stage_start = nullptr; int nstage = 0, stage_rows = 0;
   const int* npart = nullptr;
   ProjTileDesc* td1_dev = nullptr;   // per-tile records of the projection
   BackTileDesc* td2_dev = nullptr;   // per-tile records of the back-projection
@@ -231,8 +252,13 @@ struct TcPlan {
 };
 
 bool tc_supported(const fira_matrix_desc& d) {
+  return d.dtype == FIRA_BF16 && d.r % 128 == 0 && d.m >= 256 && d.n >= 256;
+}
+
+long long tc_staging_pitch(const fira_matrix_desc& d) {
   const long long ld = d.ld ? d.ld : d.n;
-  return d.dtype == FIRA_BF16 && d.r % 128 == 0 && d.m >= 256 && d.n >= 256 && d.n % 8 == 0 && ld % 8 == 0;
+  if (d.n % 8 == 0 && ld % 8 == 0) return 0;
+  return ((long long)d.n + 63) / 64 * 64;
 }
 
 size_t tc_colpart_floats(const fira_matrix_desc& d) {
@@ -260,7 +286,9 @@ size_t tc_tables_bytes(const fira_hparams& hp, const fira_matrix_desc* descs, in
          align_up(sizeof(BackTileDesc) * tiles2) + align_up(sizeof(ProjTileDesc) * tiles1);
 }
 
-static bool encode_matrix_maps(const MatDev& mt, TcMaps& mp, bool only_g) {
+static bool encode_matrix_maps(const MatDev& mt0, TcMaps& mp, bool only_g) {
+  MatDev mt = mt0;
+  if (mt.Gs) { mt.G = mt.Gs; mt.W = mt.Ws; mt.ld = mt.lds; }   // the kernels see the aligned copies
   // G is [m][n]: left -> 64 d rows of two 64-wide chunks of l (one chunked box when n % 64 == 0,
   // else two plain boxes); right -> box of 64 d x 128 l rows
   if (mt.left && mt.n % 64 == 0) {
@@ -288,9 +316,10 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
   c->tc = pl;
   cudaDeviceGetAttribute(&pl->num_sms, cudaDevAttrMultiProcessorCount, c->device);
   const std::vector<int>& lst = c->tc_list;
-  std::vector<int> k1{0}, k2{0}, cs{0}, rs{0}, np;
+  std::vector<int> k1{0}, k2{0}, cs{0}, rs{0}, np, sl, ss{0};
   for (int i : lst) {
     const MatDev& mt = c->mats[i];
+    if (mt.Gs) { sl.push_back(i); ss.push_back(ss.back() + mt.m); }
     const int bn = host_tile_bn(mt.r);
     k1.push_back(k1.back() + ((mt.l + 2 * BM - 1) / (2 * BM)) * (mt.r / bn));
     k2.push_back(k2.back() + ((mt.m + 2 * BM - 1) / (2 * BM)) * ((mt.n + BN_MAX - 1) / BN_MAX));
@@ -305,13 +334,16 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
     return o;
   };
   const size_t o_list = push_block(lst), o_k1 = push_block(k1), o_k2 = push_block(k2),
-               o_cs = push_block(cs), o_rs = push_block(rs), o_np = push_block(np);
+               o_cs = push_block(cs), o_rs = push_block(rs), o_np = push_block(np),
+               o_sl = push_block(sl), o_ss = push_block(ss);
   pl->list = c->ints_dev + o_list; pl->nlist = (int)lst.size();
   pl->k1_start = c->ints_dev + o_k1; pl->k1_tiles = k1.back();
   pl->k2_start = c->ints_dev + o_k2; pl->k2_tiles = k2.back();
   pl->col_start = c->ints_dev + o_cs; pl->col_blocks = cs.back();
   pl->row_start = c->ints_dev + o_rs; pl->rows_total = rs.back();
   pl->npart = c->ints_dev + o_np;
+  pl->stage_list = c->ints_dev + o_sl; pl->stage_start = c->ints_dev + o_ss;
+  pl->nstage = (int)sl.size(); pl->stage_rows = ss.back();
   pl->maps.resize(lst.size());
   char* tab = c->tc_maps_dev;
   pl->maps_dev = reinterpret_cast<TcMaps*>(tab); tab += align_up(sizeof(TcMaps) * lst.size());
@@ -386,10 +418,10 @@ fira_status tc_update_pointers(fira_ctx* c) {
 }
 
 int tc_phase_names(const char** out) {
-  static const char* names[6] = {"k_tc_prep", "k_tc_project", "k_tc_colfactors",
-                                 "k_finalize(tc)", "k_tc_form_x", "k_tc_back_project"};
-  for (int i = 0; i < 6; ++i) out[i] = names[i];
-  return 6;
+  static const char* names[8] = {"k_tc_stage(in)", "k_tc_prep", "k_tc_project", "k_tc_colfactors",
+                                 "k_finalize(tc)", "k_tc_form_x", "k_tc_back_project", "k_tc_stage(out)"};
+  for (int i = 0; i < 8; ++i) out[i] = names[i];
+  return 8;
 }
 
 int launch_tc_step(fira_ctx* c, const Hyper& hp) {
@@ -407,6 +439,8 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   }
   PhaseTimer* tm = &c->timer;
   const MatDev* mats = c->mats_dev;
+  if (pl->nstage) k_tc_stage<<<pl->stage_rows, 256, 0, st>>>(mats, pl->stage_list, pl->nstage, pl->stage_start, 0);
+  tm->mark(st);
   k_tc_prep<<<(pl->nlist + 127) / 128, 128, 0, st>>>(mats, pl->list, pl->nlist, hp, pl->fast_dev);
   tm->mark(st);
   // both tensor kernels: clusters of two CTAs, at most one CTA per SM
@@ -423,7 +457,9 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   k_tc_back_project<<<2 * std::min(pl->k2_tiles, pl->num_sms / 2), K2_THREADS, K2_SMEM_BYTES, st>>>(
       pl->maps_dev, pl->td2_dev, pl->k2_tiles, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);
-  return 6;
+  if (pl->nstage) k_tc_stage<<<pl->stage_rows, 256, 0, st>>>(mats, pl->stage_list, pl->nstage, pl->stage_start, 1);
+  tm->mark(st);
+  return pl->nstage ? 8 : 6;
 }
 
 }  // namespace fira

@@ -8,9 +8,12 @@ struct fira_ctx;
 
 namespace fira {
 
-// Whether the tensor-core kernels can take this matrix (shape and alignment rules
-// of the TMA loads); otherwise it runs on the fp32 CUDA-core kernels.
+// Whether the tensor-core kernels can take this matrix (type, rank and size rules of the
+// tiles); otherwise it runs on the fp32 CUDA-core kernels.
 bool tc_supported(const fira_matrix_desc& d);
+// Row pitch (elements) of the aligned copies of G and W that the tensor-core path makes when the
+// caller's rows are not 16-byte aligned (odd widths or pitches); 0 when TMA can read them in place.
+long long tc_staging_pitch(const fira_matrix_desc& d);
 // Scratch sizes (floats) of the per-(r-tile, l) column partial sums and of the
 // partial sums of ||S||^2.
 size_t tc_colpart_floats(const fira_matrix_desc& d);
@@ -26,7 +29,7 @@ fira_status tc_update_pointers(fira_ctx* c);
 // Enqueues the tensor-core phases for the matrices of the tc list; returns the
 // number of launches (negative: error, message set).
 int launch_tc_step(fira_ctx* c, const Hyper& hp);
-// Names of this engine's kernels in launch order (at most 8).
+// Names of this engine's phases in launch order (8).
 int tc_phase_names(const char** out);
 
 }  // namespace fira

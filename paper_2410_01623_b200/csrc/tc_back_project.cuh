@@ -261,7 +261,7 @@ k_tc_back_project(const TcMaps* __restrict__ maps, const BackTileDesc* __restric
       if (left) {
         if (tid_g < K2_KS_GROUP / 4) {
           const int box = K2_GROUPS * (tid_g >> 3) + g;  // 8 float4 per box of 32 columns
-          const int j = d.j0 + K2_ECOLS * box + 4 * (tid_g & 7);   // n is a multiple of 8
+          const int j = d.j0 + K2_ECOLS * box + 4 * (tid_g & 7);   // (the k table is padded to 64 floats)
           const float4 kv = (j < d.n) ? *reinterpret_cast<const float4*>(d.kvec + j) : make_float4(0.f, 0.f, 0.f, 0.f);
           *reinterpret_cast<float4*>(ks + 4 * tid_g) = kv;
         }

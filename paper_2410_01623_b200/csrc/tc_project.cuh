@@ -323,10 +323,15 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
               acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);
             }
             const int l = lbase + 64 * (w & 1) + 8 * lane;
-            if (lane < 8 && l < d.L) {                    // L is a multiple of 8
+            if (lane < 8 && l < d.L) {
               float* o = gs + (long long)khalf * d.L + l;
-              *reinterpret_cast<float4*>(o) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-              *reinterpret_cast<float4*>(o + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+              if ((d.L & 3) == 0 && l + 8 <= d.L) {      // rows of the table stay 16-byte aligned
+                *reinterpret_cast<float4*>(o) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                *reinterpret_cast<float4*>(o + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+              } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) if (l + e < d.L) o[e] = acc[e];
+              }
             }
           } else {
             const int l = lbase + 32 * w + lane;

@@ -23,11 +23,12 @@ def test_llama_7b_layer_two_steps():
         assert d["norm_prev"] == pytest.approx(tr.st[i].prev_norm, rel=2e-2)
 
 
-def test_llama_1b_layer_odd_width_falls_back_to_cuda_cores():
-    """2048 x 5461: rows of 10922 bytes cannot be addressed by TMA, so the matrices of
-    that shape run on the fp32 CUDA-core kernels; the square ones and 5461 x 2048 (rows of
-    4096 bytes) stay on the tensor cores."""
+def test_llama_1b_layer_odd_width_on_tensor_cores():
+    """2048 x 5461: rows of 10922 bytes cannot be addressed by TMA, so the library works on
+    copies with an aligned pitch; every matrix of the layer runs on the tensor cores."""
     wl = wk.workload("llama-1b", layers=1)
-    tr = workload_trajectory(wl, 1, gen_device="cuda", check=[0, 4, 6])
-    assert [tr.f.diagnostics(i)["engine"] for i in range(7)] == [1, 1, 1, 1, 0, 0, 1]
+    tr = workload_trajectory(wl, 2, gen_device="cuda", check=[0, 4, 6])
+    assert [tr.f.diagnostics(i)["engine"] for i in range(7)] == [1] * 7
     tr.assert_ok()
+    for i in (0, 4, 6):
+        assert tr.f.diagnostics(i)["norm_prev"] == pytest.approx(tr.st[i].prev_norm, rel=2e-2)
