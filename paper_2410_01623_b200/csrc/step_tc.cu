@@ -96,7 +96,51 @@ __global__ void k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict
 
 // Copies between the caller's G and W and the copies with aligned rows, one block per row of a
 // staged matrix.  dir 0: G -> Gs, W -> Ws; dir 1: Ws -> W.  The caller's rows start on 2-byte
-// boundaries only, so elements move one at a time.
+// boundaries only; the copies' rows on 128-byte ones.  Both directions move 8-byte words on the
+// aligned side and assemble them from (or cut them into) two neighbouring aligned words of the other
+// side; a few elements at the ends of a row move one at a time.  No byte outside a row is written,
+// and none outside [first row, last row] of either buffer is read.
+
+// Row of n elements from `src` (any 2-byte alignment) to `dst` (8-byte aligned).
+__device__ __forceinline__ void copy_row_to_aligned(unsigned short* __restrict__ dst,
+                                                    const unsigned short* __restrict__ src, int n, bool first_row) {
+  const unsigned long long s = reinterpret_cast<unsigned long long>(src);
+  const int o = (int)(s & 7);                                   // bytes past an 8-byte boundary
+  const unsigned long long* sw = reinterpret_cast<const unsigned long long*>(s - o);
+  unsigned long long* dw = reinterpret_cast<unsigned long long*>(dst);
+  // words k < nw read sw[k], sw[k + 1]: bytes up to o + 2 n of the row; word 0 reaches o bytes back
+  int nw = (o + 2 * n) / 8 - 1;
+  if (nw < 0 || (o != 0 && first_row)) nw = 0;
+  if (o == 0) {
+    nw = n / 4;
+    for (int k = threadIdx.x; k < nw; k += blockDim.x) dw[k] = sw[k];
+  } else {
+    const int sh = 8 * o;
+    for (int k = threadIdx.x; k < nw; k += blockDim.x) dw[k] = (sw[k] >> sh) | (sw[k + 1] << (64 - sh));
+  }
+  for (int jj = 4 * nw + threadIdx.x; jj < n; jj += blockDim.x) dst[jj] = src[jj];
+}
+
+// Row of n elements from `src` (8-byte aligned, readable up to `pitch` elements) to `dst` (any alignment).
+__device__ __forceinline__ void copy_row_from_aligned(unsigned short* __restrict__ dst,
+                                                      const unsigned short* __restrict__ src, int n, int pitch) {
+  const unsigned long long d = reinterpret_cast<unsigned long long>(dst);
+  const int head = (int)(((8 - (d & 7)) & 7) / 2);              // elements before dst's first 8-byte boundary
+  if (head >= n) { for (int jj = threadIdx.x; jj < n; jj += blockDim.x) dst[jj] = src[jj]; return; }
+  unsigned long long* dw = reinterpret_cast<unsigned long long*>(dst + head);
+  const unsigned long long* sw = reinterpret_cast<const unsigned long long*>(src);
+  int nw = (n - head) / 4;                                      // whole aligned words of dst
+  if (head == 0) {
+    for (int k = threadIdx.x; k < nw; k += blockDim.x) dw[k] = sw[k];
+  } else {
+    nw = min(nw, pitch / 4 - 1);                                // word k reads sw[k] and sw[k + 1]
+    const int sh = 16 * head;
+    for (int k = threadIdx.x; k < nw; k += blockDim.x) dw[k] = (sw[k] >> sh) | (sw[k + 1] << (64 - sh));
+  }
+  for (int jj = threadIdx.x; jj < head; jj += blockDim.x) dst[jj] = src[jj];
+  for (int jj = head + 4 * nw + threadIdx.x; jj < n; jj += blockDim.x) dst[jj] = src[jj];
+}
+
 __global__ void __launch_bounds__(256)
 k_tc_stage(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
            const int* __restrict__ row_start, int dir) {
@@ -108,9 +152,10 @@ k_tc_stage(const MatDev* __restrict__ mats, const int* __restrict__ list, int nl
   unsigned short* gs = reinterpret_cast<unsigned short*>(mt.Gs) + i * mt.lds;
   unsigned short* ws = reinterpret_cast<unsigned short*>(mt.Ws) + i * mt.lds;
   if (dir == 0) {
-    for (int j = threadIdx.x; j < mt.n; j += 256) { gs[j] = g[j]; ws[j] = w[j]; }
+    copy_row_to_aligned(gs, g, mt.n, i == 0);
+    copy_row_to_aligned(ws, w, mt.n, i == 0);
   } else {
-    for (int j = threadIdx.x; j < mt.n; j += 256) w[j] = ws[j];
+    copy_row_from_aligned(w, ws, mt.n, (int)mt.lds);
   }
 }
 
