@@ -8,6 +8,7 @@
 #include <new>
 
 #include "context.cuh"
+#include "simt_gemm.cuh"
 #include "step_tc.cuh"
 
 namespace fira {
@@ -83,7 +84,7 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
     const size_t ll = std::max(d.m, d.n), r = d.r;
     L.offK[i] = w; w += align_up(ll * 4);
     if (L.engine[i] == 0) {
-      const size_t tiles = (size_t)((d.m + 63) / 64) * ((d.n + 63) / 64);
+      const size_t tiles = (size_t)simt_tiles(d.m) * simt_tiles(d.n);
       L.offRt[i] = w; w += align_up(ll * r * 4);
       L.offXt[i] = w; w += align_up(ll * r * 4);
       L.offPart[i] = w; w += align_up(tiles * 4);
@@ -226,9 +227,9 @@ fira_status fira_init(fira_ctx** out, const fira_hparams* hp, const fira_matrix_
     std::vector<int> pt{0}, rs{0}, wt{0}, np;
     for (int i : lst) {
       const MatDev& mt = c->mats[i];
-      pt.push_back(pt.back() + ((mt.l + 63) / 64) * ((mt.r + 63) / 64));
+      pt.push_back(pt.back() + simt_tiles(mt.l) * simt_tiles(mt.r));
       rs.push_back(rs.back() + mt.l);
-      const int tiles = ((mt.m + 63) / 64) * ((mt.n + 63) / 64);
+      const int tiles = simt_tiles(mt.m) * simt_tiles(mt.n);
       wt.push_back(wt.back() + tiles);
       np.push_back(tiles);
     }

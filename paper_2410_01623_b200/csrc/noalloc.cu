@@ -18,6 +18,7 @@
 #include <algorithm>
 
 #include "context.cuh"
+#include "simt_gemm.cuh"
 
 namespace fira {
 
@@ -38,7 +39,7 @@ struct Carve {
 
 Carve carve(int m, int n, int r) {
   const size_t l = std::max(m, n);
-  const size_t tiles = (size_t)((m + 63) / 64) * ((n + 63) / 64);
+  const size_t tiles = (size_t)simt_tiles(m) * simt_tiles(n);
   Carve c;
   size_t o = 0;
   c.off_mats = o; o += align_up(sizeof(MatDev));
@@ -126,8 +127,8 @@ extern "C" fira_status fira_step_single_noalloc(const fira_hparams* hp, const fi
   mt.l = std::max(desc->m, desc->n); mt.d = std::min(desc->m, desc->n);
   mt.engine = 0;
 
-  const int ptiles = ((mt.l + 63) / 64) * ((mt.r + 63) / 64);
-  const int wtiles = ((mt.m + 63) / 64) * ((mt.n + 63) / 64);
+  const int ptiles = simt_tiles(mt.l) * simt_tiles(mt.r);
+  const int wtiles = simt_tiles(mt.m) * simt_tiles(mt.n);
   // [list(1)] [proj_start(2)] [row_start(2)] [w_start(2)] [npart(1)]
   const int ints[8] = {0, 0, ptiles, 0, mt.l, 0, wtiles, wtiles};
   int* ints_dev = reinterpret_cast<int*>(base + cv.off_ints);

@@ -84,30 +84,30 @@ k_gauss(const RefreshMat* __restrict__ rm) {
 }
 
 // ------------------------------------------------------------------ grouped product
-__global__ void __launch_bounds__(GEMM_THREADS)
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
 k_rgemm(const GemmDesc* __restrict__ descs, int ndesc, const int* __restrict__ tile_start) {
-  __shared__ __align__(16) float As[TK][TM + 4];
-  __shared__ __align__(16) float Bs[TK][TN + 4];
+  __shared__ __align__(16) float As[TK][SIMT_TILE + 4];
+  __shared__ __align__(16) float Bs[TK][SIMT_TILE + 4];
   const int p = find_matrix(tile_start, ndesc, blockIdx.x);
   const GemmDesc g = descs[p];
   const int tile = blockIdx.x - tile_start[p];
-  const int jt = (g.J + TN - 1) / TN;
-  const int i0 = (tile / jt) * TM, j0 = (tile % jt) * TN;
-  float acc[4][4] = {};
+  const int jt = (g.J + SIMT_TILE - 1) / SIMT_TILE;
+  const int i0 = (tile / jt) * SIMT_TILE, j0 = (tile % jt) * SIMT_TILE;
+  float acc[4 * SIMT_Q][4 * SIMT_Q] = {};
   if (g.a_bf16)
-    gemm_tile<__nv_bfloat16, float>((const __nv_bfloat16*)g.A, g.sAi, g.sAk, g.B, g.sBk, g.sBj,
+    gemm_tile<SIMT_Q, __nv_bfloat16, float>((const __nv_bfloat16*)g.A, g.sAi, g.sAk, g.B, g.sBk, g.sBj,
                                     g.I, g.J, g.K, i0, j0, acc, As, Bs);
   else
-    gemm_tile<float, float>((const float*)g.A, g.sAi, g.sAk, g.B, g.sBk, g.sBj, g.I, g.J, g.K,
+    gemm_tile<SIMT_Q, float, float>((const float*)g.A, g.sAi, g.sAk, g.B, g.sBk, g.sBj, g.I, g.J, g.K,
                             i0, j0, acc, As, Bs);
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 #pragma unroll
-  for (int x = 0; x < 4; ++x) {
-    const int i = i0 + ty * 4 + x;
+  for (int x = 0; x < 4 * SIMT_Q; ++x) {
+    const int i = i0 + tile_coord(ty, x);
     if (i >= g.I) continue;
 #pragma unroll
-    for (int y = 0; y < 4; ++y) {
-      const int j = j0 + tx * 4 + y;
+    for (int y = 0; y < 4 * SIMT_Q; ++y) {
+      const int j = j0 + tile_coord(tx, y);
       if (j < g.J) g.C[(long long)i * g.sCi + j] = acc[x][y];
     }
   }
@@ -151,7 +151,7 @@ k_cholesky(const RefreshMat* __restrict__ rm, float shift_rel, unsigned* __restr
     // (a) C[I, J] -= L[I, :J0] L[J, :J0]^T for every row tile I >= J
     for (int I0 = J0; I0 < r; I0 += TM) {
       float acc[4][4] = {};
-      gemm_tile<float, float>(C, r, 1, C, 1, r, r, J0 + jb, J0, I0, J0, acc, As, Bs);
+      gemm_tile<1, float, float>(C, r, 1, C, 1, r, r, J0 + jb, J0, I0, J0, acc, As, Bs);
 #pragma unroll
       for (int x = 0; x < 4; ++x) {
         const int i = I0 + ty * 4 + x;
@@ -223,7 +223,7 @@ k_trsm_rows(const TrsmDesc* __restrict__ descs, int ndesc, const int* __restrict
   for (int J0 = 0; J0 < r; J0 += CB) {
     const int jb = min(CB, r - J0);
     float acc[4][4] = {};
-    gemm_tile<float, float>(t.X, r, 1, t.L, 1, r, t.rows, J0 + jb, J0, I0, J0, acc, As, Bs);
+    gemm_tile<1, float, float>(t.X, r, 1, t.L, 1, r, t.rows, J0 + jb, J0, I0, J0, acc, As, Bs);
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
       const int il = ty * 4 + x;
@@ -329,7 +329,7 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     std::vector<GemmDesc> gAZ, gAtY, gYY, gZZ;
     std::vector<TrsmDesc> tY, tZ;
     std::vector<int> sAZ{0}, sAtY{0}, sYY{0}, sTY{0}, sTZ{0};
-    auto tiles = [](int I, int J) { return ((I + TM - 1) / TM) * ((J + TN - 1) / TN); };
+    auto tiles = [](int I, int J) { return simt_tiles(I) * simt_tiles(J); };
     for (const RefreshMat& m : rms) {
       GemmDesc g;
       // Y[d][j] = sum_l A(d,l) Z[l][j]

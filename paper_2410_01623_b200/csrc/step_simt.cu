@@ -19,36 +19,38 @@ namespace fira {
 
 namespace {
 
+__device__ __forceinline__ int simt_tiles_dev(int extent) { return (extent + SIMT_TILE - 1) / SIMT_TILE; }
+
 // ---------------------------------------------------------------- phase 1
 template <typename T>
-__device__ __forceinline__ void project_tile(const MatDev& mt, int tile, float (*As)[TM + 4],
-                                             float (*Bs)[TN + 4]) {
-  const int rt = (mt.r + TN - 1) / TN;
-  const int i0 = (tile / rt) * TM, j0 = (tile % rt) * TN;
-  float acc[4][4] = {};
+__device__ __forceinline__ void project_tile(const MatDev& mt, int tile, float (*As)[SIMT_TILE + 4],
+                                             float (*Bs)[SIMT_TILE + 4]) {
+  const int rt = simt_tiles_dev(mt.r);
+  const int i0 = (tile / rt) * SIMT_TILE, j0 = (tile % rt) * SIMT_TILE;
+  float acc[4 * SIMT_Q][4 * SIMT_Q] = {};
   const T* G = static_cast<const T*>(mt.G);
   const T* P = static_cast<const T*>(mt.P);
   // A(i = l, k = d): G[d][l] when left, G[l][d] when right.
   const long long sAi = mt.left ? 1 : mt.ld, sAk = mt.left ? mt.ld : 1;
-  gemm_tile<T, T>(G, sAi, sAk, P, mt.r, 1, mt.l, mt.r, mt.d, i0, j0, acc, As, Bs);
+  gemm_tile<SIMT_Q, T, T>(G, sAi, sAk, P, mt.r, 1, mt.l, mt.r, mt.d, i0, j0, acc, As, Bs);
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
 #pragma unroll
-  for (int x = 0; x < 4; ++x) {
-    const int i = i0 + ty * 4 + x;
+  for (int x = 0; x < 4 * SIMT_Q; ++x) {
+    const int i = i0 + tile_coord(ty, x);
     if (i >= mt.l) continue;
 #pragma unroll
-    for (int y = 0; y < 4; ++y) {
-      const int j = j0 + tx * 4 + y;
+    for (int y = 0; y < 4 * SIMT_Q; ++y) {
+      const int j = j0 + tile_coord(tx, y);
       if (j < mt.r) mt.Rt[(long long)i * mt.r + j] = acc[x][y];
     }
   }
 }
 
-__global__ void __launch_bounds__(GEMM_THREADS)
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
 k_project(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
           const int* __restrict__ tile_start) {
-  __shared__ __align__(16) float As[TK][TM + 4];
-  __shared__ __align__(16) float Bs[TK][TN + 4];
+  __shared__ __align__(16) float As[TK][SIMT_TILE + 4];
+  __shared__ __align__(16) float Bs[TK][SIMT_TILE + 4];
   const int p = find_matrix(tile_start, nlist, blockIdx.x);
   const MatDev mt = mats[list[p]];
   const int tile = blockIdx.x - tile_start[p];
@@ -97,19 +99,19 @@ enum { MODE_NORM = 0, MODE_UPDATE = 1 };
 
 template <typename T, int MODE>
 __device__ __forceinline__ void back_tile(const MatDev& mt, int tile, float lr, float a_res,
-                                          float (*As)[TM + 4], float (*Bs)[TN + 4], float* red) {
-  const int ct = (mt.n + TN - 1) / TN;
-  const int i0 = (tile / ct) * TM, j0 = (tile % ct) * TN;
-  float acc[4][4] = {};
+                                          float (*As)[SIMT_TILE + 4], float (*Bs)[SIMT_TILE + 4], float* red) {
+  const int ct = simt_tiles_dev(mt.n);
+  const int i0 = (tile / ct) * SIMT_TILE, j0 = (tile % ct) * SIMT_TILE;
+  float acc[4 * SIMT_Q][4 * SIMT_Q] = {};
   const T* P = static_cast<const T*>(mt.P);
   const float* X = (MODE == MODE_NORM) ? mt.Rt : mt.Xt;
   const long long r = mt.r;
   if (mt.left) {
     // D[d][l] = sum_j Pi[d][j] X[l][j]
-    gemm_tile<T, float>(P, r, 1, X, 1, r, mt.m, mt.n, mt.r, i0, j0, acc, As, Bs);
+    gemm_tile<SIMT_Q, T, float>(P, r, 1, X, 1, r, mt.m, mt.n, mt.r, i0, j0, acc, As, Bs);
   } else {
     // D[l][d] = sum_j X[l][j] Pi[d][j]
-    gemm_tile<float, T>(X, r, 1, P, 1, r, mt.m, mt.n, mt.r, i0, j0, acc, As, Bs);
+    gemm_tile<SIMT_Q, float, T>(X, r, 1, P, 1, r, mt.m, mt.n, mt.r, i0, j0, acc, As, Bs);
   }
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const T* G = static_cast<const T*>(mt.G);
@@ -117,12 +119,12 @@ __device__ __forceinline__ void back_tile(const MatDev& mt, int tile, float lr, 
   const float lam = (MODE == MODE_UPDATE) ? mt.sc->lambda : 1.f;
   float ss = 0.f;
 #pragma unroll
-  for (int x = 0; x < 4; ++x) {
-    const int i = i0 + ty * 4 + x;
+  for (int x = 0; x < 4 * SIMT_Q; ++x) {
+    const int i = i0 + tile_coord(ty, x);
     if (i >= mt.m) continue;
 #pragma unroll
-    for (int y = 0; y < 4; ++y) {
-      const int j = j0 + tx * 4 + y;
+    for (int y = 0; y < 4 * SIMT_Q; ++y) {
+      const int j = j0 + tile_coord(tx, y);
       if (j >= mt.n) continue;
       const float kf = mt.kvec[mt.left ? j : i];
       const long long off = (long long)i * mt.ld + j;
@@ -150,11 +152,11 @@ __device__ __forceinline__ void back_tile(const MatDev& mt, int tile, float lr, 
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(GEMM_THREADS)
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
 k_back_project(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
                const int* __restrict__ tile_start, float lr, float a_res) {
-  __shared__ __align__(16) float As[TK][TM + 4];
-  __shared__ __align__(16) float Bs[TK][TN + 4];
+  __shared__ __align__(16) float As[TK][SIMT_TILE + 4];
+  __shared__ __align__(16) float Bs[TK][SIMT_TILE + 4];
   __shared__ float red[GEMM_THREADS / 32];
   const int p = find_matrix(tile_start, nlist, blockIdx.x);
   const MatDev mt = mats[list[p]];
