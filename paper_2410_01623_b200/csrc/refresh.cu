@@ -114,19 +114,30 @@ k_rgemm(const GemmDesc* __restrict__ descs, int ndesc, const int* __restrict__ t
 }
 
 // ------------------------------------------------------------------ Cholesky
-// One block per matrix: C (r x r, symmetric, row major) -> lower factor L in
-// place (the strict upper triangle is left as it was).  Left-looking over 64-wide
-// block columns.  shift_rel * trace(C)/r is added to the diagonal first.  A
-// non-positive or non-finite pivot is replaced and flagged.
+// One cluster of CHOL_CTAS blocks per matrix: C (r x r, symmetric, row major) -> lower factor L in
+// place (the strict upper triangle is left as it was).  Left-looking over 64-wide block columns:
+// the row tiles of the panel update and the rows of the solve below the diagonal block are dealt
+// out to the blocks of the cluster, which meet at a cluster barrier (release/acquire, so that what
+// one block wrote to C is what the others read) after each phase; every block factors the 64 x 64
+// diagonal block for itself in shared memory.  shift_rel * trace(C)/r is added to the diagonal
+// first.  A non-positive or non-finite pivot is replaced and flagged.
 constexpr int CB = 64;
+constexpr int CHOL_CTAS = 8;
 
-__global__ void __launch_bounds__(GEMM_THREADS)
+__device__ __forceinline__ void cluster_barrier() {
+  __threadfence();
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__global__ void __cluster_dims__(CHOL_CTAS, 1, 1) __launch_bounds__(GEMM_THREADS)
 k_cholesky(const RefreshMat* __restrict__ rm, float shift_rel, unsigned* __restrict__ status) {
   __shared__ __align__(16) float As[TK][TM + 4];
   __shared__ __align__(16) float Bs[TK][TN + 4];
   __shared__ float D[CB][CB + 1];
   __shared__ float red[GEMM_THREADS];
-  const RefreshMat m = rm[blockIdx.x];
+  const RefreshMat m = rm[blockIdx.x / CHOL_CTAS];
+  const int rank = blockIdx.x % CHOL_CTAS;
   const int r = m.r;
   float* C = m.C;
   const int tid = threadIdx.x;
@@ -141,15 +152,16 @@ k_cholesky(const RefreshMat* __restrict__ rm, float shift_rel, unsigned* __restr
   const float mean_diag = red[0] / (float)r;
   const float shift = shift_rel * mean_diag;
   const float floor_pivot = fmaxf(1e-30f, 1e-12f * mean_diag);
-  __syncthreads();
-  for (int i = tid; i < r; i += GEMM_THREADS) C[(long long)i * r + i] += shift;
-  __syncthreads();
+  cluster_barrier();                       // every block has read the unshifted diagonal
+  if (rank == 0)
+    for (int i = tid; i < r; i += GEMM_THREADS) C[(long long)i * r + i] += shift;
+  cluster_barrier();
 
   const int tx = tid & 15, ty = tid >> 4;
   for (int J0 = 0; J0 < r; J0 += CB) {
     const int jb = min(CB, r - J0);
-    // (a) C[I, J] -= L[I, :J0] L[J, :J0]^T for every row tile I >= J
-    for (int I0 = J0; I0 < r; I0 += TM) {
+    // (a) C[I, J] -= L[I, :J0] L[J, :J0]^T for the row tiles I >= J, dealt out to the blocks
+    for (int I0 = J0 + TM * rank; I0 < r; I0 += TM * CHOL_CTAS) {
       float acc[4][4] = {};
       gemm_tile<1, float, float>(C, r, 1, C, 1, r, r, J0 + jb, J0, I0, J0, acc, As, Bs);
 #pragma unroll
@@ -163,8 +175,8 @@ k_cholesky(const RefreshMat* __restrict__ rm, float shift_rel, unsigned* __restr
         }
       }
     }
-    __syncthreads();
-    // (b) factor the diagonal block in shared memory
+    cluster_barrier();
+    // (b) every block factors the diagonal block in its own shared memory
     for (int e = tid; e < CB * CB; e += GEMM_THREADS) {
       const int i = e / CB, j = e % CB;
       D[i][j] = (i < jb && j < jb) ? C[(long long)(J0 + i) * r + J0 + j] : (i == j ? 1.f : 0.f);
@@ -173,7 +185,7 @@ k_cholesky(const RefreshMat* __restrict__ rm, float shift_rel, unsigned* __restr
     for (int k = 0; k < jb; ++k) {
       if (tid == 0) {
         float pv = D[k][k];
-        if (!(pv > floor_pivot) || !isfinite(pv)) { pv = floor_pivot; atomicOr(status, DEV_STATUS_NONFINITE); }
+        if (!(pv > floor_pivot) || !isfinite(pv)) { pv = floor_pivot; if (rank == 0) atomicOr(status, DEV_STATUS_NONFINITE); }
         D[k][k] = sqrtf(pv);
       }
       __syncthreads();
@@ -187,12 +199,16 @@ k_cholesky(const RefreshMat* __restrict__ rm, float shift_rel, unsigned* __restr
       }
       __syncthreads();
     }
-    for (int e = tid; e < jb * jb; e += GEMM_THREADS) {
-      const int i = e / jb, j = e % jb;
-      if (j <= i) C[(long long)(J0 + i) * r + J0 + j] = D[i][j];
+    // all blocks have copied the unfactored block before block 0 overwrites it
+    cluster_barrier();
+    if (rank == 0) {
+      for (int e = tid; e < jb * jb; e += GEMM_THREADS) {
+        const int i = e / jb, j = e % jb;
+        if (j <= i) C[(long long)(J0 + i) * r + J0 + j] = D[i][j];
+      }
     }
-    // (c) rows below: L[i, J] = C[i, J] L_JJ^-T, one thread per row
-    for (int i = J0 + jb + tid; i < r; i += GEMM_THREADS) {
+    // (c) rows below: L[i, J] = C[i, J] L_JJ^-T, one thread per row, rows dealt out to the blocks
+    for (int i = J0 + jb + rank * GEMM_THREADS + tid; i < r; i += GEMM_THREADS * CHOL_CTAS) {
       float* row = C + (long long)i * r + J0;
       for (int c = 0; c < jb; ++c) {
         float v = row[c];
@@ -200,7 +216,7 @@ k_cholesky(const RefreshMat* __restrict__ rm, float shift_rel, unsigned* __restr
         row[c] = v / D[c][c];
       }
     }
-    __syncthreads();
+    cluster_barrier();
   }
 }
 
@@ -376,7 +392,7 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     auto orth = [&](const GemmDesc* gram, const TrsmDesc* tr, const int* tr_start, int tr_tiles) {
       for (int pass = 0; pass < 2; ++pass) {
         k_rgemm<<<sYY.back(), GEMM_THREADS, 0, st>>>(gram, nm, dsYY);
-        k_cholesky<<<nm, GEMM_THREADS, 0, st>>>(rm_dev, pass == 0 ? 1e-6f : 0.f, c->status_dev);
+        k_cholesky<<<nm * CHOL_CTAS, GEMM_THREADS, 0, st>>>(rm_dev, pass == 0 ? 1e-6f : 0.f, c->status_dev);
         k_trsm_rows<<<tr_tiles, GEMM_THREADS, 0, st>>>(tr, nm, tr_start);
       }
     };
