@@ -39,7 +39,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=None, help="override the layer count")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--refresh", default="layer", choices=["none", "layer", "full"],
+    ap.add_argument("--refresh", default="full", choices=["none", "layer", "full"],
                     help="time the projection refresh (separately from the step)")
     return ap.parse_args()
 

@@ -18,6 +18,7 @@
 
 #include "context.cuh"
 #include "simt_gemm.cuh"
+#include "step_tc.cuh"
 
 namespace fira {
 
@@ -29,6 +30,9 @@ struct RefreshMat {
   float* Y;   // d x r
   float* Z;   // l x r
   float* C;   // r x r
+  __nv_bfloat16* Yb;   // bf16 copies of Y and Z: operands of the tensor-core products (tc only)
+  __nv_bfloat16* Zb;
+  int tc;              // the products A Z and A^T Y of this matrix run on the tensor cores
   long long ld;
   int d, l, r;
   int left, bf16;
@@ -281,6 +285,24 @@ k_store_projection(const RefreshMat* __restrict__ rm) {
   }
 }
 
+// bf16 copy of the iterate that the next tensor-core product reads (which = 0: Y, 1: Z).
+__global__ void __launch_bounds__(256)
+k_iterate_to_bf16(const RefreshMat* __restrict__ rm, int which) {
+  const RefreshMat m = rm[blockIdx.y];
+  if (!m.tc) return;
+  const float* src = which ? m.Z : m.Y;
+  __nv_bfloat16* dst = which ? m.Zb : m.Yb;
+  const long long quads = (long long)(which ? m.l : m.d) * m.r / 4;      // r is a multiple of 128
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < quads;
+       q += (long long)gridDim.x * blockDim.x) {
+    const float4 v = reinterpret_cast<const float4*>(src)[q];
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    uint2 u;
+    u.x = *reinterpret_cast<unsigned*>(&a); u.y = *reinterpret_cast<unsigned*>(&b);
+    reinterpret_cast<uint2*>(dst)[q] = u;
+  }
+}
+
 // descriptor tables of a chunk: per-matrix entries plus alignment slack
 constexpr size_t TABLE_PER_MATRIX = 1024;
 constexpr size_t TABLE_SLACK = 16 * 1024;
@@ -288,9 +310,28 @@ static_assert(sizeof(RefreshMat) + 4 * sizeof(GemmDesc) + 2 * sizeof(TrsmDesc) +
 
 }  // namespace
 
+// bf16 matrices that TMA can read in place: their big products run on the tensor cores
+static bool refresh_on_tc(const fira_matrix_desc& d) {
+  return d.dtype == FIRA_BF16 && tc_supported(d) && tc_staging_pitch(d) == 0;
+}
+
+static TcGemmJob refresh_job(const fira_matrix_desc& d, bool az) {
+  TcGemmJob j;
+  memset(&j, 0, sizeof(j));
+  j.m = d.m; j.n = d.n; j.ld = d.ld ? d.ld : d.n; j.r = d.r;
+  const bool left = d.m <= d.n;
+  j.mn_major = az ? !left : left;      // A Z: rows d, k = l;  A^T Y: rows l, k = d
+  return j;
+}
+
 static size_t refresh_data_bytes(const fira_matrix_desc& d) {
   const size_t dd = std::min(d.m, d.n), ll = std::max(d.m, d.n), r = d.r;
-  return align_up(dd * r * 4) + align_up(ll * r * 4) + align_up(r * r * 4);
+  size_t b = align_up(dd * r * 4) + align_up(ll * r * 4) + align_up(r * r * 4);
+  if (refresh_on_tc(d)) {
+    const TcGemmJob a = refresh_job(d, true), t = refresh_job(d, false);
+    b += align_up(dd * r * 2) + align_up(ll * r * 2) + tc_gemm_table_bytes(&a, 1) + tc_gemm_table_bytes(&t, 1);
+  }
+  return b;
 }
 
 size_t refresh_bytes_per_matrix(const fira_matrix_desc& d) {
@@ -336,6 +377,12 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
       rm.Y = (float*)base; base += align_up((size_t)mt.d * mt.r * 4);
       rm.Z = (float*)base; base += align_up((size_t)mt.l * mt.r * 4);
       rm.C = (float*)base; base += align_up((size_t)mt.r * mt.r * 4);
+      rm.tc = refresh_on_tc(c->descs[idx]) ? 1 : 0;
+      rm.Yb = rm.Zb = nullptr;
+      if (rm.tc) {
+        rm.Yb = (__nv_bfloat16*)base; base += align_up((size_t)mt.d * mt.r * 2);
+        rm.Zb = (__nv_bfloat16*)base; base += align_up((size_t)mt.l * mt.r * 2);
+      }
       data_end = std::max(data_end, (size_t)(base - c->work_base));
       rm.ld = mt.ld; rm.d = mt.d; rm.l = mt.l; rm.r = mt.r; rm.left = mt.left; rm.bf16 = mt.bf16;
       rm.key = seed * 0x9E3779B97F4A7C15ull + (unsigned long long)idx * 0xD1B54A32D192ED03ull + 1ull;
@@ -346,17 +393,26 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     std::vector<TrsmDesc> tY, tZ;
     std::vector<int> sAZ{0}, sAtY{0}, sYY{0}, sTY{0}, sTZ{0};
     auto tiles = [](int I, int J) { return simt_tiles(I) * simt_tiles(J); };
-    for (const RefreshMat& m : rms) {
+    std::vector<TcGemmJob> jAZ, jAtY;
+    for (size_t a = 0; a < rms.size(); ++a) {
+      const RefreshMat& m = rms[a];
       GemmDesc g;
       // Y[d][j] = sum_l A(d,l) Z[l][j]
       g.A = m.G; g.a_bf16 = m.bf16;
       g.sAi = m.left ? m.ld : 1; g.sAk = m.left ? 1 : m.ld;
       g.B = m.Z; g.sBk = m.r; g.sBj = 1; g.C = m.Y; g.sCi = m.r; g.I = m.d; g.J = m.r; g.K = m.l;
-      gAZ.push_back(g); sAZ.push_back(sAZ.back() + tiles(g.I, g.J));
+      if (!m.tc) { gAZ.push_back(g); sAZ.push_back(sAZ.back() + tiles(g.I, g.J)); }
       // Z[l][j] = sum_d A(d,l) Y[d][j]
       g.sAi = m.left ? 1 : m.ld; g.sAk = m.left ? m.ld : 1;
       g.B = m.Y; g.C = m.Z; g.I = m.l; g.K = m.d;
-      gAtY.push_back(g); sAtY.push_back(sAtY.back() + tiles(g.I, g.J));
+      if (!m.tc) { gAtY.push_back(g); sAtY.push_back(sAtY.back() + tiles(g.I, g.J)); }
+      if (m.tc) {
+        const fira_matrix_desc& dd = c->descs[which[pos + a]];
+        TcGemmJob j = refresh_job(dd, true);
+        j.G = m.G; j.B = m.Zb; j.C = m.Y; jAZ.push_back(j);
+        j = refresh_job(dd, false);
+        j.G = m.G; j.B = m.Yb; j.C = m.Z; jAtY.push_back(j);
+      }
       // C = Y^T Y and C = Z^T Z
       g.a_bf16 = 0; g.sAi = 1; g.sAk = m.r; g.sBk = m.r; g.sBj = 1; g.C = m.C; g.sCi = m.r; g.I = m.r; g.J = m.r;
       g.A = m.Y; g.B = m.Y; g.K = m.d; gYY.push_back(g);
@@ -388,6 +444,33 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     const int* dsTY = (const int*)put(sTY.data(), sTY.size() * sizeof(int));
     const int* dsTZ = (const int*)put(sTZ.data(), sTZ.size() * sizeof(int));
     if (cerr != cudaSuccess) { set_error(std::string("refresh tables: ") + cudaGetErrorString(cerr)); return FIRA_ERR_CUDA; }
+    // tables of the tensor-core products (tensor maps and tile records), after the others
+    const int ntc = (int)jAZ.size(), nsimt = nm - ntc;
+    char* tabAZ = nullptr; char* tabAtY = nullptr;
+    int tilesAZ = 0, tilesAtY = 0;
+    if (ntc) {
+      const size_t bAZ = tc_gemm_table_bytes(jAZ.data(), ntc), bAtY = tc_gemm_table_bytes(jAtY.data(), ntc);
+      tabAZ = tp; tabAtY = tp + bAZ;
+      if ((size_t)(tabAtY + bAtY - c->work_base) > c->work_bytes) {
+        set_error("scratch buffer too small for the projection refresh"); return FIRA_ERR_WORKSPACE_TOO_SMALL;
+      }
+      fira_status ps = tc_gemm_prepare(c, jAZ.data(), ntc, tabAZ, bAZ, &tilesAZ);
+      if (ps == FIRA_OK) ps = tc_gemm_prepare(c, jAtY.data(), ntc, tabAtY, bAtY, &tilesAtY);
+      if (ps != FIRA_OK) return ps;
+    }
+    // A Z -> Y and A^T Y -> Z: CUDA-core products for some matrices, tensor-core products (bf16 copy
+    // of the iterate as the second operand, fp32 accumulation) for the others
+    auto product = [&](bool az) -> fira_status {
+      if (nsimt) {
+        if (az) k_rgemm<<<sAZ.back(), GEMM_THREADS, 0, st>>>(dAZ, nsimt, dsAZ);
+        else k_rgemm<<<sAtY.back(), GEMM_THREADS, 0, st>>>(dAtY, nsimt, dsAtY);
+      }
+      if (ntc) {
+        k_iterate_to_bf16<<<dim3(296, nm), 256, 0, st>>>(rm_dev, az ? 1 : 0);
+        return az ? tc_gemm_run(c, tabAZ, ntc, tilesAZ) : tc_gemm_run(c, tabAtY, ntc, tilesAtY);
+      }
+      return FIRA_OK;
+    };
 
     auto orth = [&](const GemmDesc* gram, const TrsmDesc* tr, const int* tr_start, int tr_tiles) {
       for (int pass = 0; pass < 2; ++pass) {
@@ -397,12 +480,13 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
       }
     };
     k_gauss<<<dim3(296, nm), 256, 0, st>>>(rm_dev);
-    k_rgemm<<<sAZ.back(), GEMM_THREADS, 0, st>>>(dAZ, nm, dsAZ);
+    fira_status prs = product(true);
+    if (prs != FIRA_OK) return prs;
     orth(dYY, dTY, dsTY, sTY.back());
     for (int it = 0; it < iters; ++it) {
-      k_rgemm<<<sAtY.back(), GEMM_THREADS, 0, st>>>(dAtY, nm, dsAtY);
+      if ((prs = product(false)) != FIRA_OK) return prs;
       orth(dZZ, dTZ, dsTZ, sTZ.back());
-      k_rgemm<<<sAZ.back(), GEMM_THREADS, 0, st>>>(dAZ, nm, dsAZ);
+      if ((prs = product(true)) != FIRA_OK) return prs;
       orth(dYY, dTY, dsTY, sTY.back());
     }
     k_store_projection<<<dim3(296, nm), 256, 0, st>>>(rm_dev);

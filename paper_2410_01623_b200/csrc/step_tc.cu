@@ -462,6 +462,71 @@ fira_status tc_update_pointers(fira_ctx* c) {
   return FIRA_OK;
 }
 
+// ---------------------------------------------------------------- refresh products
+static size_t gemm_job_tiles(const TcGemmJob& j) {
+  const int L = j.mn_major ? j.n : j.m;
+  return (size_t)((L + 2 * BM - 1) / (2 * BM)) * (j.r / host_tile_bn(j.r));
+}
+
+size_t tc_gemm_table_bytes(const TcGemmJob* jobs, int njobs) {
+  size_t tiles = 0;
+  for (int i = 0; i < njobs; ++i) tiles += gemm_job_tiles(jobs[i]);
+  return align_up(sizeof(TcMaps) * (size_t)njobs) + align_up(sizeof(ProjTileDesc) * tiles);
+}
+
+fira_status tc_gemm_prepare(fira_ctx* c, const TcGemmJob* jobs, int njobs, char* table_dev, size_t table_bytes,
+                            int* ntiles_out) {
+  if (tc_gemm_table_bytes(jobs, njobs) > table_bytes) { set_error("refresh: table area too small"); return FIRA_ERR_WORKSPACE_TOO_SMALL; }
+  std::vector<TcMaps> maps((size_t)njobs);
+  std::vector<ProjTileDesc> tiles;
+  for (int q = 0; q < njobs; ++q) {
+    const TcGemmJob& j = jobs[q];
+    const int L = j.mn_major ? j.n : j.m, D = j.mn_major ? j.m : j.n;
+    const int bn = host_tile_bn(j.r);
+    const bool chunked = j.mn_major && j.n % 64 == 0;
+    TcMaps& mp = maps[q];
+    memset(&mp, 0, sizeof(mp));
+    if (chunked) {
+      if (!encode_map_chunked(&mp.g1a, j.G, j.m, j.n, j.ld, 64, 2)) return FIRA_ERR_CUDA;
+    } else if (!encode_map(&mp.g1a, j.G, j.m, j.n, j.ld, 64, j.mn_major ? 64 : 128)) return FIRA_ERR_CUDA;
+    if (!encode_map_chunked(&mp.g1b, j.B, D, j.r, j.r, 64, bn / 128)) return FIRA_ERR_CUDA;
+    if (!encode_map(&mp.em, j.C, L, j.r, j.r, K1_ECOLS, K1_EROWS, 1)) return FIRA_ERR_CUDA;
+    for (int l0 = 0; l0 < L; l0 += 2 * BM)
+      for (int r0 = 0; r0 < j.r; r0 += bn) {
+        ProjTileDesc d;
+        d.colpart = nullptr; d.slot = q; d.l0 = l0; d.r0 = r0;
+        d.nkb = (D + BK - 1) / BK; d.L = L;
+        d.bn_left = bn | ((j.r / bn) << 16) | (j.mn_major ? (int)0x80000000 : 0) | (chunked ? PROJ_A_CHUNKED : 0);
+        tiles.push_back(d);
+      }
+  }
+  char* tiles_dev = table_dev + align_up(sizeof(TcMaps) * (size_t)njobs);
+  cudaError_t e = cudaMemcpyAsync(table_dev, maps.data(), sizeof(TcMaps) * maps.size(), cudaMemcpyHostToDevice, c->stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(tiles_dev, tiles.data(), sizeof(ProjTileDesc) * tiles.size(), cudaMemcpyHostToDevice, c->stream);
+  if (e != cudaSuccess) { set_error(std::string("refresh tables: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
+  *ntiles_out = (int)tiles.size();
+  return FIRA_OK;
+}
+
+fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntiles) {
+  static bool attr_set = false;
+  static int num_sms = 0;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_tc_project<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, c->device);
+    if (e != cudaSuccess) { set_error(std::string("refresh product set-up: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
+    attr_set = true;
+  }
+  if (ntiles == 0) return FIRA_OK;
+  const TcMaps* maps = reinterpret_cast<const TcMaps*>(table_dev);
+  const ProjTileDesc* tiles = reinterpret_cast<const ProjTileDesc*>(table_dev + align_up(sizeof(TcMaps) * (size_t)njobs));
+  Hyper hp{};
+  k_tc_project<EPI_PLAIN><<<2 * std::min(ntiles, num_sms / 2), K1_THREADS, K1_SMEM_BYTES, c->stream>>>(
+      maps, tiles, ntiles, nullptr, hp, c->status_dev);
+  return FIRA_OK;
+}
+
 int tc_phase_names(const char** out) {
   static const char* names[8] = {"k_tc_stage(in)", "k_tc_prep", "k_tc_project", "k_tc_colfactors",
                                  "k_finalize(tc)", "k_tc_form_x", "k_tc_back_project", "k_tc_stage(out)"};
@@ -474,7 +539,7 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   if (!pl || pl->nlist == 0) return 0;
   cudaStream_t st = c->stream;
   if (!pl->attrs_set) {
-    cudaError_t e1 = cudaFuncSetAttribute(k_tc_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
+    cudaError_t e1 = cudaFuncSetAttribute(k_tc_project<EPI_ADAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
     cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES);
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
       set_error(std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
@@ -489,7 +554,7 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   k_tc_prep<<<(pl->nlist + 127) / 128, 128, 0, st>>>(mats, pl->list, pl->nlist, hp, pl->fast_dev);
   tm->mark(st);
   // both tensor kernels: clusters of two CTAs, at most one CTA per SM
-  k_tc_project<<<2 * std::min(pl->k1_tiles, pl->num_sms / 2), K1_THREADS, K1_SMEM_BYTES, st>>>(
+  k_tc_project<EPI_ADAM><<<2 * std::min(pl->k1_tiles, pl->num_sms / 2), K1_THREADS, K1_SMEM_BYTES, st>>>(
       pl->maps_dev, pl->td1_dev, pl->k1_tiles, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);
   k_tc_colfactors<<<pl->col_blocks, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->col_start, hp);

@@ -32,4 +32,21 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp);
 // Names of this engine's phases in launch order (8).
 int tc_phase_names(const char** out);
 
+// ---- products of the projection refresh on the tensor cores
+// C[l][j] (fp32, L x r) = sum over k < D of A(k, l) B[k][j], with A taken in place from the bf16
+// matrix G (m x n, pitch ld, rows 16-byte aligned): mn_major = 1: G is [k][l] (D = m, L = n);
+// mn_major = 0: G is [l][k] (L = m, D = n).  B is bf16 [D][r].  r % 128 == 0.
+struct TcGemmJob {
+  const void* G; long long ld; int m, n; int mn_major;
+  const void* B; float* C; int r;
+};
+// Device bytes of the tables (tensor maps, tile records) of a job list.
+size_t tc_gemm_table_bytes(const TcGemmJob* jobs, int njobs);
+// Builds the tables on the host and uploads them to table_dev (256-byte aligned) on the context's
+// stream; *ntiles_out is what tc_gemm_run needs.
+fira_status tc_gemm_prepare(fira_ctx* c, const TcGemmJob* jobs, int njobs, char* table_dev, size_t table_bytes,
+                            int* ntiles_out);
+// One grouped launch over the prepared jobs.
+fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntiles);
+
 }  // namespace fira

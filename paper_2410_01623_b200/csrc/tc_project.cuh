@@ -99,6 +99,13 @@ __device__ __forceinline__ ProjTileDesc load_desc(const ProjTileDesc* __restrict
   return d;
 }
 
+// EPI_ADAM: the step's kernel as described above.  EPI_PLAIN: the same product with the accumulator
+// written out as it is, C[l][j] (fp32, through the `em` map): the products A^T Y and A Z of the
+// projection refresh.  Then no M/V boxes are loaded, the output box of a row half is built in that
+// half's N/R buffer, and the loader and the G^2 warps have nothing to do.
+enum { EPI_ADAM = 0, EPI_PLAIN = 1 };
+
+template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(K1_THREADS, 1)
 k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ tdesc, int total_tiles,
              const float* __restrict__ fast, Hyper hp, unsigned* __restrict__ status) {
@@ -161,7 +168,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         const int l0 = d.l0 + BM * (int)rank;             // this CTA's unprojected indices
         const int rb0 = d.r0 + (bn / 2) * (int)rank;      // this CTA's half of the rank range
         const int nparts = (d.bn_left >> 16) & 0xff;
-        int gturn = d.r0 / bn;                            // next k-block that the G^2 warps read
+        int gturn = EPI == EPI_ADAM ? d.r0 / bn : -1;     // next k-block that the G^2 warps read
         const uint32_t bytes = 2 * (A_STAGE_BYTES + (bn / 2) * BK * 2);   // both CTAs together
         for (int kb = 0; kb < d.nkb; ++kb) {
           if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -206,7 +213,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         const int bn = d.bn_left & 0xffff;
         const uint32_t idesc = ptx::make_idesc_bf16(2 * BM, bn, left, 1);
         const int nparts = (d.bn_left >> 16) & 0xff;
-        int gturn = d.r0 / bn;                            // next k-block that the G^2 warps read
+        int gturn = EPI == EPI_ADAM ? d.r0 / bn : -1;     // next k-block that the G^2 warps read
         if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->tmem_empty[buf]), bphase ^ 1u, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t dcol = tmem + buf * BN_MAX;
@@ -236,7 +243,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------ epilogue loader: M and V boxes
-    if (lane == 0 && smem_ok) {
+    if (EPI == EPI_ADAM && lane == 0 && smem_ok) {
       int mv = 0; uint32_t mvphase = 0; bool ok = true;
       ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
       for (int t = pair; t < total_tiles && ok; t += npairs) {
@@ -259,7 +266,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     }
   } else if (warp >= 8) {
     // ------------------------------------------------------------ sums of G^2 over the A stages
-    if (smem_ok) {
+    if (EPI == EPI_ADAM && smem_ok) {
       const int w = warp - 8;
       const int khalf = w >> 1;                          // left: d rows 32 khalf .. + 31 of a stage
       int base = 0; uint32_t aphase = 0; bool ok = true;  // stage of the tile's first k-block; parities of afull
@@ -357,10 +364,14 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           const int j = d.r0 + K1_ECOLS * (b >> 1), row = l0 + K1_EROWS * nr;
           if (row < d.L) {
             const uint32_t src = mvbuf_u32 + mv * K1_MVBUF_BYTES, srn = nrbuf_u32 + nr * K1_NRBUF_BYTES;
-            ptx::tma_store_2d(&mp->em, src, j, row);
-            ptx::tma_store_2d(&mp->ev, src + K1_FBOX_BYTES, j, row);
-            ptx::tma_store_2d(&mp->en, srn, j, row);
-            ptx::tma_store_2d(&mp->er, srn + K1_HBOX_BYTES, j, row);
+            if (EPI == EPI_ADAM) {
+              ptx::tma_store_2d(&mp->em, src, j, row);
+              ptx::tma_store_2d(&mp->ev, src + K1_FBOX_BYTES, j, row);
+              ptx::tma_store_2d(&mp->en, srn, j, row);
+              ptx::tma_store_2d(&mp->er, srn + K1_HBOX_BYTES, j, row);
+            } else {
+              ptx::tma_store_2d(&mp->em, srn, j, row);      // the fp32 output box sits in the N/R buffer
+            }
             ptx::bulk_commit_group();
             ptx::bulk_wait_group_read<0>();              // the boxes have been read: the buffers are free
           }
@@ -399,7 +410,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
       if (t + npairs < total_tiles) nd = load_desc(tdesc, t + npairs);
       const int bn = d.bn_left & 0xffff;
       const int l = d.l0 + BM * (int)rank + row;
-      const float bias = fast[2 * d.slot];
+      const float bias = EPI == EPI_ADAM ? fast[2 * d.slot] : 0.f;
       if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->tmem_full[buf]), bphase, abort_flag)) break;
       ptx::tc_fence_after();
       const uint32_t tcol = tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX;
@@ -416,10 +427,17 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive_cluster(te);
         }
-        if (!ptx::mbar_wait(ptx::smem_u32(&ctl->efull[mv][half]), mvphase, abort_flag)) { ok = false; break; }
+        if (EPI == EPI_ADAM && !ptx::mbar_wait(ptx::smem_u32(&ctl->efull[mv][half]), mvphase, abort_flag)) { ok = false; break; }
         if (!ptx::mbar_wait(nrempty, nrphase ^ 1u, abort_flag)) { ok = false; break; }
         unsigned char* mb = mvbuf + (size_t)mv * K1_MVBUF_BYTES;
         unsigned char* vb = mb + K1_FBOX_BYTES;
+        if (EPI == EPI_PLAIN) {
+          // 32 fp32 values of this row: eight 16-byte slots of a 128-byte row, slot ^= row % 8
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            *reinterpret_cast<uint4*>(nb + frow + (((uint32_t)q ^ fsw) << 4)) =
+                make_uint4(rr[4 * q], rr[4 * q + 1], rr[4 * q + 2], rr[4 * q + 3]);
+        } else {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {                    // 8 columns at a time
           const uint32_t f0 = frow + (((uint32_t)(2 * q) ^ fsw) << 4);
@@ -448,6 +466,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           *reinterpret_cast<uint4*>(nb + h) = pack8_bf16(nv);
           *reinterpret_cast<uint4*>(rb + h) = pack8_bf16(rv);
         }
+        }
         // hand the finished boxes to the storer: this thread's writes are visible to
         // the async proxy (TMA) before it arrives
         ptx::fence_proxy_async_smem();
@@ -457,7 +476,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         if (mv >= K1_MVBUFS) mv -= K1_MVBUFS;
         if (++mvuse == K1_MVBUFS) { mvuse = 0; mvphase ^= 1u; }
       }
-      if (ok && l < d.L) {
+      if (EPI == EPI_ADAM && ok && l < d.L) {
         // colpart[2 part][l] = partial ||N_l||^2, colpart[2 part + 1][l] = partial ||R_l||^2
         const int part = d.r0 / bn;
         d.colpart[(long long)(2 * part) * d.L + l] = nn;

@@ -39,6 +39,25 @@ def test_bf16_projection_is_orthonormal_to_storage_precision():
     assert fo.principal_angles(P, Po).max() <= 8e-3            # one bf16 rounding of the basis
 
 
+@pytest.mark.parametrize("shape,r", [((512, 1024), 128), ((1024, 512), 128), ((640, 1000), 256),
+                                     ((1000, 640), 256), ((512, 1365), 128)])
+def test_bf16_refresh_with_tensor_core_products(shape, r):
+    """bf16 matrices of tensor-core size: the products A Z and A^T Y of the iteration run on the
+    tensor cores with a bf16 copy of the iterate (ragged tiles, both orientations; the odd-width
+    case stays on the CUDA cores).  The subspace must still be the SVD's to the precision of a
+    bf16 basis, and the stored basis orthonormal to storage precision."""
+    m, n = shape
+    G = wk.planted_gradient(m, n, r, seed=m + 3 * n, gap=4.0).cuda().to(torch.bfloat16)
+    f = fb.Fira([shape], r, torch.bfloat16, fb.make_hparams())
+    f.refresh_projection([G], seed=11, iters=6)
+    assert f.poll() == 0
+    P = to_np64(f.get_projection(0))
+    assert np.abs(P.T @ P - np.eye(r)).max() < 1e-2
+    Po = fo.refresh_projection(to_np64(G), r)
+    assert fo.principal_angles(P, Po).max() <= 8e-3
+    assert fo.captured_energy(to_np64(G), P) >= 0.999 * fo.captured_energy(to_np64(G), Po)
+
+
 def test_gapless_gradient_captures_the_energy():
     """Gaussian gradients have no gap at r, so the subspace itself is ill-defined;
     what is fixed is the energy inside it, compared with the optimum sum of sigma_i^2."""
