@@ -5,11 +5,18 @@
 //   Z <- Gaussian (l x r);  Y <- orth(A Z)
 //   repeat `iters` times:   Z <- orth(A^T Y);  Y <- orth(A Z)
 //   projection <- Y  (d x r)
-// orth() is CholeskyQR applied twice: C = Y^T Y, C = L L^T, Y <- Y L^-T.  It
-// changes the basis, never the spanned subspace, so a small diagonal shift in the
-// first pass (which keeps the factorisation defined for ill-conditioned Y) costs
-// no accuracy of the subspace.  The paper calls a library SVD here; the iteration
-// converges to the same subspace at the rate (sigma_{r+1}/sigma_r)^2 per round.
+// orth() is CholeskyQR: C = Y^T Y, C = L L^T, Y <- Y L^-T, once for the intermediate
+// iterates and twice for the basis that is kept.  It changes the basis, never the
+// spanned subspace, so a small diagonal shift in the first pass (which keeps the
+// factorisation defined for ill-conditioned Y) costs no accuracy of the subspace.
+// The paper calls a library SVD here; the iteration converges to the same subspace
+// at the rate (sigma_{r+1}/sigma_r)^2 per round.
+//
+// The two big products run on the CUDA cores in fp32, except for bf16 matrices of
+// tensor-core size with TMA-readable rows: there G is exact in bf16 already, the
+// iterate is rounded to bf16 and the products run on the projection kernel of the
+// step (fp32 accumulation); the basis is stored in bf16 anyway.  Gram products,
+// Cholesky and the triangular solves stay in fp32.
 //
 // Random numbers: Philox4x32-10 (Salmon et al., "Parallel random numbers: as easy
 // as 1, 2, 3", SC'11), keyed by the caller's seed, turned into normals by the
@@ -472,8 +479,11 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
       return FIRA_OK;
     };
 
-    auto orth = [&](const GemmDesc* gram, const TrsmDesc* tr, const int* tr_start, int tr_tiles) {
-      for (int pass = 0; pass < 2; ++pass) {
+    // CholeskyQR; the second pass brings the basis to fp32 orthonormality and is needed only for the
+    // basis that is kept: one pass (deviation about cond^2 * 2^-24) keeps an intermediate iterate
+    // well conditioned, which is all the next product asks of it.
+    auto orth = [&](const GemmDesc* gram, const TrsmDesc* tr, const int* tr_start, int tr_tiles, int passes) {
+      for (int pass = 0; pass < passes; ++pass) {
         k_rgemm<<<sYY.back(), GEMM_THREADS, 0, st>>>(gram, nm, dsYY);
         k_cholesky<<<nm * CHOL_CTAS, GEMM_THREADS, 0, st>>>(rm_dev, pass == 0 ? 1e-6f : 0.f, c->status_dev);
         k_trsm_rows<<<tr_tiles, GEMM_THREADS, 0, st>>>(tr, nm, tr_start);
@@ -482,12 +492,12 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     k_gauss<<<dim3(296, nm), 256, 0, st>>>(rm_dev);
     fira_status prs = product(true);
     if (prs != FIRA_OK) return prs;
-    orth(dYY, dTY, dsTY, sTY.back());
+    orth(dYY, dTY, dsTY, sTY.back(), iters == 0 ? 2 : 1);
     for (int it = 0; it < iters; ++it) {
       if ((prs = product(false)) != FIRA_OK) return prs;
-      orth(dZZ, dTZ, dsTZ, sTZ.back());
+      orth(dZZ, dTZ, dsTZ, sTZ.back(), 1);
       if ((prs = product(true)) != FIRA_OK) return prs;
-      orth(dYY, dTY, dsTY, sTY.back());
+      orth(dYY, dTY, dsTY, sTY.back(), it + 1 == iters ? 2 : 1);
     }
     k_store_projection<<<dim3(296, nm), 256, 0, st>>>(rm_dev);
     RF_CUDA(cudaGetLastError());
