@@ -72,6 +72,10 @@ ALU_FP32_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
 # kernel name -> (bound, algorithmic share): flops as a fraction of the step's 4mnr, or
 # "bytes" for the streaming kernels
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch on 2 layers of the llama-7b list
+# (profiles/k_tc_kernels_2layers_ncu_full.md)
+NCU_DRAM_BYTES_2_LAYERS = {"k_tc_project": 1.912e9 + 1.169e9, "k_tc_back_project": 2.004e9 + 0.779e9}
+
 KERNEL_MODEL = {
     "k_project": ("alu", 0.5), "k_back_project<norm>": ("alu", 0.5), "k_back_project<update>": ("alu", 0.5),
     "k_tc_project": ("tensor", 0.5), "k_tc_back_project": ("tensor", 0.5),
@@ -334,8 +338,13 @@ def main():
     else:
         peak, unit, ach = peaks["hbm_gbs"], "GB/s", None
         peak_kind = f"copy bandwidth, {peaks['source']}"
+    # DRAM bytes per launch from the ncu capture summarised under profiles/ (2 of the 32 layers,
+    # scaled by the layer count: every layer has the same shapes, so traffic grows in proportion)
+    traffic = None
+    if wl.name == "llama-7b" and top[0] in NCU_DRAM_BYTES_2_LAYERS:
+        traffic = NCU_DRAM_BYTES_2_LAYERS[top[0]] * (nmat / 14.0)
     roofline = {"kernel": top[0], "bound": bound, "achieved": ach, "peak": peak, "unit": unit,
-                "frac": (ach / peak) if ach else None, "traffic": None, "peak_kind": peak_kind,
+                "frac": (ach / peak) if ach else None, "traffic": traffic, "peak_kind": peak_kind,
                 "kernel_ms": top[1], "kernel_share": top[1] / max(sum(p[1] for p in phases), 1e-9),
                 "step_roofline_ms": roof_ms, "step_frac_of_roofline": roof_ms / ms_step,
                 "phases_ms": {k: round(v, 4) for k, v in phases}, "phase_steps": nrec}
