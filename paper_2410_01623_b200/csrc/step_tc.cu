@@ -176,7 +176,7 @@ k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, i
       nn += mt.colpart[(long long)(2 * q) * mt.l + l];
       rn += mt.colpart[(long long)(2 * q + 1) * mt.l + l];
     }
-    for (int q = 2 * nparts; q < 4 * nparts; ++q) gs += mt.colpart[(long long)q * mt.l + l];   // ||G_l||^2 in parts
+    for (int q = 2 * nparts; q < (2 + K1_GSQ_SPLIT) * nparts; ++q) gs += mt.colpart[(long long)q * mt.l + l];   // ||G_l||^2 in parts
     const float k = sqrtf(nn) / (sqrtf(rn) + hp.eps);
     mt.kvec[l] = k;
     contrib = k * k * fmaxf(gs - rn, 0.f);
@@ -308,7 +308,7 @@ long long tc_staging_pitch(const fira_matrix_desc& d) {
 
 size_t tc_colpart_floats(const fira_matrix_desc& d) {
   const size_t l = std::max(d.m, d.n);
-  return 4 * (size_t)(d.r / host_tile_bn(d.r)) * l;   // N^2 and R^2 per r-tile, then two partial G^2 per r-tile
+  return (2 + K1_GSQ_SPLIT) * (size_t)(d.r / host_tile_bn(d.r)) * l;   // N^2 and R^2 per r-tile, then the partial G^2
 }
 
 size_t tc_part_floats(const fira_matrix_desc& d) { return ((size_t)std::max(d.m, d.n) + 255) / 256; }

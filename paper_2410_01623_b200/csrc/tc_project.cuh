@@ -29,13 +29,13 @@
 //
 // ||G_l||^2: G passes through shared memory as the A operand anyway.  The r / BN tiles that share a
 // panel of G split its k-blocks between them (tile `part` takes k-blocks part, part + r / BN, ...):
-// four more warps square and sum such an A stage while its MMAs run (the MMA issuer tells both CTAs
+// eight more warps square and sum such an A stage while its MMAs run (the MMA issuer tells both CTAs
 // when the stage has landed; the producer waits for the warps before it overwrites the stage, on
 // those k-blocks only).  This replaces a separate pass over G in HBM.
 //
 // Warp roles: 0 operand producer (TMA); 1 MMA issuer (even CTA only) and TMEM owner;
 // 2 epilogue loader (TMA); 3-6 epilogue; 7 one thread that stores the finished boxes;
-// 8-11 sums of G^2.
+// 8-15 sums of G^2.
 constexpr int K1_STAGES = 5;
 constexpr int K1_STAGE_BYTES = 2 * A_STAGE_BYTES;       // A: 128 l x 64 d, B half: 128 r x 64 d
 constexpr int K1_ECOLS = 32;                            // columns per epilogue box
@@ -47,7 +47,8 @@ constexpr int K1_NRBUFS = 2;                            // {N box, R box}, one p
 constexpr int K1_MVBUF_BYTES = 2 * K1_FBOX_BYTES;
 constexpr int K1_NRBUF_BYTES = 2 * K1_HBOX_BYTES;
 constexpr int K1_BOX_THREADS = 64;                      // two warps work on a box
-constexpr int K1_GSQ_WARPS = 4;
+constexpr int K1_GSQ_WARPS = 8;
+constexpr int K1_GSQ_SPLIT = K1_GSQ_WARPS / 2;          // partial sums of G^2 per tile and l
 constexpr int K1_THREADS = 32 * (8 + K1_GSQ_WARPS);
 constexpr size_t K1_SMEM_BYTES = (size_t)K1_STAGES * K1_STAGE_BYTES + (size_t)K1_MVBUFS * K1_MVBUF_BYTES +
                                  (size_t)K1_NRBUFS * K1_NRBUF_BYTES + 512;
@@ -268,7 +269,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     // ------------------------------------------------------------ sums of G^2 over the A stages
     if (EPI == EPI_ADAM && smem_ok) {
       const int w = warp - 8;
-      const int khalf = w >> 1;                          // left: d rows 32 khalf .. + 31 of a stage
+      const int kq = w >> 1;                             // left: d rows 16 kq .. + 15 of a stage
       int base = 0; uint32_t aphase = 0; bool ok = true;  // stage of the tile's first k-block; parities of afull
       ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
       for (int t = pair; t < total_tiles && ok; t += npairs) {
@@ -289,12 +290,12 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
             const unsigned char* sa = tiles + (size_t)stage * K1_STAGE_BYTES;
             if (left) {
               // chunk w % 2: [64 d rows][64 l], 128-byte rows, 16-byte slot ^= row % 8.
-              // lane: slot lane % 8 (8 values of l), rows 32 khalf + lane / 8, + 4, ...
+              // lane: slot lane % 8 (8 values of l), rows 16 kq + lane / 8, + 4, ...
               const unsigned char* ch = sa + (w & 1) * CHUNK_BYTES;
               const int slot = lane & 7;
 #pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const int k = 32 * khalf + (lane >> 3) + 4 * i;
+              for (int i = 0; i < 4; ++i) {
+                const int k = 16 * kq + (lane >> 3) + 4 * i;
                 const uint4 u = *reinterpret_cast<const uint4*>(ch + k * 128 + ((slot ^ (k & 7)) << 4));
                 float g[8];
                 unpack8_bf16(u, g);
@@ -302,11 +303,11 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
                 for (int e = 0; e < 8; ++e) acc[e] = fmaf(g[e], g[e], acc[e]);
               }
             } else {
-              // [128 l rows][64 d], 128-byte rows, slot ^= row % 8: one row per thread
-              const int row = 32 * w + lane;
+              // [128 l rows][64 d], 128-byte rows, slot ^= row % 8: half a row per thread
+              const int row = 32 * (w & 3) + lane;
               const unsigned char* rp = sa + row * 128;
 #pragma unroll
-              for (int q = 0; q < 8; ++q) {
+              for (int q = 4 * (w >> 2); q < 4 * (w >> 2) + 4; ++q) {
                 const uint4 u = *reinterpret_cast<const uint4*>(rp + ((q ^ (row & 7)) << 4));
                 float g[8];
                 unpack8_bf16(u, g);
@@ -320,8 +321,8 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         }
         base = (base + d.nkb) % K1_STAGES;
         if (ok) {
-          // slots after the 2 nparts partial sums of N^2 and R^2: [2 part + khalf][l]
-          float* gs = d.colpart + (long long)(2 * nparts + 2 * part) * d.L;
+          // slots after the 2 nparts partial sums of N^2 and R^2: [K1_GSQ_SPLIT part + quarter][l]
+          float* gs = d.colpart + (long long)(2 * nparts + K1_GSQ_SPLIT * part) * d.L;
           const int lbase = d.l0 + BM * (int)rank;
           if (left) {
 #pragma unroll
@@ -331,7 +332,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
             }
             const int l = lbase + 64 * (w & 1) + 8 * lane;
             if (lane < 8 && l < d.L) {
-              float* o = gs + (long long)khalf * d.L + l;
+              float* o = gs + (long long)kq * d.L + l;
               if ((d.L & 3) == 0 && l + 8 <= d.L) {      // rows of the table stay 16-byte aligned
                 *reinterpret_cast<float4*>(o) = make_float4(acc[0], acc[1], acc[2], acc[3]);
                 *reinterpret_cast<float4*>(o + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
@@ -341,8 +342,8 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
               }
             }
           } else {
-            const int l = lbase + 32 * w + lane;
-            if (l < d.L) { gs[l] = acc[0]; gs[d.L + l] = 0.f; }
+            const int l = lbase + 32 * (w & 3) + lane;   // slots 0 and 1: the two halves of the row; 2, 3: unused
+            if (l < d.L) { gs[(long long)(w >> 2) * d.L + l] = acc[0]; gs[(long long)(2 + (w >> 2)) * d.L + l] = 0.f; }
           }
         }
       }
