@@ -36,6 +36,12 @@ design notes of the repository as well):
   * Norms: Frobenius for matrices, l2 for columns.
   * A projection switch keeps M, V, the remembered norm and t (Section 4.2,
     "Loss spike analysis").
+  * Ablation variants (Section 5.4 "Ablation Study", Eq. 6, 8, 9-10): `scaling`
+    = "column" (Fira, Eq. 11), "matrix" (Fira-matrix: one factor
+    ||N||_F / (||R||_F + eps) for the whole matrix, Eq. 9 with the same + eps),
+    "none" (Fira-w.o.-scaling: the factor is 1; without the limiter this is
+    GaLore-add, Eq. 8); `residual=False` drops S altogether (GaLore, Eq. 6): then
+    there is no norm to limit or to remember.
   * bf16 storage: when `store="bf16"` the new W is rounded to bfloat16
     (round to nearest, ties to even) after the update, because on that path W
     IS a bf16 tensor.  Nothing else is rounded.
@@ -59,6 +65,8 @@ class Hyper:
     alpha: float = 0.25
     gamma: float = 1.01
     alpha_lowrank_only: bool = False
+    scaling: str = "column"      # "column" | "matrix" | "none"
+    residual: bool = True
 
 
 @dataclasses.dataclass
@@ -112,6 +120,12 @@ def column_factors(N: np.ndarray, R: np.ndarray, eps: float) -> np.ndarray:
     return np.sqrt((N * N).sum(axis=0)) / (np.sqrt((R * R).sum(axis=0)) + eps)
 
 
+def matrix_factor(N: np.ndarray, R: np.ndarray, eps: float) -> float:
+    """Norm-based scaling, matrix level (Eq. 9, with the + eps of Algorithm 1's
+    column form): phi = ||N||_F / (||R||_F + eps)."""
+    return float(np.sqrt((N * N).sum()) / (np.sqrt((R * R).sum()) + eps))
+
+
 def limiter_factor(norm_S: float, prev_norm: Optional[float], hp: Hyper) -> float:
     """Norm-growth limiter (Eq. 12 in Algorithm 1's form):
     lambda = gamma / max(||S|| / (||S_prev|| + eps), gamma);  1 on the first step."""
@@ -125,7 +139,18 @@ def _step_left(W, G, P, st: State, hp: Hyper):
     R = P.T @ G                                   # low-rank gradient
     S = G - P @ R                                 # (I - P P^T) G
     N = adam_direction(R, st, hp)                 # psi_t(R_t)
-    k = column_factors(N, R, hp.eps)              # K
+    if not hp.residual:                           # GaLore (Eq. 6): W <- W - eta alpha P N
+        st.t += 1
+        diag = dict(k=np.zeros(G.shape[1]), lam=1.0, norm_scaled=0.0, norm_after=st.prev_norm, R=R, N=N)
+        return W - hp.lr * hp.alpha * (P @ N), diag
+    if hp.scaling == "column":
+        k = column_factors(N, R, hp.eps)          # K
+    elif hp.scaling == "matrix":
+        k = np.full(G.shape[1], matrix_factor(N, R, hp.eps))
+    elif hp.scaling == "none":
+        k = np.ones(G.shape[1])
+    else:
+        raise ValueError(hp.scaling)
     S = S * k[None, :]                            # S[:, i] <- k_i S[:, i]
     norm_scaled = float(np.sqrt((S * S).sum()))
     lam = limiter_factor(norm_scaled, st.prev_norm, hp)

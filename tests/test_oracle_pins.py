@@ -38,9 +38,11 @@ HAND_HP = fo.Hyper(lr=1.0, beta1=0.5, beta2=0.75, eps=0.5, alpha=0.5, gamma=1.5)
 HADAMARD = 0.5 * np.array([[1.0, 1, 1, 1], [1, -1, 1, -1], [1, 1, -1, -1], [1, -1, -1, 1]])
 
 
-def hand_trajectory():
+def hand_trajectory(scaling="column", residual=True):
     """Expected W after steps 1..3, the factors and the limiter values, from the
-    closed forms above using scalar arithmetic only."""
+    closed forms above using scalar arithmetic only.  `scaling` and `residual`
+    select the ablation variants of Section 5.4 (matrix-level factor, factor 1,
+    no residual term)."""
     eps = 0.5
     shifts = [1.0, 2.0 / math.sqrt(7.0), 4.0 / math.sqrt(37.0)]
     resid_mult = [1.0, 3.0, 9.0]
@@ -55,6 +57,18 @@ def hand_trajectory():
             nn = math.sqrt(N[0][j] ** 2 + N[1][j] ** 2)
             rn = math.sqrt(R_ROWS[0][j] ** 2 + R_ROWS[1][j] ** 2)
             k.append(nn / (rn + eps))
+        if scaling == "matrix":
+            nn_all = math.sqrt(sum(N[i][j] ** 2 for i in range(2) for j in range(6)))
+            rn_all = math.sqrt(sum(R_ROWS[i][j] ** 2 for i in range(2) for j in range(6)))
+            k = [nn_all / (rn_all + eps)] * 6
+        elif scaling == "none":
+            k = [1.0] * 6
+        if not residual:
+            for j in range(6):
+                for i in range(2):
+                    W[i][j] -= 1.0 * 0.5 * N[i][j]
+            out.append(dict(W=np.array(W), k=np.zeros(6), lam=1.0, norm_after=None))
+            continue
         S = [[k[j] * resid_mult[step] * S_ROWS[i][j] for j in range(6)] for i in range(2)]
         norm = math.sqrt(sum(S[i][j] ** 2 for i in range(2) for j in range(6)))
         if prev is None:
@@ -144,6 +158,76 @@ def test_hand_case_right_projection():
     # constant low-rank gradient: M_3 = (1 - beta1^3) R, laid out m x r
     np.testing.assert_allclose(st.M, (1 - 0.5 ** 3) * R_ROWS.T, atol=1e-14)
     np.testing.assert_allclose(st.V, (1 - 0.75 ** 3) * (R_ROWS.T ** 2), atol=1e-14)
+
+
+@pytest.mark.parametrize("scaling,residual", [("matrix", True), ("none", True), ("column", False)])
+def test_hand_case_ablation_variants(scaling, residual):
+    """Fira-matrix (Eq. 9-10), Fira-w.o.-scaling and GaLore (Eq. 6) on the hand case: scalar
+    closed forms, three steps; the matrix-level and unit factors change which steps the
+    limiter cuts, the GaLore variant leaves the rows outside the subspace untouched."""
+    hp = fo.Hyper(**{**HAND_HP.__dict__, "scaling": scaling, "residual": residual})
+    st = fo.new_state(4, 6, 2)
+    W = W0_AXIS.copy()
+    lams = []
+    for G, want in zip(hand_gradients(), hand_trajectory(scaling, residual)):
+        W, d = fo.fira_step(W, G, P_AXIS, st, hp)
+        np.testing.assert_allclose(W, want["W"], rtol=0, atol=1e-12)
+        np.testing.assert_allclose(d["k"], want["k"], rtol=1e-13)
+        assert d["lam"] == pytest.approx(want["lam"], rel=1e-13)
+        assert (st.prev_norm is None) if want["norm_after"] is None else \
+            st.prev_norm == pytest.approx(want["norm_after"], rel=1e-13)
+        lams.append(d["lam"])
+    if residual:
+        assert lams[0] == 1.0 and lams[1] < 1.0 and lams[2] < 1.0      # residual x3 per step, gamma = 1.5
+    else:
+        np.testing.assert_array_equal(W[2:], W0_AXIS[2:])
+
+
+def test_unscaled_unlimited_variant_is_galore_add():
+    """Factor 1 and gamma = inf: Eq. 8, W - eta P psi(R) - eta (G - P R) (alpha = 1), with psi(R)
+    taken from the GaLore variant of the same state."""
+    rng = np.random.default_rng(11)
+    m, n, r = 7, 11, 3
+    W, proj = _random_problem(rng, m, n, r)
+    hp_add = fo.Hyper(lr=0.3, alpha=1.0, gamma=math.inf, scaling="none")
+    hp_gal = fo.Hyper(lr=0.3, alpha=1.0, residual=False)
+    st_a, st_g = fo.new_state(m, n, r), fo.new_state(m, n, r)
+    Wa, Wg = W.copy(), W.copy()
+    for _ in range(3):
+        G = rng.standard_normal((m, n))
+        Wa_new, _ = fo.fira_step(Wa, G, proj, st_a, hp_add)
+        Wg_new, _ = fo.fira_step(Wg, G, proj, st_g, hp_gal)
+        # same moments, so the GaLore step is eta P psi(R): add the raw residual to get Eq. 8
+        np.testing.assert_allclose(Wa - Wa_new, (Wg - Wg_new) + 0.3 * (G - proj @ (proj.T @ G)), atol=1e-12)
+        np.testing.assert_allclose(st_a.M, st_g.M, atol=0)
+        assert np.abs(proj.T @ ((Wg - Wg_new) - proj @ (proj.T @ (Wg - Wg_new)))).max() < 1e-12
+        Wa, Wg = Wa_new, Wg_new
+
+
+def test_matrix_level_factor_special_case_and_proportionality():
+    """(i) When every column of G is the same vector all column norms agree, so the matrix-level
+    factor of Eq. 9 equals every column factor of Eq. 11 (eps negligible): Fira-matrix = Fira.
+    (ii) In general the applied residual is ONE scalar times (I - P P^T) G, and that scalar is
+    ||N||_F / ||R||_F."""
+    rng = np.random.default_rng(12)
+    m, n, r = 6, 10, 2
+    W, proj = _random_problem(rng, m, n, r)
+    sa, sb = fo.new_state(m, n, r), fo.new_state(m, n, r)
+    Wa, Wb = W.copy(), W.copy()
+    for _ in range(3):
+        G = np.repeat(rng.standard_normal((m, 1)), n, axis=1)
+        Wa, _ = fo.fira_step(Wa, G, proj, sa, fo.Hyper(scaling="column", eps=1e-30))
+        Wb, _ = fo.fira_step(Wb, G, proj, sb, fo.Hyper(scaling="matrix", eps=1e-30))
+        np.testing.assert_allclose(Wa, Wb, rtol=0, atol=1e-13)
+    st = fo.new_state(m, n, r)
+    hp = fo.Hyper(lr=0.1, alpha=0.5, gamma=math.inf, scaling="matrix", eps=1e-30)
+    G = rng.standard_normal((m, n))
+    Wn, d = fo.fira_step(W, G, proj, st, hp)
+    S = (W - Wn) / (hp.lr * hp.alpha) - proj @ d["N"]
+    raw = G - proj @ (proj.T @ G)
+    ratio = S / raw
+    assert np.ptp(ratio) < 1e-10
+    assert ratio.mean() == pytest.approx(np.linalg.norm(d["N"]) / np.linalg.norm(d["R"]), rel=1e-12)
 
 
 def test_alpha_lowrank_only_reading():
