@@ -76,6 +76,11 @@ typedef enum { FIRA_F32 = 0, FIRA_BF16 = 1 } fira_dtype;
 #define FIRA_FLAG_ALPHA_LOWRANK_ONLY 1u /* G~ = alpha P N + S instead of alpha (P N + S) */
 #define FIRA_FLAG_AUTO_REFRESH 2u       /* fira_step() refreshes a matrix's projection when t mod T == 0 */
 #define FIRA_FLAG_FORCE_SIMT 4u         /* bf16 matrices also use the fp32 CUDA-core kernels */
+/* Ablation variants of Section 5.4 ("Ablation Study"); epilogue switches of the same kernels.  The
+ * first two exclude each other. */
+#define FIRA_FLAG_MATRIX_SCALING 8u     /* Fira-matrix: one factor ||N||_F / (||R||_F + eps) per matrix (Eq. 9-10) */
+#define FIRA_FLAG_NO_SCALING 16u        /* Fira-w.o.-scaling: the factor is 1 (with gamma = inf: GaLore-add, Eq. 8) */
+#define FIRA_FLAG_NO_RESIDUAL 32u       /* GaLore (Eq. 6): W <- W - lr alpha P N; the remembered norm is left alone */
 
 /* Inputs of Algorithm 1.  eps > 0; 0 <= beta < 1; gamma >= 1 or +inf; T >= 0 (0: never). */
 typedef struct {

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libfira.so")
 FIRA_OK = 0
 FIRA_F32, FIRA_BF16 = 0, 1
 FLAG_ALPHA_LOWRANK_ONLY, FLAG_AUTO_REFRESH, FLAG_FORCE_SIMT = 1, 2, 4
+FLAG_MATRIX_SCALING, FLAG_NO_SCALING, FLAG_NO_RESIDUAL = 8, 16, 32
 
 STATUS_NAMES = {0: "FIRA_OK", 1: "FIRA_ERR_INVALID_ARG", 2: "FIRA_ERR_WORKSPACE_TOO_SMALL",
                 3: "FIRA_ERR_UNSUPPORTED", 4: "FIRA_ERR_CUDA", 5: "FIRA_ERR_DEVICE_TIMEOUT",

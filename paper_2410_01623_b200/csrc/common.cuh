@@ -39,6 +39,7 @@ struct MatDev {
   float* Xt;          // scratch: l x r fp32, first N then X = a_low N - a_res lambda k R
   float* kvec;        // scratch: l factors
   float* part;        // scratch: partial sums of ||S||^2
+  float* aux;         // scratch: 2 l floats, ||N_l||^2 and ||R_l||^2 (matrix-level factor only)
   __nv_bfloat16* Nb;  // scratch of the tensor-core path: l x r bf16 N
   __nv_bfloat16* Rb;  //   "      l x r bf16 R
   __nv_bfloat16* Xb;  //   "      l x r bf16 X
@@ -56,6 +57,12 @@ struct MatDev {
 
 struct Hyper {
   float beta1, beta2, eps, lr, a_low, a_res, gamma;
+  unsigned mode;      // HYPER_* bits: ablation variants (Section 5.4)
+};
+enum HyperMode : unsigned {
+  HYPER_MATRIX_SCALING = 1u,   // one factor per matrix (Eq. 9)
+  HYPER_NO_SCALING = 2u,       // factor 1
+  HYPER_NO_RESIDUAL = 4u,      // no residual term (Eq. 6)
 };
 
 enum DeviceStatusBits : unsigned {

@@ -45,7 +45,7 @@ struct Layout {
   size_t off_mats = 0, off_status = 0, off_ints = 0, off_tcmaps = 0, off_work = 0;
   size_t ints_count = 0;
   // byte offsets per matrix inside the work area
-  std::vector<size_t> offRt, offXt, offK, offPart, offNb, offRb, offXb, offColpart, offGs, offWs;
+  std::vector<size_t> offRt, offXt, offK, offPart, offNb, offRb, offXb, offColpart, offGs, offWs, offAux;
   std::vector<int> engine;
   size_t step_work_bytes = 0, refresh_min_bytes = 0;
   size_t scratch_bytes = 0;

@@ -34,6 +34,9 @@ fira_status validate(const fira_hparams* hp, const fira_matrix_desc* descs, int3
   if (isnan(hp->gamma) || hp->gamma < 1.f) { set_error("gamma must be >= 1 or +inf"); return FIRA_ERR_INVALID_ARG; }
   if (!isfinite(hp->lr) || !isfinite(hp->alpha)) { set_error("lr and alpha must be finite"); return FIRA_ERR_INVALID_ARG; }
   if (hp->T < 0) { set_error("T must be >= 0"); return FIRA_ERR_INVALID_ARG; }
+  if ((hp->flags & FIRA_FLAG_MATRIX_SCALING) && (hp->flags & FIRA_FLAG_NO_SCALING)) {
+    set_error("FIRA_FLAG_MATRIX_SCALING and FIRA_FLAG_NO_SCALING exclude each other"); return FIRA_ERR_INVALID_ARG;
+  }
   for (int i = 0; i < count; ++i) {
     const fira_matrix_desc& d = descs[i];
     if (d.m <= 0 || d.n <= 0 || d.r <= 0 || d.r > std::min(d.m, d.n)) {
@@ -77,12 +80,13 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
   size_t refresh_max = 0;
   L.offRt.assign(count, 0); L.offXt.assign(count, 0); L.offK.assign(count, 0); L.offPart.assign(count, 0);
   L.offNb.assign(count, 0); L.offRb.assign(count, 0); L.offXb.assign(count, 0);
-  L.offColpart.assign(count, 0); L.offGs.assign(count, 0); L.offWs.assign(count, 0);
+  L.offColpart.assign(count, 0); L.offGs.assign(count, 0); L.offWs.assign(count, 0); L.offAux.assign(count, 0);
   for (int i = 0; i < count; ++i) {
     fira_matrix_desc d = descs[i];
     if (d.ld == 0) d.ld = d.n;
     const size_t ll = std::max(d.m, d.n), r = d.r;
     L.offK[i] = w; w += align_up(ll * 4);
+    L.offAux[i] = w; w += align_up(2 * ll * 4);
     if (L.engine[i] == 0) {
       const size_t tiles = (size_t)simt_tiles(d.m) * simt_tiles(d.n);
       L.offRt[i] = w; w += align_up(ll * r * 4);
@@ -121,6 +125,10 @@ static Hyper make_hyper(const fira_hparams& hp, float lr) {
   h.lr = lr < 0.f ? hp.lr : lr;
   h.a_low = hp.alpha;
   h.a_res = (hp.flags & FIRA_FLAG_ALPHA_LOWRANK_ONLY) ? 1.f : hp.alpha;
+  h.mode = 0;
+  if (hp.flags & FIRA_FLAG_MATRIX_SCALING) h.mode |= HYPER_MATRIX_SCALING;
+  if (hp.flags & FIRA_FLAG_NO_SCALING) h.mode |= HYPER_NO_SCALING;
+  if (hp.flags & FIRA_FLAG_NO_RESIDUAL) { h.mode |= HYPER_NO_RESIDUAL; h.a_res = 0.f; }
   h.gamma = hp.gamma;
   return h;
 }
@@ -196,6 +204,7 @@ fira_status fira_init(fira_ctx** out, const fira_hparams* hp, const fira_matrix_
     mt.V = (float*)(c->state_base + L.offV[i]);
     mt.sc = (MatScalars*)(c->state_base + L.offS[i]);
     mt.kvec = (float*)(c->work_base + L.offK[i]);
+    mt.aux = (float*)(c->work_base + L.offAux[i]);
     mt.part = (float*)(c->work_base + L.offPart[i]);
     if (mt.engine == 0) {
       mt.Rt = (float*)(c->work_base + L.offRt[i]);

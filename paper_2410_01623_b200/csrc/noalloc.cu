@@ -155,11 +155,16 @@ extern "C" fira_status fira_step_single_noalloc(const fira_hparams* hp, const fi
   pl.row_start = ints_dev + 3; pl.rows_total = mt.l;
   pl.w_tile_start = ints_dev + 5; pl.w_tiles = wtiles;
   pl.npart = ints_dev + 7;
+  if (hp->flags & (FIRA_FLAG_MATRIX_SCALING | FIRA_FLAG_NO_SCALING | FIRA_FLAG_NO_RESIDUAL)) {
+    set_error("fira_step_single_noalloc: the ablation-variant flags are not supported by this entry point");
+    return FIRA_ERR_UNSUPPORTED;
+  }
   Hyper h;
   h.beta1 = hp->beta1; h.beta2 = hp->beta2; h.eps = hp->eps;
   h.lr = lr < 0.f ? hp->lr : lr;
   h.a_low = hp->alpha;
   h.a_res = (hp->flags & FIRA_FLAG_ALPHA_LOWRANK_ONLY) ? 1.f : hp->alpha;
+  h.mode = 0;
   h.gamma = hp->gamma;
   PhaseTimer no_timer;
   launch_simt_step(pl, h, status_dev, st, &no_timer);

@@ -91,7 +91,15 @@ k_adam_rows(const MatDev* __restrict__ mats, const int* __restrict__ list, int n
     nn += __shfl_xor_sync(0xffffffffu, nn, o);
     rn += __shfl_xor_sync(0xffffffffu, rn, o);
   }
-  if (lane == 0) mt.kvec[l] = sqrtf(nn) / (sqrtf(rn) + hp.eps);
+  if (lane == 0) {
+    if (hp.mode & HYPER_MATRIX_SCALING) {        // the factor comes from the whole matrix: k_finalize
+      mt.aux[l] = nn; mt.aux[mt.l + l] = rn; mt.kvec[l] = 1.f;
+    } else if (hp.mode & HYPER_NO_SCALING) {
+      mt.kvec[l] = 1.f;
+    } else {
+      mt.kvec[l] = sqrtf(nn) / (sqrtf(rn) + hp.eps);
+    }
+  }
 }
 
 // ---------------------------------------------------------------- phases 3 and 6
@@ -192,9 +200,25 @@ k_finalize(const MatDev* __restrict__ mats, const int* __restrict__ list, int nl
   const int npart = npart_of[blockIdx.x];
   double acc = 0.0;
   for (int i = threadIdx.x; i < npart; i += 256) acc += (double)mt.part[i];
+  // Matrix-level factor (Eq. 9): the phases before ran with k = 1, so `part` holds ||G - P R||^2;
+  // the factor scales the norm here and fills the k table for the phases after.
+  float kmat = 1.f;
+  if (hp.mode & HYPER_MATRIX_SCALING) {
+    __shared__ double sn[256], sr[256];
+    double an = 0.0, ar = 0.0;
+    for (int i = threadIdx.x; i < mt.l; i += 256) { an += (double)mt.aux[i]; ar += (double)mt.aux[mt.l + i]; }
+    sn[threadIdx.x] = an; sr[threadIdx.x] = ar;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+      if (threadIdx.x < o) { sn[threadIdx.x] += sn[threadIdx.x + o]; sr[threadIdx.x] += sr[threadIdx.x + o]; }
+      __syncthreads();
+    }
+    kmat = (float)(sqrt(sn[0]) / (sqrt(sr[0]) + (double)hp.eps));
+    for (int i = threadIdx.x; i < mt.l; i += 256) mt.kvec[i] = kmat;
+  }
   float kmin = INFINITY, kmax = -INFINITY;
   for (int i = threadIdx.x; i < mt.l; i += 256) {
-    const float kv = mt.kvec[i];
+    const float kv = (hp.mode & HYPER_MATRIX_SCALING) ? kmat : mt.kvec[i];
     kmin = fminf(kmin, kv);
     kmax = fmaxf(kmax, kv);
   }
@@ -210,9 +234,17 @@ k_finalize(const MatDev* __restrict__ mats, const int* __restrict__ list, int nl
   }
   if (threadIdx.x == 0) {
     const double tot = sred[0] > 0.0 ? sred[0] : 0.0;
-    const float norm = (float)sqrt(tot);
+    const float norm = kmat * (float)sqrt(tot);
     const float prev = mt.sc->prev_norm;
     float lam = 1.f;
+    if (hp.mode & HYPER_NO_RESIDUAL) {           // Eq. 6: no residual, nothing to limit or remember
+      mt.sc->norm_scaled = 0.f;
+      mt.sc->lambda = 1.f;
+      mt.sc->k_min = 0.f;
+      mt.sc->k_max = 0.f;
+      mt.sc->t = mt.sc->t + 1;
+      return;
+    }
     if (prev >= 0.f && !isinf(hp.gamma)) {
       const float ratio = norm / (prev + hp.eps);
       lam = hp.gamma / fmaxf(ratio, hp.gamma);

@@ -177,7 +177,9 @@ k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, i
       rn += mt.colpart[(long long)(2 * q + 1) * mt.l + l];
     }
     for (int q = 2 * nparts; q < (2 + K1_GSQ_SPLIT) * nparts; ++q) gs += mt.colpart[(long long)q * mt.l + l];   // ||G_l||^2 in parts
-    const float k = sqrtf(nn) / (sqrtf(rn) + hp.eps);
+    float k = sqrtf(nn) / (sqrtf(rn) + hp.eps);
+    if (hp.mode & HYPER_MATRIX_SCALING) { mt.aux[l] = nn; mt.aux[mt.l + l] = rn; k = 1.f; }   // see k_finalize
+    if (hp.mode & HYPER_NO_SCALING) k = 1.f;
     mt.kvec[l] = k;
     contrib = k * k * fmaxf(gs - rn, 0.f);
   }

@@ -34,7 +34,10 @@ def rel_err(a: np.ndarray, b: np.ndarray) -> float:
 
 def oracle_hyper(hp: fb.Hparams) -> fo.Hyper:
     return fo.Hyper(lr=hp.lr, beta1=hp.beta1, beta2=hp.beta2, eps=hp.eps, alpha=hp.alpha,
-                    gamma=hp.gamma, alpha_lowrank_only=bool(hp.flags & fb.FLAG_ALPHA_LOWRANK_ONLY))
+                    gamma=hp.gamma, alpha_lowrank_only=bool(hp.flags & fb.FLAG_ALPHA_LOWRANK_ONLY),
+                    scaling=("matrix" if hp.flags & fb.FLAG_MATRIX_SCALING else
+                             "none" if hp.flags & fb.FLAG_NO_SCALING else "column"),
+                    residual=not (hp.flags & fb.FLAG_NO_RESIDUAL))
 
 
 class Trajectory:

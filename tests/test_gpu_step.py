@@ -70,6 +70,34 @@ def test_alpha_lowrank_only_flag():
     tr.assert_ok()
 
 
+@pytest.mark.parametrize("flags", [fb.FLAG_MATRIX_SCALING, fb.FLAG_NO_SCALING, fb.FLAG_NO_RESIDUAL,
+                                   fb.FLAG_NO_SCALING | fb.FLAG_ALPHA_LOWRANK_ONLY])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_ablation_variants(flags, dtype):
+    """Fira-matrix, Fira-w.o.-scaling and GaLore (Section 5.4, Eq. 6, 8, 9) as switches of the
+    same kernels, both orientations, with a jump that the limiter must cut where there is one."""
+    tr = _random_case([(150, 333), (333, 150), (64, 200)], [37, 37, 16], dtype, steps=5, seed=19,
+                      spike=(4,), flags=flags)
+    tr.assert_ok()
+    for i in range(3):
+        d = tr.f.diagnostics(i)
+        if flags & fb.FLAG_NO_RESIDUAL:
+            assert tr.st[i].prev_norm is None and d["lam"] == 1.0
+        else:
+            assert d["norm_prev"] == pytest.approx(tr.st[i].prev_norm, rel=1e-3 if dtype == torch.float32 else 2e-2)
+            if flags & fb.FLAG_MATRIX_SCALING:
+                assert d["k_min"] == d["k_max"]
+            if flags & fb.FLAG_NO_SCALING:
+                assert d["k_min"] == d["k_max"] == 1.0
+    if not flags & fb.FLAG_NO_RESIDUAL:
+        assert any(l < 1.0 for row in tr.lams for l in row)
+
+
+def test_variant_flags_that_exclude_each_other_are_rejected():
+    with pytest.raises(fb.FiraError):
+        fb.Fira([(64, 96)], 8, torch.float32, fb.make_hparams(flags=fb.FLAG_MATRIX_SCALING | fb.FLAG_NO_SCALING))
+
+
 @pytest.mark.parametrize("gamma", [math.inf, 1.0])
 def test_gamma_extremes(gamma):
     hp = fb.make_hparams(gamma=gamma)

@@ -122,6 +122,24 @@ def test_alpha_lowrank_only_and_gamma_inf_on_tensor_cores():
     assert all(l == 1.0 for row in tr.lams for l in row)
 
 
+@pytest.mark.parametrize("flags", [fb.FLAG_MATRIX_SCALING, fb.FLAG_NO_SCALING, fb.FLAG_NO_RESIDUAL])
+def test_ablation_variants_on_tensor_cores(flags):
+    """The ablation variants of Section 5.4 on the tensor-core kernels (left, right, odd width)."""
+    shapes = [(512, 768), (768, 512), (512, 1365)]
+    tr = _case(shapes, 128, steps=4, seed=43, spike=(3,), flags=flags)
+    assert [tr.f.diagnostics(i)["engine"] for i in range(3)] == [1, 1, 1]
+    tr.assert_ok()
+    for i in range(3):
+        d = tr.f.diagnostics(i)
+        if flags & fb.FLAG_NO_RESIDUAL:
+            assert tr.st[i].prev_norm is None
+        else:
+            assert d["norm_prev"] == pytest.approx(tr.st[i].prev_norm, rel=2e-2)
+            assert d["k_min"] == d["k_max"]
+    if not flags & fb.FLAG_NO_RESIDUAL:
+        assert any(l < 1.0 for row in tr.lams for l in row)
+
+
 def test_run_twice_is_bitwise_deterministic_on_tensor_cores():
     a = _case([(512, 1376), (1376, 512)], 128, steps=3, seed=37, spike=(2,))
     b = _case([(512, 1376), (1376, 512)], 128, steps=3, seed=37, spike=(2,))
