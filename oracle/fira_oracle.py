@@ -192,6 +192,23 @@ def fira_step(W: np.ndarray, G: np.ndarray, proj: np.ndarray, st: State, hp: Hyp
     return np.ascontiguousarray(Wn), diag
 
 
+def adam_dense_step(W: np.ndarray, G: np.ndarray, st: State, hp: Hyper, store: Optional[str] = None):
+    """Eq. 1-4 for a parameter that is not projected (embeddings, output head, norm gains: the
+    experiments follow GaLore's set-up, which leaves these to plain Adam):
+    W <- W - eta psi_t(G) with the moments of Eq. 2-3 in the shape of W.  st.M, st.V have W's shape."""
+    W = np.asarray(W, dtype=np.float64)
+    G = np.asarray(G, dtype=np.float64)
+    Wn = W - hp.lr * adam_direction(G, st, hp)
+    st.t += 1
+    if store == "bf16":
+        Wn = round_to_bf16(Wn)
+    elif store == "f32":
+        Wn = Wn.astype(np.float32).astype(np.float64)
+    elif store is not None:
+        raise ValueError(store)
+    return Wn
+
+
 def refresh_projection(G: np.ndarray, r: int) -> np.ndarray:
     """Eq. 7: G = U Sigma V^T, P = [u_1 .. u_r] (m <= n); for m > n the first r
     right singular vectors (n x r).  Full SVD by the library routine."""

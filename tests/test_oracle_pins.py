@@ -266,6 +266,30 @@ def test_full_rank_identity_projection_is_adam():
         np.testing.assert_allclose(W, p.detach().numpy(), rtol=0, atol=1e-13)
 
 
+def test_dense_adam_step_against_library_adam_and_first_step_closed_form():
+    """Plain Adam on an unprojected parameter: Eq. 4's form equals the library's Adam when its
+    epsilon is eps / sqrt(1 - beta2^s); with eps -> 0 the two coincide at every step.  First step:
+    W_1 = W_0 - eta G / (|G| + eps / sqrt(1 - beta2))."""
+    rng = np.random.default_rng(21)
+    W0 = rng.standard_normal((5, 7))
+    Gs = [rng.standard_normal((5, 7)) for _ in range(4)]
+    hp = fo.Hyper(lr=0.05, beta1=0.9, beta2=0.99, eps=1e-30)
+    st = fo.State(M=np.zeros((5, 7)), V=np.zeros((5, 7)))
+    Wt = torch.tensor(W0.copy(), dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([Wt], lr=0.05, betas=(0.9, 0.99), eps=1e-30)
+    W = W0.copy()
+    for G in Gs:
+        W = fo.adam_dense_step(W, G, st, hp)
+        Wt.grad = torch.tensor(G, dtype=torch.float64)
+        opt.step()
+        np.testing.assert_allclose(W, Wt.detach().numpy(), rtol=0, atol=1e-12)
+    assert st.t == 4
+    hp2 = fo.Hyper(lr=0.5, beta1=0.5, beta2=0.75, eps=0.5)
+    st2 = fo.State(M=np.zeros((5, 7)), V=np.zeros((5, 7)))
+    W1 = fo.adam_dense_step(W0, Gs[0], st2, hp2)
+    np.testing.assert_allclose(W1, W0 - 0.5 * Gs[0] / (np.abs(Gs[0]) + 0.5 / math.sqrt(0.25)), atol=1e-14)
+
+
 def test_first_step_closed_form():
     # s = 1: M = (1-b1) R, V = (1-b2) R^2  =>  N = R / (|R| + eps / sqrt(1-b2))
     rng = np.random.default_rng(3)
