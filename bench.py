@@ -82,6 +82,32 @@ KERNEL_MODEL = {
 }
 
 
+def time_adam_dense(dev, dtype, numel=64 * 1024 * 1024, tensors=2, iters=10):
+    """fira_adam_dense on `tensors` flat tensors of `numel` elements (far larger than L2):
+    achieved bytes per second against the measured copy bandwidth."""
+    import torch
+    from paper_2410_01623_b200 import binding as fb
+    hp = fb.make_hparams()
+    W = [torch.zeros(numel, dtype=dtype, device=dev) for _ in range(tensors)]
+    G = [torch.ones(numel, dtype=dtype, device=dev) for _ in range(tensors)]
+    M = [torch.zeros(numel, device=dev) for _ in range(tensors)]
+    V = [torch.zeros(numel, device=dev) for _ in range(tensors)]
+    for t in range(3):
+        fb.adam_dense(hp, W, G, M, V, t)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(iters):
+        fb.adam_dense(hp, W, G, M, V, 3 + t)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    es = 2 if dtype == torch.bfloat16 else 4
+    gbs = tensors * numel * (3 * es + 16) / (ms * 1e-3) / 1e9
+    peak = measured_peaks()["hbm_gbs"]
+    return {"ms": ms, "elements": tensors * numel, "bytes_per_element": 3 * es + 16, "GB/s": gbs,
+            "frac_of_hbm_peak": gbs / peak}
+
+
 class ClockSampler:
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -299,6 +325,11 @@ def main():
     status = f.poll()
     ms_step = max_over_ranks(ms_total, world, dev) / args.steps
 
+    # ---- plain Adam for unprojected parameters (fira_adam_dense): HBM-bound, timed on its own
+    adam_dense = None
+    if args.refresh != "none" and rank == 0:
+        adam_dense = time_adam_dense(dev, wl.torch_dtype)
+
     # ---- refresh, timed separately (one layer, scaled, unless --refresh full)
     refresh = None
     if args.refresh != "none" and rank == 0:
@@ -359,7 +390,7 @@ def main():
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
         "config": workload_config(wl, args), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-        "roofline": roofline, "cpu_baseline": cpu, "refresh": refresh, "device_status": status,
+        "roofline": roofline, "cpu_baseline": cpu, "refresh": refresh, "adam_dense": adam_dense, "device_status": status,
         "engines": sorted({f.diagnostics(i)["engine"] for i in range(0, nmat, max(1, nmat // 8))}),
     }
     print(json.dumps(line))

@@ -134,6 +134,20 @@ FIRA_API fira_status fira_init(fira_ctx** out, const fira_hparams* hp, const fir
  * "if t mod T = 0" branch). */
 FIRA_API fira_status fira_step(fira_ctx* ctx, void* const* W_dev, const void* const* G_dev, float lr);
 
+/* Plain Adam, Eq. 1-4 applied directly, for the parameters that are not projected (embeddings,
+ * output head, norm gains: Section 5.1 follows GaLore's set-up, which leaves these to Adam), so
+ * that a whole model can be stepped through this library:
+ *   M <- b1 M + (1-b1) G;  V <- b2 V + (1-b2) G^2;  W <- W - lr sqrt(1-b2^s)/(1-b1^s) M/(sqrt V + eps)
+ * with s = t + 1 (t = steps taken before this one; the caller counts).  W_dev, G_dev, M_dev, V_dev
+ * are host arrays of `count` device pointers (16-byte aligned) to flat tensors of numel[i]
+ * elements; W and G have type `dtype`, M and V are fp32 and owned by the caller (zero before the
+ * first step).  Uses beta1, beta2, eps of hp (alpha, gamma, T and the flags do not apply); lr < 0
+ * uses hp->lr.  Needs no context and no workspace.  Asynchronous on cuda_stream. */
+FIRA_API fira_status fira_adam_dense(const fira_hparams* hp, int32_t count, void* const* W_dev,
+                                     const void* const* G_dev, float* const* M_dev, float* const* V_dev,
+                                     const int64_t* numel, fira_dtype dtype, int64_t t, float lr,
+                                     void* cuda_stream);
+
 /* The same pass as fira_step() (Algorithm 1's loop body) for callers whose weights
  * and gradients live in HOST memory: W_host and G_host are host arrays of `count`
  * host pointers (m x ld elements each; page-locked memory makes the copies

@@ -76,6 +76,9 @@ SIGNATURES = {
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_float, C.c_void_p]),
     "fira_noalloc_max_scratch_bytes": (C.c_size_t, []),
+    "fira_adam_dense": (C.c_int, [C.POINTER(Hparams), C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
+                                  C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int,
+                                  C.c_int64, C.c_float, C.c_void_p]),
     "fira_status_string": (C.c_char_p, [C.c_int]),
     "fira_last_error": (C.c_char_p, []),
     "fira_destroy": (None, [C.c_void_p]),
@@ -115,6 +118,25 @@ def ptr_array(tensors: Sequence[Optional[torch.Tensor]]):
 def make_hparams(lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8, alpha=0.25, gamma=1.01, T=0,
                  flags=0) -> Hparams:
     return Hparams(beta1, beta2, eps, lr, alpha, gamma, T, flags)
+
+
+def adam_dense(hp: Hparams, Ws: Sequence[torch.Tensor], Gs: Sequence[torch.Tensor], Ms: Sequence[torch.Tensor],
+               Vs: Sequence[torch.Tensor], t: int, lr: Optional[float] = None) -> None:
+    """fira_adam_dense: one plain Adam step (Eq. 1-4) of a list of unprojected tensors, in place.
+    Argument marshalling only."""
+    n = len(Ws)
+    assert n == len(Gs) == len(Ms) == len(Vs) and n > 0
+    dt = Ws[0].dtype
+    for w, g, m, v in zip(Ws, Gs, Ms, Vs):
+        assert w.is_cuda and w.is_contiguous() and g.is_contiguous() and m.is_contiguous() and v.is_contiguous()
+        assert w.dtype == g.dtype == dt and m.dtype == v.dtype == torch.float32
+        assert w.numel() == g.numel() == m.numel() == v.numel()
+    numel = (C.c_int64 * n)(*[w.numel() for w in Ws])
+    stream = torch.cuda.current_stream(Ws[0].device).cuda_stream
+    with torch.cuda.device(Ws[0].device):
+        check(lib().fira_adam_dense(C.byref(hp), n, ptr_array(Ws), ptr_array(Gs), ptr_array(Ms), ptr_array(Vs),
+                                    numel, 1 if dt == torch.bfloat16 else 0, int(t),
+                                    -1.0 if lr is None else float(lr), C.c_void_p(stream)))
 
 
 class Fira:

@@ -8,7 +8,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libfira.so")
-SOURCES = ["fira_api.cu", "step_simt.cu", "step_tc.cu", "refresh.cu", "noalloc.cu"]
+SOURCES = ["fira_api.cu", "step_simt.cu", "step_tc.cu", "refresh.cu", "noalloc.cu", "adam_dense.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 
