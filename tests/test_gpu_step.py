@@ -243,3 +243,38 @@ def test_step_host_matches_device_step():
     torch.cuda.synchronize()
     for i in range(2):
         assert torch.equal(Wh[i], Wd[i].cpu())
+
+
+@pytest.mark.parametrize("dtype,shape,r,pad", [(torch.float32, (150, 333), 37, 5), (torch.float32, (333, 150), 37, 3),
+                                               (torch.bfloat16, (512, 768), 128, 8), (torch.bfloat16, (768, 512), 128, 64),
+                                               (torch.bfloat16, (512, 768), 128, 3), (torch.bfloat16, (300, 333), 37, 1)])
+def test_padded_row_pitch(dtype, shape, r, pad):
+    """W and G as views of wider buffers (ld = n + pad): the CUDA-core kernels, the tensor-core
+    kernels reading in place (pitch a multiple of 8 elements) and through aligned copies (odd
+    pitch).  The padding columns must come back untouched."""
+    m, n = shape
+    ld = n + pad
+    g = torch.Generator().manual_seed(m + pad)
+    hp = fb.make_hparams(lr=1e-2, alpha=0.25, gamma=1.01)
+    f = fb.Fira([shape], r, dtype, hp, lds=[ld])
+    q, _ = torch.linalg.qr(torch.randn(min(m, n), r, generator=g, dtype=torch.float64))
+    f.set_projection(0, q.to(dtype).cuda())
+    P = to_np64(f.get_projection(0))
+    Wbuf = torch.full((m, ld), 7.0, dtype=dtype, device="cuda")
+    Gbuf = torch.full((m, ld), float("nan"), dtype=dtype, device="cuda")     # the padding is never read
+    W0 = (torch.randn(m, n, generator=g) * 0.02).to(dtype)
+    Wbuf[:, :n] = W0.cuda()
+    st = fo.new_state(m, n, r)
+    ohp = fo.Hyper(lr=hp.lr, alpha=hp.alpha, gamma=hp.gamma, eps=hp.eps)
+    Wo = to_np64(W0)
+    kind = "bf16" if dtype == torch.bfloat16 else "f32"
+    for s_ in range(3):
+        G = torch.randn(m, n, generator=g).to(dtype)
+        Gbuf[:, :n] = G.cuda()
+        f.step([Wbuf], [Gbuf])
+        Wo, _ = fo.fira_step(Wo, to_np64(G), P, st, ohp, store=kind)
+    assert f.poll() == 0
+    assert rel_err(to_np64(Wbuf[:, :n]), Wo) <= (2e-2 if dtype == torch.bfloat16 else 1e-5)
+    assert rel_err(to_np64(Wbuf[:, :n]) - to_np64(W0), Wo - to_np64(W0)) <= (3e-2 if dtype == torch.bfloat16 else 2e-4)
+    assert (Wbuf[:, n:] == 7.0).all()
+
