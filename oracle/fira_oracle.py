@@ -42,6 +42,10 @@ design notes of the repository as well):
     "none" (Fira-w.o.-scaling: the factor is 1; without the limiter this is
     GaLore-add, Eq. 8); `residual=False` drops S altogether (GaLore, Eq. 6): then
     there is no norm to limit or to remember.
+  * Other base optimizers (Algorithm 2 names Adam and RMSProp as examples of the
+    adaptive optimizer; the appendix reports Fira + Adagrad): `psi` = "rmsprop" or
+    "adagrad" replaces Eq. 2-4 by the textbook update of that optimizer on R; the
+    paper gives no formulas for them.  M is then unused.
   * bf16 storage: when `store="bf16"` the new W is rounded to bfloat16
     (round to nearest, ties to even) after the update, because on that path W
     IS a bf16 tensor.  Nothing else is rounded.
@@ -66,6 +70,7 @@ class Hyper:
     gamma: float = 1.01
     alpha_lowrank_only: bool = False
     scaling: str = "column"      # "column" | "matrix" | "none"
+    psi: str = "adam"            # base optimizer psi_t: "adam" | "rmsprop" | "adagrad"
     residual: bool = True
 
 
@@ -107,6 +112,14 @@ def adam_direction(R: np.ndarray, st: State, hp: Hyper) -> np.ndarray:
     """Eq. 2-4 applied to the low-rank gradient (Algorithm 1, the psi_t block):
     M <- b1 M + (1-b1) R;  V <- b2 V + (1-b2) R^2;
     N = sqrt(1-b2^s)/(1-b1^s) * M / (sqrt(V) + eps), element-wise, s = t+1."""
+    if hp.psi == "rmsprop":     # Tieleman & Hinton: V <- b2 V + (1-b2) R^2, N = R / (sqrt V + eps)
+        st.V = hp.beta2 * st.V + (1.0 - hp.beta2) * (R * R)
+        return R / (np.sqrt(st.V) + hp.eps)
+    if hp.psi == "adagrad":     # Duchi et al.: V <- V + R^2, N = R / (sqrt V + eps)
+        st.V = st.V + R * R
+        return R / (np.sqrt(st.V) + hp.eps)
+    if hp.psi != "adam":
+        raise ValueError(hp.psi)
     s = st.t + 1
     st.M = hp.beta1 * st.M + (1.0 - hp.beta1) * R
     st.V = hp.beta2 * st.V + (1.0 - hp.beta2) * (R * R)

@@ -290,6 +290,28 @@ def test_dense_adam_step_against_library_adam_and_first_step_closed_form():
     np.testing.assert_allclose(W1, W0 - 0.5 * Gs[0] / (np.abs(Gs[0]) + 0.5 / math.sqrt(0.25)), atol=1e-14)
 
 
+@pytest.mark.parametrize("psi", ["rmsprop", "adagrad"])
+def test_other_base_optimizers_against_the_library(psi):
+    """r = m with P = I: no residual, and W <- W - eta alpha psi(G) must be the library's RMSprop /
+    Adagrad on the whole matrix (same eps placement: outside the square root)."""
+    rng = np.random.default_rng(31)
+    m, n = 4, 7
+    W0 = rng.standard_normal((m, n))
+    hp = fo.Hyper(lr=0.05, beta2=0.9, eps=1e-6, alpha=1.0, psi=psi)
+    st = fo.new_state(m, n, m)
+    Wt = torch.tensor(W0.copy(), dtype=torch.float64, requires_grad=True)
+    opt = (torch.optim.RMSprop([Wt], lr=0.05, alpha=0.9, eps=1e-6) if psi == "rmsprop"
+           else torch.optim.Adagrad([Wt], lr=0.05, eps=1e-6))
+    W = W0.copy()
+    for _ in range(4):
+        G = rng.standard_normal((m, n))
+        W, d = fo.fira_step(W, G, np.eye(m), st, hp)
+        Wt.grad = torch.tensor(G, dtype=torch.float64)
+        opt.step()
+        np.testing.assert_allclose(W, Wt.detach().numpy(), rtol=0, atol=1e-12)
+    assert np.all(st.M == 0.0)
+
+
 def test_first_step_closed_form():
     # s = 1: M = (1-b1) R, V = (1-b2) R^2  =>  N = R / (|R| + eps / sqrt(1-b2))
     rng = np.random.default_rng(3)
