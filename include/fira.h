@@ -81,6 +81,11 @@ typedef enum { FIRA_F32 = 0, FIRA_BF16 = 1 } fira_dtype;
 #define FIRA_FLAG_MATRIX_SCALING 8u     /* Fira-matrix: one factor ||N||_F / (||R||_F + eps) per matrix (Eq. 9-10) */
 #define FIRA_FLAG_NO_SCALING 16u        /* Fira-w.o.-scaling: the factor is 1 (with gamma = inf: GaLore-add, Eq. 8) */
 #define FIRA_FLAG_NO_RESIDUAL 32u       /* GaLore (Eq. 6): W <- W - lr alpha P N; the remembered norm is left alone */
+/* Another base optimizer psi_t in place of Adam's Eq. 2-4 (Algorithm 2 names RMSProp, the appendix
+ * reports Fira + Adagrad; the paper prints no formulas, the textbook ones are used).  M is unused.
+ * The two exclude each other. */
+#define FIRA_FLAG_PSI_RMSPROP 64u       /* V <- beta2 V + (1-beta2) R^2;  N = R / (sqrt V + eps) */
+#define FIRA_FLAG_PSI_ADAGRAD 128u      /* V <- V + R^2;                  N = R / (sqrt V + eps) */
 
 /* Inputs of Algorithm 1.  eps > 0; 0 <= beta < 1; gamma >= 1 or +inf; T >= 0 (0: never). */
 typedef struct {

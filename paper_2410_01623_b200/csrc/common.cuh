@@ -63,6 +63,8 @@ enum HyperMode : unsigned {
   HYPER_MATRIX_SCALING = 1u,   // one factor per matrix (Eq. 9)
   HYPER_NO_SCALING = 2u,       // factor 1
   HYPER_NO_RESIDUAL = 4u,      // no residual term (Eq. 6)
+  HYPER_PSI_RMSPROP = 8u,      // base optimizer: RMSProp instead of Adam
+  HYPER_PSI_ADAGRAD = 16u,     // base optimizer: Adagrad instead of Adam
 };
 
 enum DeviceStatusBits : unsigned {

@@ -37,6 +37,9 @@ fira_status validate(const fira_hparams* hp, const fira_matrix_desc* descs, int3
   if ((hp->flags & FIRA_FLAG_MATRIX_SCALING) && (hp->flags & FIRA_FLAG_NO_SCALING)) {
     set_error("FIRA_FLAG_MATRIX_SCALING and FIRA_FLAG_NO_SCALING exclude each other"); return FIRA_ERR_INVALID_ARG;
   }
+  if ((hp->flags & FIRA_FLAG_PSI_RMSPROP) && (hp->flags & FIRA_FLAG_PSI_ADAGRAD)) {
+    set_error("FIRA_FLAG_PSI_RMSPROP and FIRA_FLAG_PSI_ADAGRAD exclude each other"); return FIRA_ERR_INVALID_ARG;
+  }
   for (int i = 0; i < count; ++i) {
     const fira_matrix_desc& d = descs[i];
     if (d.m <= 0 || d.n <= 0 || d.r <= 0 || d.r > std::min(d.m, d.n)) {
@@ -129,6 +132,8 @@ static Hyper make_hyper(const fira_hparams& hp, float lr) {
   if (hp.flags & FIRA_FLAG_MATRIX_SCALING) h.mode |= HYPER_MATRIX_SCALING;
   if (hp.flags & FIRA_FLAG_NO_SCALING) h.mode |= HYPER_NO_SCALING;
   if (hp.flags & FIRA_FLAG_NO_RESIDUAL) { h.mode |= HYPER_NO_RESIDUAL; h.a_res = 0.f; }
+  if (hp.flags & FIRA_FLAG_PSI_RMSPROP) h.mode |= HYPER_PSI_RMSPROP;
+  if (hp.flags & FIRA_FLAG_PSI_ADAGRAD) h.mode |= HYPER_PSI_ADAGRAD;
   h.gamma = hp.gamma;
   return h;
 }

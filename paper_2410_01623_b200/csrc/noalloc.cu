@@ -155,8 +155,9 @@ extern "C" fira_status fira_step_single_noalloc(const fira_hparams* hp, const fi
   pl.row_start = ints_dev + 3; pl.rows_total = mt.l;
   pl.w_tile_start = ints_dev + 5; pl.w_tiles = wtiles;
   pl.npart = ints_dev + 7;
-  if (hp->flags & (FIRA_FLAG_MATRIX_SCALING | FIRA_FLAG_NO_SCALING | FIRA_FLAG_NO_RESIDUAL)) {
-    set_error("fira_step_single_noalloc: the ablation-variant flags are not supported by this entry point");
+  if (hp->flags & (FIRA_FLAG_MATRIX_SCALING | FIRA_FLAG_NO_SCALING | FIRA_FLAG_NO_RESIDUAL | FIRA_FLAG_PSI_RMSPROP |
+                   FIRA_FLAG_PSI_ADAGRAD)) {
+    set_error("fira_step_single_noalloc: the variant flags are not supported by this entry point");
     return FIRA_ERR_UNSUPPORTED;
   }
   Hyper h;

@@ -77,11 +77,20 @@ k_adam_rows(const MatDev* __restrict__ mats, const int* __restrict__ list, int n
   float nn = 0.f, rn = 0.f;
   for (int j = lane; j < mt.r; j += 32) {
     const float rv = mt.Rt[base + j];
-    const float mv = hp.beta1 * mt.M[base + j] + (1.f - hp.beta1) * rv;
-    const float vv = hp.beta2 * mt.V[base + j] + (1.f - hp.beta2) * rv * rv;
-    mt.M[base + j] = mv;
+    float vv, nv;
+    if (hp.mode & HYPER_PSI_RMSPROP) {
+      vv = hp.beta2 * mt.V[base + j] + (1.f - hp.beta2) * rv * rv;
+      nv = rv / (sqrtf(vv) + hp.eps);
+    } else if (hp.mode & HYPER_PSI_ADAGRAD) {
+      vv = mt.V[base + j] + rv * rv;
+      nv = rv / (sqrtf(vv) + hp.eps);
+    } else {
+      const float mv = hp.beta1 * mt.M[base + j] + (1.f - hp.beta1) * rv;
+      vv = hp.beta2 * mt.V[base + j] + (1.f - hp.beta2) * rv * rv;
+      mt.M[base + j] = mv;
+      nv = bias * mv / (sqrtf(vv) + hp.eps);
+    }
     mt.V[base + j] = vv;
-    const float nv = bias * mv / (sqrtf(vv) + hp.eps);
     mt.Xt[base + j] = nv;
     nn = fmaf(nv, nv, nn);
     rn = fmaf(rv, rv, rn);

@@ -515,7 +515,7 @@ fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntile
   static bool attr_set = false;
   static int num_sms = 0;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(k_tc_project<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(k_tc_project<EPI_PLAIN, PSI_ADAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, c->device);
     if (e != cudaSuccess) { set_error(std::string("refresh product set-up: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
     attr_set = true;
@@ -524,7 +524,7 @@ fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntile
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(table_dev);
   const ProjTileDesc* tiles = reinterpret_cast<const ProjTileDesc*>(table_dev + align_up(sizeof(TcMaps) * (size_t)njobs));
   Hyper hp{};
-  k_tc_project<EPI_PLAIN><<<2 * std::min(ntiles, num_sms / 2), K1_THREADS, K1_SMEM_BYTES, c->stream>>>(
+  k_tc_project<EPI_PLAIN, PSI_ADAM><<<2 * std::min(ntiles, num_sms / 2), K1_THREADS, K1_SMEM_BYTES, c->stream>>>(
       maps, tiles, ntiles, nullptr, hp, c->status_dev);
   return FIRA_OK;
 }
@@ -541,7 +541,9 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   if (!pl || pl->nlist == 0) return 0;
   cudaStream_t st = c->stream;
   if (!pl->attrs_set) {
-    cudaError_t e1 = cudaFuncSetAttribute(k_tc_project<EPI_ADAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
+    cudaError_t e1 = cudaFuncSetAttribute(k_tc_project<EPI_ADAM, PSI_ADAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
+    if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(k_tc_project<EPI_ADAM, PSI_RMSPROP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
+    if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(k_tc_project<EPI_ADAM, PSI_ADAGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
     cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES);
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
       set_error(std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
@@ -556,8 +558,16 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   k_tc_prep<<<(pl->nlist + 127) / 128, 128, 0, st>>>(mats, pl->list, pl->nlist, hp, pl->fast_dev);
   tm->mark(st);
   // both tensor kernels: clusters of two CTAs, at most one CTA per SM
-  k_tc_project<EPI_ADAM><<<2 * std::min(pl->k1_tiles, pl->num_sms / 2), K1_THREADS, K1_SMEM_BYTES, st>>>(
-      pl->maps_dev, pl->td1_dev, pl->k1_tiles, pl->fast_dev, hp, c->status_dev);
+  const int k1_grid = 2 * std::min(pl->k1_tiles, pl->num_sms / 2);
+  if (hp.mode & HYPER_PSI_RMSPROP)
+    k_tc_project<EPI_ADAM, PSI_RMSPROP><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(
+        pl->maps_dev, pl->td1_dev, pl->k1_tiles, pl->fast_dev, hp, c->status_dev);
+  else if (hp.mode & HYPER_PSI_ADAGRAD)
+    k_tc_project<EPI_ADAM, PSI_ADAGRAD><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(
+        pl->maps_dev, pl->td1_dev, pl->k1_tiles, pl->fast_dev, hp, c->status_dev);
+  else
+    k_tc_project<EPI_ADAM, PSI_ADAM><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(
+        pl->maps_dev, pl->td1_dev, pl->k1_tiles, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);
   k_tc_colfactors<<<pl->col_blocks, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->col_start, hp);
   tm->mark(st);

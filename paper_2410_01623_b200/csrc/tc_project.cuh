@@ -105,8 +105,11 @@ __device__ __forceinline__ ProjTileDesc load_desc(const ProjTileDesc* __restrict
 // projection refresh.  Then no M/V boxes are loaded, the output box of a row half is built in that
 // half's N/R buffer, and the loader and the G^2 warps have nothing to do.
 enum { EPI_ADAM = 0, EPI_PLAIN = 1 };
+// PSI: the base optimizer of the EPI_ADAM epilogue (0 Adam, Eq. 2-4; 1 RMSProp; 2 Adagrad: M is then
+// carried through unchanged).
+enum { PSI_ADAM = 0, PSI_RMSPROP = 1, PSI_ADAGRAD = 2 };
 
-template <int EPI>
+template <int EPI, int PSI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(K1_THREADS, 1)
 k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ tdesc, int total_tiles,
              const float* __restrict__ fast, Hyper hp, unsigned* __restrict__ status) {
@@ -453,9 +456,14 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             rv[e] = __uint_as_float(rr[8 * q + e]);
-            mo[e] = hp.beta1 * mo[e] + (1.f - hp.beta1) * rv[e];
-            vo[e] = hp.beta2 * vo[e] + (1.f - hp.beta2) * rv[e] * rv[e];
-            nv[e] = __fdividef(bias * mo[e], fast_sqrt(vo[e]) + hp.eps);
+            if (PSI == PSI_ADAM) {
+              mo[e] = hp.beta1 * mo[e] + (1.f - hp.beta1) * rv[e];
+              vo[e] = hp.beta2 * vo[e] + (1.f - hp.beta2) * rv[e] * rv[e];
+              nv[e] = __fdividef(bias * mo[e], fast_sqrt(vo[e]) + hp.eps);
+            } else {
+              vo[e] = PSI == PSI_RMSPROP ? hp.beta2 * vo[e] + (1.f - hp.beta2) * rv[e] * rv[e] : vo[e] + rv[e] * rv[e];
+              nv[e] = __fdividef(rv[e], fast_sqrt(vo[e]) + hp.eps);
+            }
             nn = fmaf(nv[e], nv[e], nn);
             rn = fmaf(rv[e], rv[e], rn);
           }

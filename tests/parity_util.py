@@ -37,7 +37,9 @@ def oracle_hyper(hp: fb.Hparams) -> fo.Hyper:
                     gamma=hp.gamma, alpha_lowrank_only=bool(hp.flags & fb.FLAG_ALPHA_LOWRANK_ONLY),
                     scaling=("matrix" if hp.flags & fb.FLAG_MATRIX_SCALING else
                              "none" if hp.flags & fb.FLAG_NO_SCALING else "column"),
-                    residual=not (hp.flags & fb.FLAG_NO_RESIDUAL))
+                    residual=not (hp.flags & fb.FLAG_NO_RESIDUAL),
+                    psi=("rmsprop" if hp.flags & fb.FLAG_PSI_RMSPROP else
+                         "adagrad" if hp.flags & fb.FLAG_PSI_ADAGRAD else "adam"))
 
 
 class Trajectory:

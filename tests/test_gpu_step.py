@@ -96,6 +96,24 @@ def test_ablation_variants(flags, dtype):
 def test_variant_flags_that_exclude_each_other_are_rejected():
     with pytest.raises(fb.FiraError):
         fb.Fira([(64, 96)], 8, torch.float32, fb.make_hparams(flags=fb.FLAG_MATRIX_SCALING | fb.FLAG_NO_SCALING))
+    with pytest.raises(fb.FiraError):
+        fb.Fira([(64, 96)], 8, torch.float32, fb.make_hparams(flags=fb.FLAG_PSI_RMSPROP | fb.FLAG_PSI_ADAGRAD))
+
+
+@pytest.mark.parametrize("flags", [fb.FLAG_PSI_RMSPROP, fb.FLAG_PSI_ADAGRAD, fb.FLAG_PSI_ADAGRAD | fb.FLAG_MATRIX_SCALING])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_other_base_optimizers(flags, dtype):
+    """RMSProp and Adagrad as the base optimizer (Algorithm 2's "adaptive optimizer" slot): M stays
+    zero, V follows the other rule, the factors and the limiter act on the new direction."""
+    tr = _random_case([(150, 333), (333, 150)], 37, dtype, steps=5, seed=23, spike=(4,), flags=flags,
+                      hp=fb.make_hparams(lr=1e-2, alpha=0.25, gamma=1.01, beta2=0.95, flags=flags))
+    tr.assert_ok()
+    for i in range(2):
+        M, V, pn, t = tr.f.get_state(i)
+        assert float(M.abs().max()) == 0.0
+        Vo = tr.st[i].V.T if tr.shapes[i][0] <= tr.shapes[i][1] else tr.st[i].V
+        assert rel_err(to_np64(V), Vo) < 1e-5
+        assert pn == pytest.approx(tr.st[i].prev_norm, rel=1e-3 if dtype == torch.float32 else 2e-2)
 
 
 @pytest.mark.parametrize("gamma", [math.inf, 1.0])

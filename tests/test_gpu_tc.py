@@ -140,6 +140,19 @@ def test_ablation_variants_on_tensor_cores(flags):
         assert any(l < 1.0 for row in tr.lams for l in row)
 
 
+@pytest.mark.parametrize("flags", [fb.FLAG_PSI_RMSPROP, fb.FLAG_PSI_ADAGRAD])
+def test_other_base_optimizers_on_tensor_cores(flags):
+    hp = fb.make_hparams(lr=1e-2, alpha=0.25, gamma=1.01, beta2=0.95, flags=flags)
+    tr = _case([(512, 768), (768, 512)], 128, steps=4, seed=47, spike=(3,), hp=hp)
+    assert [tr.f.diagnostics(i)["engine"] for i in range(2)] == [1, 1]
+    tr.assert_ok()
+    for i in range(2):
+        M, V, pn, t = tr.f.get_state(i)
+        assert float(M.abs().max()) == 0.0
+        Vo = tr.st[i].V.T if tr.shapes[i][0] <= tr.shapes[i][1] else tr.st[i].V
+        assert rel_err(to_np64(V), Vo) < 1e-5
+
+
 def test_run_twice_is_bitwise_deterministic_on_tensor_cores():
     a = _case([(512, 1376), (1376, 512)], 128, steps=3, seed=37, spike=(2,))
     b = _case([(512, 1376), (1376, 512)], 128, steps=3, seed=37, spike=(2,))
