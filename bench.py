@@ -74,7 +74,7 @@ ALU_FP32_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # "bytes" for the streaming kernels
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch on 2 layers of the llama-7b list
 # (profiles/k_tc_kernels_2layers_ncu_full.md)
-NCU_DRAM_BYTES_2_LAYERS = {"k_tc_project": 1.912e9 + 1.169e9, "k_tc_back_project": 2.004e9 + 0.779e9}
+NCU_DRAM_BYTES_2_LAYERS = {"k_tc_project": 1.916e9 + 1.172e9, "k_tc_back_project": 2.013e9 + 0.780e9}
 
 KERNEL_MODEL = {
     "k_project": ("alu", 0.5), "k_back_project<norm>": ("alu", 0.5), "k_back_project<update>": ("alu", 0.5),
