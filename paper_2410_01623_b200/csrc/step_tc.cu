@@ -512,14 +512,17 @@ fira_status tc_gemm_prepare(fira_ctx* c, const TcGemmJob* jobs, int njobs, char*
 }
 
 fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntiles) {
-  static bool attr_set = false;
-  static int num_sms = 0;
-  if (!attr_set) {
+  // the shared-memory attribute of a kernel is a per-device setting
+  static int sms_of_device[64] = {};
+  if (c->device < 0 || c->device >= 64) { set_error("refresh product: device index out of range"); return FIRA_ERR_CUDA; }
+  if (!sms_of_device[c->device]) {
+    int n = 0;
     cudaError_t e = cudaFuncSetAttribute(k_tc_project<EPI_PLAIN, PSI_ADAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, c->device);
-    if (e != cudaSuccess) { set_error(std::string("refresh product set-up: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
-    attr_set = true;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, c->device);
+    if (e != cudaSuccess || n <= 0) { set_error(std::string("refresh product set-up: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
+    sms_of_device[c->device] = n;
   }
+  const int num_sms = sms_of_device[c->device];
   if (ntiles == 0) return FIRA_OK;
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(table_dev);
   const ProjTileDesc* tiles = reinterpret_cast<const ProjTileDesc*>(table_dev + align_up(sizeof(TcMaps) * (size_t)njobs));
