@@ -17,8 +17,7 @@ whole algorithm applied to the transposed problem, so the factors are per row
 of G.  `fira_step` handles it by literally transposing W and G, running the
 m <= n code and transposing back.
 
-Readings of the paper where it is silent or inconsistent (all listed in the
-design notes of the repository as well):
+Readings of the paper where it is silent or inconsistent:
   * Bias-correction exponent: Algorithm 1 starts at t = 0 and increments after
     the update, which read literally gives 0/0 on the first step.  The exponent
     used is s = t + 1, the number of Adam updates including the current one,
