@@ -5,6 +5,7 @@ of each shape checked element by element against the fp64 oracle."""
 import pytest
 import torch
 
+from paper_2410_01623_b200 import binding as fb
 from paper_2410_01623_b200 import workloads as wk
 from tests.parity_util import workload_trajectory
 
@@ -32,3 +33,30 @@ def test_llama_1b_layer_odd_width_on_tensor_cores():
     tr.assert_ok()
     for i in (0, 4, 6):
         assert tr.f.diagnostics(i)["norm_prev"] == pytest.approx(tr.st[i].prev_norm, rel=2e-2)
+
+
+def test_two_7b_layers_run_twice_bitwise():
+    """Many tiles per CTA pair, every role of the persistent kernels re-entered hundreds of times:
+    two runs of the same three steps must agree bit for bit in W, in the moments and in the
+    diagnostics (which depend on the sums of G^2 taken inside the projection kernel)."""
+    wl = wk.workload("llama-7b", layers=2)
+
+    def run():
+        f = fb.Fira(wl.shapes, wl.r, wl.torch_dtype, fb.make_hparams(lr=wl.lr, alpha=wl.alpha), "cuda")
+        W = [wk.initial_weight(wl, i, "cuda") for i in range(len(wl.shapes))]
+        P = {}
+        for i, (m, n) in enumerate(wl.shapes):
+            if min(m, n) not in P:
+                P[min(m, n)] = wk.random_projection(wl, i, "cuda")
+            f.set_projection(i, P[min(m, n)])
+        for s in range(1, 4):
+            f.step(W, [wk.gradient(wl, i, s, "cuda") for i in range(len(wl.shapes))])
+        assert f.poll() == 0
+        return W, [f.diagnostics(i) for i in range(len(wl.shapes))], [f.get_state(i)[:2] for i in (0, 4, 6, 13)]
+
+    Wa, da, sa = run()
+    Wb, db, sb = run()
+    assert all(torch.equal(a, b) for a, b in zip(Wa, Wb))
+    assert da == db
+    assert all(torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]) for a, b in zip(sa, sb))
+
