@@ -60,3 +60,18 @@ def test_two_7b_layers_run_twice_bitwise():
     assert da == db
     assert all(torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]) for a, b in zip(sa, sb))
 
+
+def test_full_llama_7b_list_sampled_matrices():
+    """The whole benchmarked workload (224 matrices, 51 GB on the device) in exactly the launch
+    configuration that the benchmark times, one step; three matrices (first square one, a 4096 x 11008
+    in the middle, the last 11008 x 4096) are checked element by element against the oracle."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 70 * 2 ** 30:
+        pytest.skip("needs about 60 GB of free device memory")
+    wl = wk.workload("llama-7b")
+    assert len(wl.shapes) == 224
+    tr = workload_trajectory(wl, 1, gen_device="cuda", check=[0, 116, 223])
+    assert wl.shapes[116] == (4096, 11008) and wl.shapes[223] == (11008, 4096)
+    tr.assert_ok()
+    assert all(tr.f.diagnostics(i)["engine"] == 1 and tr.f.diagnostics(i)["t"] == 1 for i in (0, 116, 223))
+
