@@ -41,6 +41,13 @@ Readings of the paper where it is silent or inconsistent:
     "none" (Fira-w.o.-scaling: the factor is 1; without the limiter this is
     GaLore-add, Eq. 8); `residual=False` drops S altogether (GaLore, Eq. 6): then
     there is no norm to limit or to remember.
+  * Fira-only-scaling (appendix "Theoretical Analysis", item "Variability of Scaling
+    Factor", and the only-scaling equation of the appendix on Fira versus full-rank
+    Adam): W <- W - eta phi(R) G.  `only_scaling=True` takes it as Algorithm 1 with the
+    scaled matrix S := G diag(k) in place of the scaled residual and without the P N
+    term; alpha and the limiter act on that S exactly as they act on the residual in
+    Algorithm 1 (alpha = 1 or `alpha_lowrank_only`, and gamma = inf, give the printed
+    equation literally).  Column and matrix level as for `scaling`.
   * Other base optimizers (Algorithm 2 names Adam and RMSProp as examples of the
     adaptive optimizer; the appendix reports Fira + Adagrad): `psi` = "rmsprop" or
     "adagrad" replaces Eq. 2-4 by the textbook update of that optimizer on R; the
@@ -71,6 +78,7 @@ class Hyper:
     scaling: str = "column"      # "column" | "matrix" | "none"
     psi: str = "adam"            # base optimizer psi_t: "adam" | "rmsprop" | "adagrad"
     residual: bool = True
+    only_scaling: bool = False   # Fira-only-scaling: W <- W - eta phi(R) G
 
 
 @dataclasses.dataclass
@@ -163,15 +171,18 @@ def _step_left(W, G, P, st: State, hp: Hyper):
         k = np.ones(G.shape[1])
     else:
         raise ValueError(hp.scaling)
+    if hp.only_scaling:                           # the factors act on the whole gradient
+        S = G
     S = S * k[None, :]                            # S[:, i] <- k_i S[:, i]
     norm_scaled = float(np.sqrt((S * S).sum()))
     lam = limiter_factor(norm_scaled, st.prev_norm, hp)
     S = S * lam
     st.prev_norm = float(np.sqrt((S * S).sum()))  # norm after limiting
+    low = np.zeros_like(G) if hp.only_scaling else P @ N
     if hp.alpha_lowrank_only:
-        Gt = hp.alpha * (P @ N) + S
+        Gt = hp.alpha * low + S
     else:
-        Gt = hp.alpha * (P @ N + S)               # G~ = alpha (P N + S)
+        Gt = hp.alpha * (low + S)                 # G~ = alpha (P N + S)
     st.t += 1
     diag = dict(k=k, lam=lam, norm_scaled=norm_scaled, norm_after=st.prev_norm,
                 R=R, N=N)

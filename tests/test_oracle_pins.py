@@ -230,6 +230,96 @@ def test_matrix_level_factor_special_case_and_proportionality():
     assert ratio.mean() == pytest.approx(np.linalg.norm(d["N"]) / np.linalg.norm(d["R"]), rel=1e-12)
 
 
+def only_scaling_hand_trajectory(scaling="column"):
+    """Fira-only-scaling on the hand case, scalar arithmetic only: every entry of W moves by
+    eta alpha lambda k_j G_ij (no P N term), and the norm that the limiter sees is that of the
+    whole scaled gradient, rows inside the subspace included."""
+    eps = 0.5
+    shifts = [1.0, 2.0 / math.sqrt(7.0), 4.0 / math.sqrt(37.0)]
+    W = [[W0_AXIS[i][j] for j in range(6)] for i in range(4)]
+    prev = None
+    out = []
+    for step, mult in enumerate((1.0, 3.0, 9.0)):
+        e = shifts[step]
+        N = [[R_ROWS[i][j] / (abs(R_ROWS[i][j]) + e) for j in range(6)] for i in range(2)]
+        k = []
+        for j in range(6):
+            nn = math.sqrt(N[0][j] ** 2 + N[1][j] ** 2)
+            rn = math.sqrt(R_ROWS[0][j] ** 2 + R_ROWS[1][j] ** 2)
+            k.append(nn / (rn + eps))
+        if scaling == "matrix":
+            nn_all = math.sqrt(sum(N[i][j] ** 2 for i in range(2) for j in range(6)))
+            rn_all = math.sqrt(sum(R_ROWS[i][j] ** 2 for i in range(2) for j in range(6)))
+            k = [nn_all / (rn_all + eps)] * 6
+        G = [[R_ROWS[i][j] for j in range(6)] for i in range(2)] + \
+            [[mult * S_ROWS[i][j] for j in range(6)] for i in range(2)]
+        norm = math.sqrt(sum((k[j] * G[i][j]) ** 2 for i in range(4) for j in range(6)))
+        if prev is None:
+            lam = 1.0
+        else:
+            ratio = norm / (prev + eps)
+            lam = 1.5 / ratio if ratio > 1.5 else 1.0
+        prev = lam * norm
+        for i in range(4):
+            for j in range(6):
+                W[i][j] -= 1.0 * 0.5 * lam * k[j] * G[i][j]
+        out.append(dict(W=np.array(W), k=np.array(k), lam=lam, norm_after=prev))
+    return out
+
+
+@pytest.mark.parametrize("scaling", ["column", "matrix"])
+def test_only_scaling_hand_case(scaling):
+    """Fira-only-scaling, W <- W - eta phi(R) G (appendix, "Variability of Scaling Factor"), column
+    and matrix level, on the hand case in three bases (axis projection, dense rotated projection,
+    transposed problem)."""
+    exp = only_scaling_hand_trajectory(scaling)
+    assert exp[1]["lam"] < 1.0                                    # the limiter acts on the scaled gradient
+    hp = fo.Hyper(**{**HAND_HP.__dict__, "scaling": scaling, "only_scaling": True})
+    st, st_h, st_t = fo.new_state(4, 6, 2), fo.new_state(4, 6, 2), fo.new_state(6, 4, 2)
+    W, Wh = W0_AXIS.copy(), HADAMARD @ W0_AXIS
+    Wt = np.ascontiguousarray(Wh.T)
+    for step, G in enumerate(hand_gradients()):
+        W, d = fo.fira_step(W, G, P_AXIS, st, hp)
+        np.testing.assert_allclose(W, exp[step]["W"], rtol=0, atol=1e-13)
+        np.testing.assert_allclose(d["k"], exp[step]["k"], rtol=0, atol=1e-14)
+        assert d["lam"] == pytest.approx(exp[step]["lam"], abs=1e-14)
+        assert st.prev_norm == pytest.approx(exp[step]["norm_after"], abs=1e-13)
+        Wh, _ = fo.fira_step(Wh, HADAMARD @ G, HADAMARD @ P_AXIS, st_h, hp)
+        np.testing.assert_allclose(Wh, HADAMARD @ exp[step]["W"], rtol=0, atol=1e-13)
+        Wt, _ = fo.fira_step(Wt, np.ascontiguousarray((HADAMARD @ G).T), HADAMARD @ P_AXIS, st_t, hp)
+        np.testing.assert_allclose(Wt, (HADAMARD @ exp[step]["W"]).T, rtol=0, atol=1e-13)
+    # literal numbers of step 1: k_1 = 1/3, G[0,1] = 1, G[2,1] = 2 -> both rows move, by k eta alpha G
+    first = only_scaling_hand_trajectory(scaling)[0]["W"] if scaling == "column" else None
+    if first is not None:
+        assert first[0, 1] == pytest.approx(-1.0 - 0.5 * (1.0 / 3.0) * 1.0, abs=1e-15)
+        assert first[2, 1] == pytest.approx(2.5 - 0.5 * (1.0 / 3.0) * 2.0, abs=1e-15)
+
+
+def test_only_scaling_printed_equation():
+    """alpha = 1 and gamma = inf give the printed equation literally: (W_t - W_{t+1}) / eta is G with
+    column j multiplied by k_j, the factors being those of the ordinary Fira step on the same state;
+    the moments advance exactly as in the ordinary step."""
+    rng = np.random.default_rng(17)
+    m, n, r = 7, 12, 3
+    W, proj = _random_problem(rng, m, n, r)
+    hp_only = fo.Hyper(lr=0.2, alpha=1.0, gamma=math.inf, only_scaling=True)
+    hp_fira = fo.Hyper(lr=0.2, alpha=1.0, gamma=math.inf)
+    so, sf = fo.new_state(m, n, r), fo.new_state(m, n, r)
+    Wo, Wf = W.copy(), W.copy()
+    for _ in range(3):
+        G = rng.standard_normal((m, n))
+        Wo_new, do = fo.fira_step(Wo, G, proj, so, hp_only)
+        Wf, df = fo.fira_step(Wf, G, proj, sf, hp_fira)
+        np.testing.assert_allclose(do["k"], df["k"], rtol=0, atol=0)
+        k_direct = np.array([np.linalg.norm(df["N"][:, j]) / (np.linalg.norm((proj.T @ G)[:, j]) + hp_only.eps)
+                             for j in range(n)])
+        np.testing.assert_allclose((Wo - Wo_new) / 0.2, G * k_direct[None, :], rtol=0, atol=1e-13)
+        np.testing.assert_array_equal(so.M, sf.M)
+        np.testing.assert_array_equal(so.V, sf.V)
+        assert so.prev_norm == pytest.approx(np.linalg.norm(G * k_direct[None, :]), rel=1e-13)
+        Wo = Wo_new
+
+
 def test_alpha_lowrank_only_reading():
     exp = hand_trajectory()[0]
     hp = copy.copy(HAND_HP)
