@@ -70,16 +70,32 @@ def measured_peaks():
 # fp32 CUDA-core peak: 148 SMs x 128 FMA lanes x 2 flop x 1.965 GHz (maximum SM clock)
 ALU_FP32_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
-# kernel name -> (bound, algorithmic share): flops as a fraction of the step's 4mnr, or
-# "bytes" for the streaming kernels
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch on 2 layers of the llama-7b list
-# (profiles/k_tc_kernels_2layers_ncu_full.md)
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from an ncu capture of 2 layers of
+# the llama-7b list (every layer has the same shapes, so the traffic of a full launch is this times
+# the layer ratio).  None: the kernel has changed since its counters were taken.
 NCU_DRAM_BYTES_2_LAYERS = {"k_tc_project": 1.916e9 + 1.172e9, "k_tc_back_project": 2.013e9 + 0.780e9}
 
-KERNEL_MODEL = {
+# kernel name -> (pipe that does its arithmetic, share of the step's 4 m n r flops)
+KERNEL_PIPE = {
     "k_project": ("alu", 0.5), "k_back_project<norm>": ("alu", 0.5), "k_back_project<update>": ("alu", 0.5),
     "k_tc_project": ("tensor", 0.5), "k_tc_back_project": ("tensor", 0.5),
 }
+
+
+def kernel_min_bytes(name, wl):
+    """The kernel's share of the step's minimum bytes: the projection product reads G and the
+    projection once and moves the fp32 moments in and out; the back-projection reads and writes W.
+    (What the two exchange through scratch memory -- N, R, X -- and the second pass over G are not
+    algorithmic bytes.)"""
+    e = 2 if wl.dtype == "bf16" else 4
+    by = 0
+    for (m, n) in wl.shapes:
+        l, d = max(m, n), min(m, n)
+        if "back_project" in name:
+            by += 2 * e * m * n
+        elif "project" in name:
+            by += e * m * n + e * wl.r * d + 16 * wl.r * l
+    return by
 
 
 def time_adam_dense(dev, dtype, numel=64 * 1024 * 1024, tensors=2, iters=10):
@@ -340,7 +356,7 @@ def main():
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) * 1e3
         refresh = {"ms": dt * (nmat / len(which)), "measured_on": f"{len(which)} of {nmat} matrices",
-                   "iters": "library default"}
+                   "rounds": 4, "iters": "library default (4 rounds)"}
 
     # ---- end to end through the host-buffer entry point
     e2e = None
@@ -357,28 +373,50 @@ def main():
 
     peaks = measured_peaks()
     fl, by = flops_and_bytes(wl)
-    roof_ms = max(fl / (peaks["bf16_tflops_sustained"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    # the step's roofline: the slower of the two products at the tensor peak and the minimum bytes at
+    # the copy bandwidth; the sustained tensor figure applies to a kernel timed inside a long step,
+    # the burst figure is given beside it
+    t_hbm = by / (peaks["hbm_gbs"] * 1e9)
+    pipe_peak = peaks["bf16_tflops_sustained"] if wl.dtype == "bf16" else ALU_FP32_TFLOPS
+    roof_ms = max(fl / (pipe_peak * 1e12), t_hbm) * 1e3
+    roof_ms_burst = max(fl / ((peaks["bf16_tflops"] if wl.dtype == "bf16" else ALU_FP32_TFLOPS) * 1e12), t_hbm) * 1e3
     top = max(phases, key=lambda p: p[1]) if phases else ("", 0.0)
-    bound, share = KERNEL_MODEL.get(top[0], ("hbm", None))
-    if bound == "tensor":
-        peak, unit, ach = peaks["bf16_tflops_sustained"], "TFLOP/s", fl * share / (top[1] * 1e-3) / 1e12
-        peak_kind = f"cuBLAS bf16 sustained, {peaks['source']}"
-    elif bound == "alu":
-        peak, unit, ach = ALU_FP32_TFLOPS, "TFLOP/s", fl * share / (top[1] * 1e-3) / 1e12
-        peak_kind = "fp32 FMA: 148 SMs x 128 lanes x 2 x 1.965 GHz (derived)"
+    pipe, share = KERNEL_PIPE.get(top[0], ("hbm", None))
+    kbytes = kernel_min_bytes(top[0], wl)
+    kflops = fl * share if share else 0.0
+    if pipe == "tensor":
+        ppeak, peak_kind = peaks["bf16_tflops_sustained"], f"cuBLAS bf16 sustained, {peaks['source']}"
+    elif pipe == "alu":
+        ppeak, peak_kind = ALU_FP32_TFLOPS, "fp32 FMA: 148 SMs x 128 lanes x 2 x 1.965 GHz (derived)"
     else:
-        peak, unit, ach = peaks["hbm_gbs"], "GB/s", None
+        ppeak, peak_kind = None, None
+    # which roof bounds THIS kernel on THIS workload: its flop time against its byte time
+    if ppeak is not None and kflops / (ppeak * 1e12) >= kbytes / (peaks["hbm_gbs"] * 1e9):
+        bound, peak, unit, ach = pipe, ppeak, "TFLOP/s", kflops / (top[1] * 1e-3) / 1e12
+    else:
+        bound, peak, unit = "hbm", peaks["hbm_gbs"], "GB/s"
+        ach = kbytes / (top[1] * 1e-3) / 1e9 if kbytes else None
         peak_kind = f"copy bandwidth, {peaks['source']}"
-    # DRAM bytes per launch from the ncu capture summarised under profiles/ (2 of the 32 layers,
-    # scaled by the layer count: every layer has the same shapes, so traffic grows in proportion)
+    # DRAM bytes per launch from an ncu capture of 2 of the 32 layers, scaled by the layer count
     traffic = None
-    if wl.name == "llama-7b" and top[0] in NCU_DRAM_BYTES_2_LAYERS:
+    if wl.name == "llama-7b" and NCU_DRAM_BYTES_2_LAYERS.get(top[0]):
         traffic = NCU_DRAM_BYTES_2_LAYERS[top[0]] * (nmat / 14.0)
     roofline = {"kernel": top[0], "bound": bound, "achieved": ach, "peak": peak, "unit": unit,
                 "frac": (ach / peak) if ach else None, "traffic": traffic, "peak_kind": peak_kind,
+                "frac_of_burst_peak": (ach / peaks["bf16_tflops"]) if (ach and bound == "tensor") else None,
                 "kernel_ms": top[1], "kernel_share": top[1] / max(sum(p[1] for p in phases), 1e-9),
+                "kernel_algorithmic_bytes": kbytes, "kernel_algorithmic_flops": kflops,
                 "step_roofline_ms": roof_ms, "step_frac_of_roofline": roof_ms / ms_step,
+                "step_roofline_ms_burst": roof_ms_burst, "step_frac_of_roofline_burst": roof_ms_burst / ms_step,
                 "phases_ms": {k: round(v, 4) for k, v in phases}, "phase_steps": nrec}
+    if refresh is not None:
+        # Eq. 7 by subspace iteration: 2 q + 1 big products of 2 m n r flops each (q rounds)
+        q = refresh["rounds"]
+        rfl = (2 * q + 1) * fl / 2
+        rpeak = peaks["bf16_tflops_sustained"] if wl.dtype == "bf16" else ALU_FP32_TFLOPS
+        refresh["achieved_tflops"] = rfl / (refresh["ms"] * 1e-3) / 1e12
+        refresh["frac"] = refresh["achieved_tflops"] / rpeak
+        refresh["peak_tflops"] = rpeak
 
     cpu = None
     if not args.no_cpu_baseline:

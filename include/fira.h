@@ -86,6 +86,14 @@ typedef enum { FIRA_F32 = 0, FIRA_BF16 = 1 } fira_dtype;
  * The two exclude each other. */
 #define FIRA_FLAG_PSI_RMSPROP 64u       /* V <- beta2 V + (1-beta2) R^2;  N = R / (sqrt V + eps) */
 #define FIRA_FLAG_PSI_ADAGRAD 128u      /* V <- V + R^2;                  N = R / (sqrt V + eps) */
+/* Fira-only-scaling (appendix "Theoretical Analysis", item "Variability of Scaling Factor"; the
+ * only-scaling equation of the appendix on Fira versus full-rank Adam):  W <- W - lr phi(R) G.  The
+ * factors k of Eq. 11 (or the one factor of Eq. 9 with FIRA_FLAG_MATRIX_SCALING) multiply the whole
+ * gradient and the P N term is dropped.  Taken as Algorithm 1 with S := G diag(k): alpha and the
+ * limiter act on it as they act on the scaled residual (alpha = 1 or FIRA_FLAG_ALPHA_LOWRANK_ONLY
+ * together with gamma = inf give the printed equation literally).  M and V advance as usual.
+ * Excludes FIRA_FLAG_NO_RESIDUAL. */
+#define FIRA_FLAG_ONLY_SCALING 256u
 
 /* Inputs of Algorithm 1.  eps > 0; 0 <= beta < 1; gamma >= 1 or +inf; T >= 0 (0: never). */
 typedef struct {
@@ -177,6 +185,14 @@ FIRA_API fira_status fira_refresh_projection(fira_ctx* ctx, const void* const* G
                                              const int32_t* which, int32_t nwhich, uint64_t seed,
                                              int32_t iters);
 
+/* The same refresh; in addition, for every selected matrix i with basis_f32_dev[i] != NULL (a host
+ * array of `count` device pointers, 16-byte aligned, d x r floats each), the basis of Eq. 7 is
+ * also written there in fp32, as it stands before it is rounded to the matrix's storage type.
+ * For a bf16 matrix the stored projection differs from it by one bf16 rounding per entry. */
+FIRA_API fira_status fira_refresh_projection_f32(fira_ctx* ctx, const void* const* G_dev,
+                                                 const int32_t* which, int32_t nwhich, uint64_t seed,
+                                                 int32_t iters, float* const* basis_f32_dev);
+
 /* Copy a projection (d x r, row major, the matrix's dtype) from / to device memory
  * (the P_t of Algorithm 1, given by the caller instead of Eq. 7). */
 FIRA_API fira_status fira_set_projection(fira_ctx* ctx, int32_t idx, const void* P_dev);
@@ -200,6 +216,15 @@ FIRA_API fira_status fira_get_diagnostics(fira_ctx* ctx, int32_t idx, fira_diag*
 /* Reads the device status word (waits for the stream): FIRA_OK, or the first
  * device-side condition recorded since the last poll, which it clears. */
 FIRA_API fira_status fira_poll(fira_ctx* ctx);
+
+/* Self-test of the failure path of the tensor-core kernels (the paper has no counterpart).  Every
+ * wait inside those kernels is bounded: a wait that runs out raises a flag that all roles of the
+ * block poll, the kernel returns, and the time-out shows up in fira_poll().  This call enqueues a
+ * one-block kernel whose wait can never be satisfied (a barrier that nothing arrives on, no copy in
+ * flight) with a limit of `rounds` tries (1 .. 2^20), so that the path can be exercised without
+ * disturbing anything: afterwards fira_poll() returns FIRA_ERR_DEVICE_TIMEOUT once, then FIRA_OK,
+ * and the context steps on as before. */
+FIRA_API fira_status fira_selftest_bounded_wait(fira_ctx* ctx, int32_t rounds);
 
 /* Number of kernel launches enqueued by the most recent fira_step() call. */
 FIRA_API int32_t fira_last_step_launches(const fira_ctx* ctx);
@@ -238,16 +263,23 @@ FIRA_API const char* fira_phase_name(const fira_ctx* ctx, int32_t phase);
  * the device (0 before the first step); both are updated.  lr < 0 uses hp->lr.
  * The result equals fira_step()'s for the same matrix on the CUDA-core kernels.
  *
- * The first call on a device looks up the array's device address; make that call
- * before any stream capture starts.  All calls share the one array, which keeps the
- * previous call's contents (each call rewrites or clears what it reads), so calls
- * that overlap on the GPU -- from different streams or threads -- race: issue them on
- * one stream or wait in between. */
+ * Host-side argument errors (including the variant flags, none of which this entry
+ * point supports: FIRA_ERR_UNSUPPORTED) are returned before anything is enqueued.
+ * Device-side conditions (a non-finite norm) are recorded in a status word inside the
+ * array; fira_noalloc_poll() waits for the given stream, returns FIRA_OK or the
+ * condition, and clears it (it allocates nothing either).
+ *
+ * The first call on a device looks up the array's device address (host threads may
+ * race to it: the look-up is serialised); make that call before any stream capture
+ * starts.  All calls share the one array, which keeps the previous call's contents
+ * (each call rewrites what it reads), so calls that overlap on the GPU -- from
+ * different streams or threads -- race: issue them on one stream or wait in between. */
 FIRA_API fira_status fira_step_single_noalloc(const fira_hparams* hp, const fira_matrix_desc* desc,
                                               void* W_dev, const void* G_dev, const void* P_dev,
                                               float* M_dev, float* V_dev, float* norm_prev_dev,
                                               int64_t* t_dev, float lr, void* cuda_stream);
 FIRA_API size_t fira_noalloc_max_scratch_bytes(void);
+FIRA_API fira_status fira_noalloc_poll(void* cuda_stream);
 
 FIRA_API const char* fira_status_string(fira_status s);
 /* Text of the most recent error on this thread ("" if none). */

@@ -21,6 +21,7 @@ FIRA_F32, FIRA_BF16 = 0, 1
 FLAG_ALPHA_LOWRANK_ONLY, FLAG_AUTO_REFRESH, FLAG_FORCE_SIMT = 1, 2, 4
 FLAG_MATRIX_SCALING, FLAG_NO_SCALING, FLAG_NO_RESIDUAL = 8, 16, 32
 FLAG_PSI_RMSPROP, FLAG_PSI_ADAGRAD = 64, 128
+FLAG_ONLY_SCALING = 256
 
 STATUS_NAMES = {0: "FIRA_OK", 1: "FIRA_ERR_INVALID_ARG", 2: "FIRA_ERR_WORKSPACE_TOO_SMALL",
                 3: "FIRA_ERR_UNSUPPORTED", 4: "FIRA_ERR_CUDA", 5: "FIRA_ERR_DEVICE_TIMEOUT",
@@ -60,6 +61,8 @@ SIGNATURES = {
     "fira_staging_bytes": (C.c_size_t, [C.c_void_p]),
     "fira_refresh_projection": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_int32),
                                           C.c_int32, C.c_uint64, C.c_int32]),
+    "fira_refresh_projection_f32": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_int32),
+                                              C.c_int32, C.c_uint64, C.c_int32, C.POINTER(C.c_void_p)]),
     "fira_set_projection": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "fira_get_projection": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "fira_get_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_float),
@@ -68,6 +71,7 @@ SIGNATURES = {
     "fira_state_elements": (C.c_int64, [C.c_void_p, C.c_int32]),
     "fira_get_diagnostics": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(Diag)]),
     "fira_poll": (C.c_int, [C.c_void_p]),
+    "fira_selftest_bounded_wait": (C.c_int, [C.c_void_p, C.c_int32]),
     "fira_last_step_launches": (C.c_int32, [C.c_void_p]),
     "fira_enable_phase_timing": (C.c_int, [C.c_void_p, C.c_int32]),
     "fira_get_phase_times": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_float),
@@ -77,6 +81,7 @@ SIGNATURES = {
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_float, C.c_void_p]),
     "fira_noalloc_max_scratch_bytes": (C.c_size_t, []),
+    "fira_noalloc_poll": (C.c_int, [C.c_void_p]),
     "fira_adam_dense": (C.c_int, [C.POINTER(Hparams), C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
                                   C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int,
                                   C.c_int64, C.c_float, C.c_void_p]),
@@ -147,8 +152,10 @@ class Fira:
     or torch.bfloat16 (storage of W, G and the projection).  The state and scratch
     buffers are torch byte tensors owned by this object."""
 
+    GUARD_BYTE = 0xA5
+
     def __init__(self, shapes: Sequence[Tuple[int, int]], r, dtype: torch.dtype, hp: Hparams,
-                 device="cuda", lds: Optional[Sequence[int]] = None):
+                 device="cuda", lds: Optional[Sequence[int]] = None, guard_bytes: int = 0):
         self.L = lib()
         self.device = torch.device(device)
         if self.device.type != "cuda":
@@ -166,15 +173,30 @@ class Fira:
         check(self.L.fira_query_workspace(C.byref(hp), self.descs, self.count, C.byref(sb), C.byref(wb)))
         self.state_bytes, self.scratch_bytes = sb.value, wb.value
         self.ctx = None
+        # guard_bytes > 0 (a multiple of 256): both buffers get that many bytes of a fixed pattern on
+        # either side, which guards_intact() checks: nothing the library launches may write there
+        assert guard_bytes % 256 == 0
+        self.guard_bytes = guard_bytes
         with torch.cuda.device(self.device):
-            self.state = torch.empty(sb.value, dtype=torch.uint8, device=self.device)
-            self.scratch = torch.empty(wb.value, dtype=torch.uint8, device=self.device)
+            self.state = torch.full((sb.value + 2 * guard_bytes,), self.GUARD_BYTE, dtype=torch.uint8,
+                                    device=self.device)
+            self.scratch = torch.full((wb.value + 2 * guard_bytes,), self.GUARD_BYTE, dtype=torch.uint8,
+                                      device=self.device)
             self.stream = torch.cuda.current_stream(self.device)
             ctx = C.c_void_p()
             check(self.L.fira_init(C.byref(ctx), C.byref(hp), self.descs, self.count,
-                                   self.state.data_ptr(), sb.value, self.scratch.data_ptr(), wb.value,
+                                   self.state.data_ptr() + guard_bytes, sb.value,
+                                   self.scratch.data_ptr() + guard_bytes, wb.value,
                                    self.stream.cuda_stream))
         self.ctx = ctx
+
+    def guards_intact(self) -> bool:
+        g = self.guard_bytes
+        if g == 0:
+            return True
+        torch.cuda.synchronize(self.device)
+        return all(bool((buf[:g] == self.GUARD_BYTE).all()) and bool((buf[-g:] == self.GUARD_BYTE).all())
+                   for buf in (self.state, self.scratch))
 
     def close(self):
         if getattr(self, "ctx", None):
@@ -203,12 +225,19 @@ class Fira:
                                     -1.0 if lr is None else lr, staging.data_ptr(), staging.numel()))
 
     def refresh_projection(self, Gs: Sequence[Optional[torch.Tensor]],
-                           which: Optional[Sequence[int]] = None, seed: int = 0, iters: int = -1):
-        if which is None:
-            check(self.L.fira_refresh_projection(self.ctx, ptr_array(Gs), None, 0, seed, iters))
+                           which: Optional[Sequence[int]] = None, seed: int = 0, iters: int = -1,
+                           basis_f32: Optional[Sequence[Optional[torch.Tensor]]] = None):
+        """basis_f32: optional list (one entry per matrix, None to skip) of (d, r) float32 device
+        tensors that receive the basis before it is rounded to the storage type."""
+        w, nw = (None, 0) if which is None else ((C.c_int32 * len(which))(*which), len(which))
+        if basis_f32 is None:
+            check(self.L.fira_refresh_projection(self.ctx, ptr_array(Gs), w, nw, seed, iters))
         else:
-            w = (C.c_int32 * len(which))(*which)
-            check(self.L.fira_refresh_projection(self.ctx, ptr_array(Gs), w, len(which), seed, iters))
+            for i, b in enumerate(basis_f32):
+                assert b is None or (b.dtype == torch.float32 and b.is_contiguous() and
+                                     b.shape == (self._dl(i)[0], self.ranks[i]))
+            check(self.L.fira_refresh_projection_f32(self.ctx, ptr_array(Gs), w, nw, seed, iters,
+                                                     ptr_array(basis_f32)))
 
     def set_projection(self, idx: int, P: torch.Tensor):
         d, _ = self._dl(idx)
@@ -250,6 +279,9 @@ class Fira:
 
     def poll(self) -> int:
         return self.L.fira_poll(self.ctx)
+
+    def selftest_bounded_wait(self, rounds: int = 1000):
+        check(self.L.fira_selftest_bounded_wait(self.ctx, rounds))
 
     def last_step_launches(self) -> int:
         return self.L.fira_last_step_launches(self.ctx)

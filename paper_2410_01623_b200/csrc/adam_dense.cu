@@ -120,6 +120,13 @@ extern "C" fira_status fira_adam_dense(const fira_hparams* hp, int32_t count, vo
     }
     if ((numel[i] + AD_BLOCK_ELEMS - 1) / AD_BLOCK_ELEMS > (1ll << 30)) { set_error("tensor too large"); return FIRA_ERR_INVALID_ARG; }
   }
+  // every chunk's block count is checked before the first launch: an error leaves all tensors untouched
+  for (int first = 0; first < count; first += AD_TENSORS) {
+    long long blocks = 0;
+    for (int q = 0; q < std::min(AD_TENSORS, count - first); ++q)
+      blocks += (numel[first + q] + AD_BLOCK_ELEMS - 1) / AD_BLOCK_ELEMS;
+    if (blocks > 0x7fffffffll) { set_error("fira_adam_dense: too many elements in one call"); return FIRA_ERR_INVALID_ARG; }
+  }
   const double s = (double)(t + 1);
   const float bias = (float)(sqrt(1.0 - pow((double)hp->beta2, s)) / (1.0 - pow((double)hp->beta1, s)));
   const float step = (lr < 0.f ? hp->lr : lr) * bias;
@@ -133,7 +140,6 @@ extern "C" fira_status fira_adam_dense(const fira_hparams* hp, int32_t count, vo
       ch.numel[q] = numel[first + q];
       ch.block_start[q] = (int)blocks;
       blocks += (numel[first + q] + AD_BLOCK_ELEMS - 1) / AD_BLOCK_ELEMS;
-      if (blocks > 0x7fffffffll) { set_error("fira_adam_dense: too many elements in one call"); return FIRA_ERR_INVALID_ARG; }
     }
     ch.block_start[ch.count] = (int)blocks;
     if (dtype == FIRA_BF16)

@@ -65,6 +65,7 @@ enum HyperMode : unsigned {
   HYPER_NO_RESIDUAL = 4u,      // no residual term (Eq. 6)
   HYPER_PSI_RMSPROP = 8u,      // base optimizer: RMSProp instead of Adam
   HYPER_PSI_ADAGRAD = 16u,     // base optimizer: Adagrad instead of Adam
+  HYPER_ONLY_SCALING = 32u,    // Fira-only-scaling: W <- W - lr phi(R) G (no P N term, S = G diag k)
 };
 
 enum DeviceStatusBits : unsigned {

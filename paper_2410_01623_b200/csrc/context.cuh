@@ -57,6 +57,6 @@ size_t refresh_bytes_per_matrix(const fira_matrix_desc& d);
 int engine_for(const fira_hparams& hp, const fira_matrix_desc& d);
 
 fira_status refresh_impl(fira_ctx* ctx, const void* const* G_dev, const std::vector<int>& which,
-                         uint64_t seed, int iters);
+                         uint64_t seed, int iters, float* const* basis_out = nullptr);
 
 }  // namespace fira

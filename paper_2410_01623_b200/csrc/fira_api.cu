@@ -40,6 +40,9 @@ fira_status validate(const fira_hparams* hp, const fira_matrix_desc* descs, int3
   if ((hp->flags & FIRA_FLAG_PSI_RMSPROP) && (hp->flags & FIRA_FLAG_PSI_ADAGRAD)) {
     set_error("FIRA_FLAG_PSI_RMSPROP and FIRA_FLAG_PSI_ADAGRAD exclude each other"); return FIRA_ERR_INVALID_ARG;
   }
+  if ((hp->flags & FIRA_FLAG_ONLY_SCALING) && (hp->flags & FIRA_FLAG_NO_RESIDUAL)) {
+    set_error("FIRA_FLAG_ONLY_SCALING and FIRA_FLAG_NO_RESIDUAL exclude each other"); return FIRA_ERR_INVALID_ARG;
+  }
   for (int i = 0; i < count; ++i) {
     const fira_matrix_desc& d = descs[i];
     if (d.m <= 0 || d.n <= 0 || d.r <= 0 || d.r > std::min(d.m, d.n)) {
@@ -134,6 +137,7 @@ static Hyper make_hyper(const fira_hparams& hp, float lr) {
   if (hp.flags & FIRA_FLAG_NO_RESIDUAL) { h.mode |= HYPER_NO_RESIDUAL; h.a_res = 0.f; }
   if (hp.flags & FIRA_FLAG_PSI_RMSPROP) h.mode |= HYPER_PSI_RMSPROP;
   if (hp.flags & FIRA_FLAG_PSI_ADAGRAD) h.mode |= HYPER_PSI_ADAGRAD;
+  if (hp.flags & FIRA_FLAG_ONLY_SCALING) h.mode |= HYPER_ONLY_SCALING;
   h.gamma = hp.gamma;
   return h;
 }
@@ -357,6 +361,11 @@ fira_status fira_step_host(fira_ctx* c, void* const* W_host, const void* const* 
 
 fira_status fira_refresh_projection(fira_ctx* c, const void* const* G_dev, const int32_t* which, int32_t nwhich,
                                     uint64_t seed, int32_t iters) {
+  return fira_refresh_projection_f32(c, G_dev, which, nwhich, seed, iters, nullptr);
+}
+
+fira_status fira_refresh_projection_f32(fira_ctx* c, const void* const* G_dev, const int32_t* which, int32_t nwhich,
+                                        uint64_t seed, int32_t iters, float* const* basis_f32_dev) {
   if (!c || !G_dev) { set_error("null argument"); return FIRA_ERR_INVALID_ARG; }
   const int count = (int)c->mats.size();
   std::vector<int> sel;
@@ -372,7 +381,10 @@ fira_status fira_refresh_projection(fira_ctx* c, const void* const* G_dev, const
     if (!G_dev[i] || ((uintptr_t)G_dev[i] & 15)) { set_error("G must be non-null and 16-byte aligned"); return FIRA_ERR_INVALID_ARG; }
   }
   if (sel.empty()) return FIRA_OK;
-  return refresh_impl(c, G_dev, sel, seed, iters);
+  if (basis_f32_dev)
+    for (int i : sel)
+      if (basis_f32_dev[i] && ((uintptr_t)basis_f32_dev[i] & 15)) { set_error("basis output must be 16-byte aligned"); return FIRA_ERR_INVALID_ARG; }
+  return refresh_impl(c, G_dev, sel, seed, iters, basis_f32_dev);
 }
 
 static fira_status check_idx(const fira_ctx* c, int32_t idx) {
@@ -460,6 +472,12 @@ fira_status fira_poll(fira_ctx* c) {
   if (st & DEV_STATUS_TIMEOUT) { set_error("a bounded device-side wait ran out"); return FIRA_ERR_DEVICE_TIMEOUT; }
   if (st & DEV_STATUS_NONFINITE) { set_error("a non-finite norm or factor was produced"); return FIRA_ERR_NONFINITE; }
   return FIRA_OK;
+}
+
+fira_status fira_selftest_bounded_wait(fira_ctx* c, int32_t rounds) {
+  if (!c) { set_error("null context"); return FIRA_ERR_INVALID_ARG; }
+  if (rounds < 1 || rounds > (1 << 20)) { set_error("rounds must lie in [1, 2^20]"); return FIRA_ERR_INVALID_ARG; }
+  return tc_selftest_bounded_wait(c, rounds);
 }
 
 int32_t fira_last_step_launches(const fira_ctx* c) { return c ? c->last_launches : -1; }

@@ -12,11 +12,17 @@
 // The paper calls a library SVD here; the iteration converges to the same subspace
 // at the rate (sigma_{r+1}/sigma_r)^2 per round.
 //
-// The two big products run on the CUDA cores in fp32, except for bf16 matrices of
-// tensor-core size with TMA-readable rows: there G is exact in bf16 already, the
-// iterate is rounded to bf16 and the products run on the projection kernel of the
-// step (fp32 accumulation); the basis is stored in bf16 anyway.  Gram products,
-// Cholesky and the triangular solves stay in fp32.
+// Everything runs on the CUDA cores in fp32, except for bf16 matrices of tensor-core size with
+// TMA-readable rows.  For those every product of the iteration is a job of the step's projection
+// kernel in its plain-output mode (fp32 accumulation in tensor memory):
+//   * A Z and A^T Y: G is exact in bf16; the iterate is rounded to bf16, and in the last round it is
+//     split into a bf16 high part and a bf16 remainder (two k-segments), so that the basis that is
+//     kept carries no bf16 rounding of the iterate;
+//   * the Gram product Y^T Y and the application of the inverse factor Y <- Y L^-T: both operands
+//     are fp32 matrices split into two bf16 parts, three k-segments (hi hi + hi lo + lo hi), which is
+//     good to about 2^-16: enough for CholeskyQR, whose second pass removes what the first left;
+//   * L^-T itself comes from the triangular-solve kernel applied to the identity (r x r, fp32).
+// Only the Cholesky factorisation and that small solve stay on the CUDA cores.
 //
 // Random numbers: Philox4x32-10 (Salmon et al., "Parallel random numbers: as easy
 // as 1, 2, 3", SC'11), keyed by the caller's seed, turned into normals by the
@@ -37,9 +43,15 @@ struct RefreshMat {
   float* Y;   // d x r
   float* Z;   // l x r
   float* C;   // r x r
-  __nv_bfloat16* Yb;   // bf16 copies of Y and Z: operands of the tensor-core products (tc only)
+  float* U;            // r x r: L^-T (tc only)
+  __nv_bfloat16* Yb;   // bf16 high parts of Y, Z, U: operands of the tensor-core products (tc only)
   __nv_bfloat16* Zb;
-  int tc;              // the products A Z and A^T Y of this matrix run on the tensor cores
+  __nv_bfloat16* Ub;
+  __nv_bfloat16* Yl;   // bf16 remainders: X - bf16(X)
+  __nv_bfloat16* Zl;
+  __nv_bfloat16* Ul;
+  float* out32;        // optional copy of the kept basis in fp32, before it is rounded for storage
+  int tc;              // every product of this matrix runs on the tensor cores
   long long ld;
   int d, l, r;
   int left, bf16;
@@ -289,45 +301,88 @@ k_store_projection(const RefreshMat* __restrict__ rm) {
        i += (long long)gridDim.x * blockDim.x) {
     if (m.bf16) ((__nv_bfloat16*)m.P)[i] = __float2bfloat16_rn(m.Y[i]);
     else ((float*)m.P)[i] = m.Y[i];
+    if (m.out32) m.out32[i] = m.Y[i];
   }
 }
 
-// bf16 copy of the iterate that the next tensor-core product reads (which = 0: Y, 1: Z).
+// bf16 operands of the next tensor-core product: hi = bf16(x) and, if asked for, lo = bf16(x - hi)
+// (which = 0: Y, 1: Z, 2: U).
 __global__ void __launch_bounds__(256)
-k_iterate_to_bf16(const RefreshMat* __restrict__ rm, int which) {
+k_split_bf16(const RefreshMat* __restrict__ rm, int which, int with_lo) {
   const RefreshMat m = rm[blockIdx.y];
   if (!m.tc) return;
-  const float* src = which ? m.Z : m.Y;
-  __nv_bfloat16* dst = which ? m.Zb : m.Yb;
-  const long long quads = (long long)(which ? m.l : m.d) * m.r / 4;      // r is a multiple of 128
+  const float* src = which == 0 ? m.Y : which == 1 ? m.Z : m.U;
+  __nv_bfloat16* hi = which == 0 ? m.Yb : which == 1 ? m.Zb : m.Ub;
+  __nv_bfloat16* lo = which == 0 ? m.Yl : which == 1 ? m.Zl : m.Ul;
+  const long long rows = which == 0 ? m.d : which == 1 ? m.l : m.r;
+  const long long quads = rows * m.r / 4;      // r is a multiple of 128
   for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < quads;
        q += (long long)gridDim.x * blockDim.x) {
     const float4 v = reinterpret_cast<const float4*>(src)[q];
-    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    const __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
     uint2 u;
-    u.x = *reinterpret_cast<unsigned*>(&a); u.y = *reinterpret_cast<unsigned*>(&b);
-    reinterpret_cast<uint2*>(dst)[q] = u;
+    u.x = *reinterpret_cast<const unsigned*>(&a); u.y = *reinterpret_cast<const unsigned*>(&b);
+    reinterpret_cast<uint2*>(hi)[q] = u;
+    if (with_lo) {
+      const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+      const __nv_bfloat162 c = __floats2bfloat162_rn(v.x - fa.x, v.y - fa.y), e = __floats2bfloat162_rn(v.z - fb.x, v.w - fb.y);
+      uint2 w;
+      w.x = *reinterpret_cast<const unsigned*>(&c); w.y = *reinterpret_cast<const unsigned*>(&e);
+      reinterpret_cast<uint2*>(lo)[q] = w;
+    }
   }
+}
+
+// U <- identity (r x r); the triangular-solve kernel then turns it into L^-T.
+__global__ void __launch_bounds__(256)
+k_identity(const RefreshMat* __restrict__ rm) {
+  const RefreshMat m = rm[blockIdx.y];
+  if (!m.tc) return;
+  const long long total = (long long)m.r * m.r;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x)
+    m.U[i] = (i / m.r == i % m.r) ? 1.f : 0.f;
 }
 
 // descriptor tables of a chunk: per-matrix entries plus alignment slack
 constexpr size_t TABLE_PER_MATRIX = 1024;
 constexpr size_t TABLE_SLACK = 16 * 1024;
-static_assert(sizeof(RefreshMat) + 4 * sizeof(GemmDesc) + 2 * sizeof(TrsmDesc) + 8 * sizeof(int) <= TABLE_PER_MATRIX, "table allowance");
+static_assert(sizeof(RefreshMat) + 4 * sizeof(GemmDesc) + 3 * sizeof(TrsmDesc) + 10 * sizeof(int) <= TABLE_PER_MATRIX, "table allowance");
 
 }  // namespace
 
-// bf16 matrices that TMA can read in place: their big products run on the tensor cores
+// bf16 matrices that TMA can read in place: their products run on the tensor cores
 static bool refresh_on_tc(const fira_matrix_desc& d) {
   return d.dtype == FIRA_BF16 && tc_supported(d) && tc_staging_pitch(d) == 0;
 }
 
-static TcGemmJob refresh_job(const fira_matrix_desc& d, bool az) {
+// The eight kinds of tensor-core jobs of one matrix: A Z and A^T Y (plain and with a split iterate),
+// the two Gram products, the two applications of L^-T.
+enum { JOB_AZ = 0, JOB_AZ_SPLIT, JOB_ATY, JOB_ATY_SPLIT, JOB_GRAM_Y, JOB_GRAM_Z, JOB_APPLY_Y, JOB_APPLY_Z, JOB_KINDS };
+
+static TcGemmJob refresh_job(const fira_matrix_desc& dsc, int kind) {
   TcGemmJob j;
   memset(&j, 0, sizeof(j));
-  j.m = d.m; j.n = d.n; j.ld = d.ld ? d.ld : d.n; j.r = d.r;
-  const bool left = d.m <= d.n;
-  j.mn_major = az ? !left : left;      // A Z: rows d, k = l;  A^T Y: rows l, k = d
+  const int d = std::min(dsc.m, dsc.n), l = std::max(dsc.m, dsc.n);
+  const bool left = dsc.m <= dsc.n;
+  j.r = dsc.r;
+  switch (kind) {
+    case JOB_AZ: case JOB_AZ_SPLIT: case JOB_ATY: case JOB_ATY_SPLIT: {
+      const bool az = kind == JOB_AZ || kind == JOB_AZ_SPLIT;
+      j.m = dsc.m; j.n = dsc.n; j.ld = dsc.ld ? dsc.ld : dsc.n;
+      j.mn_major = az ? !left : left;      // A Z: rows d, k = l;  A^T Y: rows l, k = d
+      if (kind == JOB_AZ_SPLIT || kind == JOB_ATY_SPLIT) { j.nseg = 2; j.asel = 0u; j.bsel = 2u; }   // A hi, A lo(iterate)
+      break;
+    }
+    case JOB_GRAM_Y: case JOB_GRAM_Z:      // C[i][j] = sum_k X[k][i] X[k][j]: "G" = X as [k][i]
+      j.m = kind == JOB_GRAM_Y ? d : l; j.n = dsc.r; j.ld = dsc.r; j.mn_major = 1;
+      j.nseg = 3; j.asel = 4u; j.bsel = 2u;   // hi hi, hi lo, lo hi
+      break;
+    default:                               // X[i][j] = sum_k X[i][k] U[k][j]: "G" = X as [i][k]
+      j.m = kind == JOB_APPLY_Y ? d : l; j.n = dsc.r; j.ld = dsc.r; j.mn_major = 0;
+      j.nseg = 3; j.asel = 4u; j.bsel = 2u;
+      break;
+  }
   return j;
 }
 
@@ -335,8 +390,8 @@ static size_t refresh_data_bytes(const fira_matrix_desc& d) {
   const size_t dd = std::min(d.m, d.n), ll = std::max(d.m, d.n), r = d.r;
   size_t b = align_up(dd * r * 4) + align_up(ll * r * 4) + align_up(r * r * 4);
   if (refresh_on_tc(d)) {
-    const TcGemmJob a = refresh_job(d, true), t = refresh_job(d, false);
-    b += align_up(dd * r * 2) + align_up(ll * r * 2) + tc_gemm_table_bytes(&a, 1) + tc_gemm_table_bytes(&t, 1);
+    b += align_up(r * r * 4) + 2 * (align_up(dd * r * 2) + align_up(ll * r * 2) + align_up(r * r * 2));
+    for (int k = 0; k < JOB_KINDS; ++k) { const TcGemmJob j = refresh_job(d, k); b += tc_gemm_table_bytes(&j, 1); }
   }
   return b;
 }
@@ -356,8 +411,10 @@ size_t refresh_bytes_per_matrix(const fira_matrix_desc& d) {
 
 // Refreshes the matrices of `which` in chunks that fit the work area.  The work
 // area is shared with the step's scratch, whose contents are dead between steps.
+// basis_out (may be null): per matrix index an optional device pointer that receives the kept
+// basis in fp32 (d x r) before it is rounded to the storage type.
 fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vector<int>& which,
-                         uint64_t seed, int iters) {
+                         uint64_t seed, int iters, float* const* basis_out) {
   if (iters < 0) iters = 4;
   cudaStream_t st = c->stream;
   size_t pos = 0;
@@ -379,47 +436,65 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
       const int idx = which[pos + a];
       const MatDev& mt = c->mats[idx];
       RefreshMat rm;
+      memset(&rm, 0, sizeof(rm));
       rm.G = G_dev[idx]; rm.P = mt.P;
+      rm.out32 = basis_out ? basis_out[idx] : nullptr;
       char* base = c->work_base + offs[a];
-      rm.Y = (float*)base; base += align_up((size_t)mt.d * mt.r * 4);
-      rm.Z = (float*)base; base += align_up((size_t)mt.l * mt.r * 4);
-      rm.C = (float*)base; base += align_up((size_t)mt.r * mt.r * 4);
+      const size_t r = mt.r;
+      rm.Y = (float*)base; base += align_up((size_t)mt.d * r * 4);
+      rm.Z = (float*)base; base += align_up((size_t)mt.l * r * 4);
+      rm.C = (float*)base; base += align_up(r * r * 4);
       rm.tc = refresh_on_tc(c->descs[idx]) ? 1 : 0;
-      rm.Yb = rm.Zb = nullptr;
       if (rm.tc) {
-        rm.Yb = (__nv_bfloat16*)base; base += align_up((size_t)mt.d * mt.r * 2);
-        rm.Zb = (__nv_bfloat16*)base; base += align_up((size_t)mt.l * mt.r * 2);
+        rm.U = (float*)base; base += align_up(r * r * 4);
+        rm.Yb = (__nv_bfloat16*)base; base += align_up((size_t)mt.d * r * 2);
+        rm.Yl = (__nv_bfloat16*)base; base += align_up((size_t)mt.d * r * 2);
+        rm.Zb = (__nv_bfloat16*)base; base += align_up((size_t)mt.l * r * 2);
+        rm.Zl = (__nv_bfloat16*)base; base += align_up((size_t)mt.l * r * 2);
+        rm.Ub = (__nv_bfloat16*)base; base += align_up(r * r * 2);
+        rm.Ul = (__nv_bfloat16*)base; base += align_up(r * r * 2);
       }
       data_end = std::max(data_end, (size_t)(base - c->work_base));
       rm.ld = mt.ld; rm.d = mt.d; rm.l = mt.l; rm.r = mt.r; rm.left = mt.left; rm.bf16 = mt.bf16;
       rm.key = seed * 0x9E3779B97F4A7C15ull + (unsigned long long)idx * 0xD1B54A32D192ED03ull + 1ull;
       rms.push_back(rm);
     }
-    // ---- descriptor tables: AZ->Y, A^T Y->Z, Y^T Y->C, Z^T Z->C, trsm(Y), trsm(Z)
+    // ---- descriptor tables of the CUDA-core kernels: AZ->Y, A^T Y->Z, Y^T Y->C, Z^T Z->C, trsm(Y), trsm(Z)
+    // for the matrices that stay there; trsm(U) for the others
     std::vector<GemmDesc> gAZ, gAtY, gYY, gZZ;
-    std::vector<TrsmDesc> tY, tZ;
-    std::vector<int> sAZ{0}, sAtY{0}, sYY{0}, sTY{0}, sTZ{0};
+    std::vector<TrsmDesc> tY, tZ, tU;
+    std::vector<int> sAZ{0}, sAtY{0}, sYY{0}, sTY{0}, sTZ{0}, sTU{0};
     auto tiles = [](int I, int J) { return simt_tiles(I) * simt_tiles(J); };
-    std::vector<TcGemmJob> jAZ, jAtY;
+    std::vector<TcGemmJob> jobs[JOB_KINDS];
     for (size_t a = 0; a < rms.size(); ++a) {
       const RefreshMat& m = rms[a];
+      if (m.tc) {
+        const fira_matrix_desc& dd = c->descs[which[pos + a]];
+        for (int k = 0; k < JOB_KINDS; ++k) {
+          TcGemmJob j = refresh_job(dd, k);
+          switch (k) {
+            case JOB_AZ: case JOB_AZ_SPLIT: j.G = m.G; j.B = m.Zb; j.B_lo = k == JOB_AZ_SPLIT ? m.Zl : nullptr; j.C = m.Y; break;
+            case JOB_ATY: case JOB_ATY_SPLIT: j.G = m.G; j.B = m.Yb; j.B_lo = k == JOB_ATY_SPLIT ? m.Yl : nullptr; j.C = m.Z; break;
+            case JOB_GRAM_Y: j.G = m.Yb; j.G_lo = m.Yl; j.B = m.Yb; j.B_lo = m.Yl; j.C = m.C; break;
+            case JOB_GRAM_Z: j.G = m.Zb; j.G_lo = m.Zl; j.B = m.Zb; j.B_lo = m.Zl; j.C = m.C; break;
+            case JOB_APPLY_Y: j.G = m.Yb; j.G_lo = m.Yl; j.B = m.Ub; j.B_lo = m.Ul; j.C = m.Y; break;
+            default: j.G = m.Zb; j.G_lo = m.Zl; j.B = m.Ub; j.B_lo = m.Ul; j.C = m.Z; break;
+          }
+          jobs[k].push_back(j);
+        }
+        tU.push_back(TrsmDesc{m.U, m.C, m.r, m.r}); sTU.push_back(sTU.back() + (m.r + TM - 1) / TM);
+        continue;
+      }
       GemmDesc g;
       // Y[d][j] = sum_l A(d,l) Z[l][j]
       g.A = m.G; g.a_bf16 = m.bf16;
       g.sAi = m.left ? m.ld : 1; g.sAk = m.left ? 1 : m.ld;
       g.B = m.Z; g.sBk = m.r; g.sBj = 1; g.C = m.Y; g.sCi = m.r; g.I = m.d; g.J = m.r; g.K = m.l;
-      if (!m.tc) { gAZ.push_back(g); sAZ.push_back(sAZ.back() + tiles(g.I, g.J)); }
+      gAZ.push_back(g); sAZ.push_back(sAZ.back() + tiles(g.I, g.J));
       // Z[l][j] = sum_d A(d,l) Y[d][j]
       g.sAi = m.left ? 1 : m.ld; g.sAk = m.left ? m.ld : 1;
       g.B = m.Y; g.C = m.Z; g.I = m.l; g.K = m.d;
-      if (!m.tc) { gAtY.push_back(g); sAtY.push_back(sAtY.back() + tiles(g.I, g.J)); }
-      if (m.tc) {
-        const fira_matrix_desc& dd = c->descs[which[pos + a]];
-        TcGemmJob j = refresh_job(dd, true);
-        j.G = m.G; j.B = m.Zb; j.C = m.Y; jAZ.push_back(j);
-        j = refresh_job(dd, false);
-        j.G = m.G; j.B = m.Yb; j.C = m.Z; jAtY.push_back(j);
-      }
+      gAtY.push_back(g); sAtY.push_back(sAtY.back() + tiles(g.I, g.J));
       // C = Y^T Y and C = Z^T Z
       g.a_bf16 = 0; g.sAi = 1; g.sAk = m.r; g.sBk = m.r; g.sBj = 1; g.C = m.C; g.sCi = m.r; g.I = m.r; g.J = m.r;
       g.A = m.Y; g.B = m.Y; g.K = m.d; gYY.push_back(g);
@@ -432,6 +507,7 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     cudaError_t cerr = cudaSuccess;
     auto put = [&](const void* src, size_t bytes) -> char* {
       char* dst = tp;
+      if (bytes == 0) return dst;
       if ((size_t)(tp + align_up(bytes) - c->work_base) > c->work_bytes) { cerr = cudaErrorInvalidValue; return dst; }
       cudaError_t e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st);
       if (e != cudaSuccess) cerr = e;
@@ -445,61 +521,82 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     const GemmDesc* dZZ = (const GemmDesc*)put(gZZ.data(), gZZ.size() * sizeof(GemmDesc));
     const TrsmDesc* dTY = (const TrsmDesc*)put(tY.data(), tY.size() * sizeof(TrsmDesc));
     const TrsmDesc* dTZ = (const TrsmDesc*)put(tZ.data(), tZ.size() * sizeof(TrsmDesc));
+    const TrsmDesc* dTU = (const TrsmDesc*)put(tU.data(), tU.size() * sizeof(TrsmDesc));
     const int* dsAZ = (const int*)put(sAZ.data(), sAZ.size() * sizeof(int));
     const int* dsAtY = (const int*)put(sAtY.data(), sAtY.size() * sizeof(int));
     const int* dsYY = (const int*)put(sYY.data(), sYY.size() * sizeof(int));
     const int* dsTY = (const int*)put(sTY.data(), sTY.size() * sizeof(int));
     const int* dsTZ = (const int*)put(sTZ.data(), sTZ.size() * sizeof(int));
+    const int* dsTU = (const int*)put(sTU.data(), sTU.size() * sizeof(int));
     if (cerr != cudaSuccess) { set_error(std::string("refresh tables: ") + cudaGetErrorString(cerr)); return FIRA_ERR_CUDA; }
-    // tables of the tensor-core products (tensor maps and tile records), after the others
-    const int ntc = (int)jAZ.size(), nsimt = nm - ntc;
-    char* tabAZ = nullptr; char* tabAtY = nullptr;
-    int tilesAZ = 0, tilesAtY = 0;
+    // tables of the tensor-core jobs (tensor maps and tile records), after the others
+    const int ntc = (int)jobs[0].size(), nsimt = nm - ntc;
+    char* tab[JOB_KINDS] = {};
+    int jtiles[JOB_KINDS] = {};
     if (ntc) {
-      const size_t bAZ = tc_gemm_table_bytes(jAZ.data(), ntc), bAtY = tc_gemm_table_bytes(jAtY.data(), ntc);
-      tabAZ = tp; tabAtY = tp + bAZ;
-      if ((size_t)(tabAtY + bAtY - c->work_base) > c->work_bytes) {
-        set_error("scratch buffer too small for the projection refresh"); return FIRA_ERR_WORKSPACE_TOO_SMALL;
+      for (int k = 0; k < JOB_KINDS; ++k) {
+        const size_t bytes = tc_gemm_table_bytes(jobs[k].data(), ntc);
+        if ((size_t)(tp + bytes - c->work_base) > c->work_bytes) {
+          set_error("scratch buffer too small for the projection refresh"); return FIRA_ERR_WORKSPACE_TOO_SMALL;
+        }
+        tab[k] = tp;
+        const fira_status ps = tc_gemm_prepare(c, jobs[k].data(), ntc, tab[k], bytes, &jtiles[k]);
+        if (ps != FIRA_OK) return ps;
+        tp += bytes;
       }
-      fira_status ps = tc_gemm_prepare(c, jAZ.data(), ntc, tabAZ, bAZ, &tilesAZ);
-      if (ps == FIRA_OK) ps = tc_gemm_prepare(c, jAtY.data(), ntc, tabAtY, bAtY, &tilesAtY);
-      if (ps != FIRA_OK) return ps;
     }
-    // A Z -> Y and A^T Y -> Z: CUDA-core products for some matrices, tensor-core products (bf16 copy
-    // of the iterate as the second operand, fp32 accumulation) for the others
-    auto product = [&](bool az) -> fira_status {
+    const dim3 ew_grid(296, nm);      // element-wise helpers: every matrix of the chunk, tc ones act
+    // A Z -> Y and A^T Y -> Z.  precise: the iterate enters with its bf16 remainder as a second k-segment.
+    auto product = [&](bool az, bool precise) -> fira_status {
       if (nsimt) {
         if (az) k_rgemm<<<sAZ.back(), GEMM_THREADS, 0, st>>>(dAZ, nsimt, dsAZ);
         else k_rgemm<<<sAtY.back(), GEMM_THREADS, 0, st>>>(dAtY, nsimt, dsAtY);
       }
       if (ntc) {
-        k_iterate_to_bf16<<<dim3(296, nm), 256, 0, st>>>(rm_dev, az ? 1 : 0);
-        return az ? tc_gemm_run(c, tabAZ, ntc, tilesAZ) : tc_gemm_run(c, tabAtY, ntc, tilesAtY);
+        k_split_bf16<<<ew_grid, 256, 0, st>>>(rm_dev, az ? 1 : 0, precise ? 1 : 0);
+        const int k = az ? (precise ? JOB_AZ_SPLIT : JOB_AZ) : (precise ? JOB_ATY_SPLIT : JOB_ATY);
+        return tc_gemm_run(c, tab[k], ntc, jtiles[k]);
       }
       return FIRA_OK;
     };
-
-    // CholeskyQR; the second pass brings the basis to fp32 orthonormality and is needed only for the
-    // basis that is kept: one pass (deviation about cond^2 * 2^-24) keeps an intermediate iterate
-    // well conditioned, which is all the next product asks of it.
-    auto orth = [&](const GemmDesc* gram, const TrsmDesc* tr, const int* tr_start, int tr_tiles, int passes) {
+    // CholeskyQR of Y (y = true) or Z; the second pass brings the basis to fp32 orthonormality and is
+    // needed only for the basis that is kept: one pass (deviation about cond^2 times the product's
+    // precision) keeps an intermediate iterate well conditioned, which is all the next product asks.
+    auto orth = [&](bool y, int passes) -> fira_status {
       for (int pass = 0; pass < passes; ++pass) {
-        k_rgemm<<<sYY.back(), GEMM_THREADS, 0, st>>>(gram, nm, dsYY);
+        if (nsimt) k_rgemm<<<sYY.back(), GEMM_THREADS, 0, st>>>(y ? dYY : dZZ, nsimt, dsYY);
+        if (ntc) {
+          k_split_bf16<<<ew_grid, 256, 0, st>>>(rm_dev, y ? 0 : 1, 1);
+          const fira_status gs = tc_gemm_run(c, tab[y ? JOB_GRAM_Y : JOB_GRAM_Z], ntc, jtiles[y ? JOB_GRAM_Y : JOB_GRAM_Z]);
+          if (gs != FIRA_OK) return gs;
+        }
         k_cholesky<<<nm * CHOL_CTAS, GEMM_THREADS, 0, st>>>(rm_dev, pass == 0 ? 1e-6f : 0.f, c->status_dev);
-        k_trsm_rows<<<tr_tiles, GEMM_THREADS, 0, st>>>(tr, nm, tr_start);
+        if (nsimt) {
+          if (y) k_trsm_rows<<<sTY.back(), GEMM_THREADS, 0, st>>>(dTY, nsimt, dsTY);
+          else k_trsm_rows<<<sTZ.back(), GEMM_THREADS, 0, st>>>(dTZ, nsimt, dsTZ);
+        }
+        if (ntc) {
+          k_identity<<<ew_grid, 256, 0, st>>>(rm_dev);
+          k_trsm_rows<<<sTU.back(), GEMM_THREADS, 0, st>>>(dTU, ntc, dsTU);      // U = L^-T
+          k_split_bf16<<<ew_grid, 256, 0, st>>>(rm_dev, 2, 1);
+          const fira_status as = tc_gemm_run(c, tab[y ? JOB_APPLY_Y : JOB_APPLY_Z], ntc, jtiles[y ? JOB_APPLY_Y : JOB_APPLY_Z]);
+          if (as != FIRA_OK) return as;
+        }
       }
+      return FIRA_OK;
     };
-    k_gauss<<<dim3(296, nm), 256, 0, st>>>(rm_dev);
-    fira_status prs = product(true);
-    if (prs != FIRA_OK) return prs;
-    orth(dYY, dTY, dsTY, sTY.back(), iters == 0 ? 2 : 1);
-    for (int it = 0; it < iters; ++it) {
-      if ((prs = product(false)) != FIRA_OK) return prs;
-      orth(dZZ, dTZ, dsTZ, sTZ.back(), 1);
-      if ((prs = product(true)) != FIRA_OK) return prs;
-      orth(dYY, dTY, dsTY, sTY.back(), it + 1 == iters ? 2 : 1);
+    k_gauss<<<ew_grid, 256, 0, st>>>(rm_dev);
+    fira_status prs = product(true, iters == 0);
+    if (prs == FIRA_OK) prs = orth(true, iters == 0 ? 2 : 1);
+    for (int it = 0; it < iters && prs == FIRA_OK; ++it) {
+      const bool last = it + 1 == iters;
+      prs = product(false, last);
+      if (prs == FIRA_OK) prs = orth(false, 1);
+      if (prs == FIRA_OK) prs = product(true, last);
+      if (prs == FIRA_OK) prs = orth(true, last ? 2 : 1);
     }
-    k_store_projection<<<dim3(296, nm), 256, 0, st>>>(rm_dev);
+    if (prs != FIRA_OK) return prs;
+    k_store_projection<<<ew_grid, 256, 0, st>>>(rm_dev);
     RF_CUDA(cudaGetLastError());
     // the next chunk reuses the work area, and the host tables above die here
     RF_CUDA(cudaStreamSynchronize(st));

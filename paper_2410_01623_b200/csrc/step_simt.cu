@@ -197,7 +197,63 @@ k_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlis
   for (int j = lane; j < mt.r; j += 32) mt.Xt[base + j] = a_low * mt.Xt[base + j] - c * mt.Rt[base + j];
 }
 
+// ---------------------------------------------------------------- Fira-only-scaling
+// W <- W - lr phi(R) G: no product.  One block per tile x tile block of W; rows are walked by the
+// warps, columns by the lanes (coalesced along the rows of G and W).
+template <typename T, int UPDATE>
+__device__ __forceinline__ float scaled_gradient_tile(const MatDev& mt, int i0, int j0, int tile, float c) {
+  const T* G = static_cast<const T*>(mt.G);
+  T* W = static_cast<T*>(mt.W);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int i1 = min(i0 + tile, mt.m), j1 = min(j0 + tile, mt.n);
+  float ss = 0.f;
+  for (int i = i0 + warp; i < i1; i += 8) {
+    const float krow = mt.left ? 0.f : mt.kvec[i];
+    for (int j = j0 + lane; j < j1; j += 32) {
+      const float kf = mt.left ? mt.kvec[j] : krow;
+      const long long off = (long long)i * mt.ld + j;
+      const float g = to_float<T>(G[off]);
+      if (UPDATE) W[off] = from_float<T>(to_float<T>(W[off]) - c * kf * g);
+      else { const float sv = kf * g; ss = fmaf(sv, sv, ss); }
+    }
+  }
+  return ss;
+}
+
+template <int UPDATE>
+__global__ void __launch_bounds__(256)
+k_scaled_gradient(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
+                  const int* __restrict__ tile_start, int tile, float lr, float a_res) {
+  __shared__ float red[8];
+  const int p = find_matrix(tile_start, nlist, blockIdx.x);
+  const MatDev mt = mats[list[p]];
+  const int t = blockIdx.x - tile_start[p];
+  const int ct = (mt.n + tile - 1) / tile;
+  const int i0 = (t / ct) * tile, j0 = (t % ct) * tile;
+  const float c = UPDATE ? lr * a_res * mt.sc->lambda : 0.f;
+  float ss = mt.bf16 ? scaled_gradient_tile<__nv_bfloat16, UPDATE>(mt, i0, j0, tile, c)
+                     : scaled_gradient_tile<float, UPDATE>(mt, i0, j0, tile, c);
+  if (!UPDATE) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float tot = 0.f;
+      for (int w = 0; w < 8; ++w) tot += red[w];
+      mt.part[t] = tot;
+    }
+  }
+}
+
 }  // namespace
+
+void launch_scaled_gradient(const MatDev* mats, const int* list, int nlist, const int* tile_start, int tiles,
+                            int tile, int update, float lr, float a_res, cudaStream_t st) {
+  if (tiles <= 0) return;
+  if (update) k_scaled_gradient<1><<<tiles, 256, 0, st>>>(mats, list, nlist, tile_start, tile, lr, a_res);
+  else k_scaled_gradient<0><<<tiles, 256, 0, st>>>(mats, list, nlist, tile_start, tile, lr, a_res);
+}
 
 // ---------------------------------------------------------------- phase 4
 __global__ void __launch_bounds__(256)
@@ -280,6 +336,17 @@ int launch_simt_step(const SimtPlan& pl, const Hyper& hp, unsigned* status_dev, 
   const int row_blocks = (pl.rows_total + 7) / 8;
   k_adam_rows<<<row_blocks, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.row_start, pl.rows_total, hp);
   tm->mark(st);
+  if (hp.mode & HYPER_ONLY_SCALING) {
+    // W <- W - lr phi(R) G: the norm of the scaled gradient, the limiter, the element-wise update
+    launch_scaled_gradient(pl.mats, pl.list, pl.nlist, pl.w_tile_start, pl.w_tiles, SIMT_TILE, 0, 0.f, hp.a_res, st);
+    tm->mark(st);
+    k_finalize<<<pl.nlist, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.npart, hp, status_dev);
+    tm->mark(st);
+    tm->mark(st);
+    launch_scaled_gradient(pl.mats, pl.list, pl.nlist, pl.w_tile_start, pl.w_tiles, SIMT_TILE, 1, hp.lr, hp.a_res, st);
+    tm->mark(st);
+    return 5;
+  }
   k_back_project<MODE_NORM><<<pl.w_tiles, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist,
                                                                  pl.w_tile_start, 0.f, hp.a_res);
   tm->mark(st);

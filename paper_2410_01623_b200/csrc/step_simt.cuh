@@ -31,4 +31,11 @@ extern const char* const kSimtPhaseNames[6];
 __global__ void k_finalize(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
                            const int* __restrict__ npart_of, Hyper hp, unsigned* __restrict__ status);
 
+// Fira-only-scaling, element-wise over tiles of `tile` x `tile` elements of W (one block of 256
+// threads per tile; tile_start holds nlist + 1 ascending tile counts; first_block is added to the
+// block index).  update = 0: part[tile] = sum over the tile of (k_l G)^2, the norm that the
+// limiter sees; update = 1: W <- W - lr a_res lambda k_l G.
+void launch_scaled_gradient(const MatDev* mats, const int* list, int nlist, const int* tile_start, int tiles,
+                            int tile, int update, float lr, float a_res, cudaStream_t st);
+
 }  // namespace fira

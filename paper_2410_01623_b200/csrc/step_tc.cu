@@ -181,7 +181,8 @@ k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, i
     if (hp.mode & HYPER_MATRIX_SCALING) { mt.aux[l] = nn; mt.aux[mt.l + l] = rn; k = 1.f; }   // see k_finalize
     if (hp.mode & HYPER_NO_SCALING) k = 1.f;
     mt.kvec[l] = k;
-    contrib = k * k * fmaxf(gs - rn, 0.f);
+    // only-scaling: S = G diag(k), so ||S_l||^2 = k_l^2 ||G_l||^2
+    contrib = k * k * ((hp.mode & HYPER_ONLY_SCALING) ? gs : fmaxf(gs - rn, 0.f));
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xffffffffu, contrib, o);
@@ -219,6 +220,28 @@ k_tc_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int n
     for (int e = 0; e < 8; ++e) x[e] = a_low * nv[e] - c * rv[e];
     *reinterpret_cast<uint4*>(mt.Xb + base + j) = pack8_bf16(x);
   }
+}
+
+// Self-test of the bounded waits: thread 0 waits on a barrier that nothing ever arrives on and gives
+// up after `rounds` tries, raising the abort flag; a thread of the second warp sits in a wait with
+// the ordinary limit, as the other roles of the product kernels do, and must leave when it sees the
+// flag.  No copy is in flight and nothing else is touched.
+__global__ void __launch_bounds__(64)
+k_selftest_bounded_wait(unsigned* __restrict__ status, uint32_t rounds) {
+  __shared__ uint64_t bars[2];
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_u32(&bars[0]), 1);
+    ptx::mbar_init(ptx::smem_u32(&bars[1]), 1);
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  bool got = true;
+  if (threadIdx.x == 0) got = ptx::mbar_wait(ptx::smem_u32(&bars[0]), 0, &abort_flag, rounds);
+  if (threadIdx.x == 32) got = ptx::mbar_wait(ptx::smem_u32(&bars[1]), 0, &abort_flag);
+  __syncthreads();
+  if (threadIdx.x == 0 && !got && abort_flag) atomicOr(status, DEV_STATUS_TIMEOUT);
 }
 
 // ============================================================================ host side
@@ -488,16 +511,29 @@ fira_status tc_gemm_prepare(fira_ctx* c, const TcGemmJob* jobs, int njobs, char*
     const bool chunked = j.mn_major && j.n % 64 == 0;
     TcMaps& mp = maps[q];
     memset(&mp, 0, sizeof(mp));
-    if (chunked) {
-      if (!encode_map_chunked(&mp.g1a, j.G, j.m, j.n, j.ld, 64, 2)) return FIRA_ERR_CUDA;
-    } else if (!encode_map(&mp.g1a, j.G, j.m, j.n, j.ld, 64, j.mn_major ? 64 : 128)) return FIRA_ERR_CUDA;
-    if (!encode_map_chunked(&mp.g1b, j.B, D, j.r, j.r, 64, bn / 128)) return FIRA_ERR_CUDA;
+    for (int part = 0; part < 2; ++part) {      // 0: the operands themselves, 1: their low parts (if any)
+      const void* ga = part ? j.G_lo : j.G;
+      const void* gb = part ? j.B_lo : j.B;
+      CUtensorMap* ma = part ? &mp.g2a : &mp.g1a;
+      CUtensorMap* mb = part ? &mp.g2b : &mp.g1b;
+      if (ga) {
+        if (chunked) {
+          if (!encode_map_chunked(ma, ga, j.m, j.n, j.ld, 64, 2)) return FIRA_ERR_CUDA;
+        } else if (!encode_map(ma, ga, j.m, j.n, j.ld, 64, j.mn_major ? 64 : 128)) return FIRA_ERR_CUDA;
+      }
+      if (gb && !encode_map_chunked(mb, gb, D, j.r, j.r, 64, bn / 128)) return FIRA_ERR_CUDA;
+    }
     if (!encode_map(&mp.em, j.C, L, j.r, j.r, K1_ECOLS, K1_EROWS, 1)) return FIRA_ERR_CUDA;
+    const int nseg = j.nseg > 1 ? j.nseg : 1;
+    const int nkb_seg = (D + BK - 1) / BK;
+    if (nseg > 3 || ((j.asel >> nseg) != 0) || ((j.bsel >> nseg) != 0) || (j.asel && !j.G_lo) || (j.bsel && !j.B_lo)) {
+      set_error("internal: bad k-segments of a refresh product"); return FIRA_ERR_INVALID_ARG;
+    }
     for (int l0 = 0; l0 < L; l0 += 2 * BM)
       for (int r0 = 0; r0 < j.r; r0 += bn) {
         ProjTileDesc d;
-        d.colpart = nullptr; d.slot = q; d.l0 = l0; d.r0 = r0;
-        d.nkb = (D + BK - 1) / BK; d.L = L;
+        d.colpart = reinterpret_cast<float*>(seg_word(nkb_seg, j.asel, j.bsel)); d.slot = q; d.l0 = l0; d.r0 = r0;
+        d.nkb = nseg * nkb_seg; d.L = L;
         d.bn_left = bn | ((j.r / bn) << 16) | (j.mn_major ? (int)0x80000000 : 0) | (chunked ? PROJ_A_CHUNKED : 0);
         tiles.push_back(d);
       }
@@ -529,6 +565,13 @@ fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntile
   Hyper hp{};
   k_tc_project<EPI_PLAIN, PSI_ADAM><<<2 * std::min(ntiles, num_sms / 2), K1_THREADS, K1_SMEM_BYTES, c->stream>>>(
       maps, tiles, ntiles, nullptr, hp, c->status_dev);
+  return FIRA_OK;
+}
+
+fira_status tc_selftest_bounded_wait(fira_ctx* c, int rounds) {
+  k_selftest_bounded_wait<<<1, 64, 0, c->stream>>>(c->status_dev, (uint32_t)rounds);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { set_error(std::string("bounded-wait self-test: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
   return FIRA_OK;
 }
 
@@ -576,6 +619,15 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
   tm->mark(st);
   k_finalize<<<pl->nlist, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->npart, hp, c->status_dev);
   tm->mark(st);
+  if (hp.mode & HYPER_ONLY_SCALING) {
+    // W <- W - lr phi(R) G: no back-projection; the element-wise update works on the caller's W and
+    // G in place (whatever their pitch), so nothing is copied back from the aligned copies
+    tm->mark(st);
+    launch_scaled_gradient(mats, pl->list, pl->nlist, pl->k2_start, pl->k2_tiles, 2 * BM, 1, hp.lr, hp.a_res, st);
+    tm->mark(st);
+    tm->mark(st);
+    return pl->nstage ? 6 : 5;
+  }
   k_tc_form_x<<<(pl->rows_total + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start,
                                                         pl->rows_total, hp.a_low, hp.a_res, pl->fast_dev);
   tm->mark(st);

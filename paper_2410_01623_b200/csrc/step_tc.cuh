@@ -29,6 +29,9 @@ fira_status tc_update_pointers(fira_ctx* c);
 // Enqueues the tensor-core phases for the matrices of the tc list; returns the
 // number of launches (negative: error, message set).
 int launch_tc_step(fira_ctx* c, const Hyper& hp);
+// Launches the self-test kernel of the bounded waits (one block; sets the time-out bit of the
+// context's status word after `rounds` tries on a barrier that nothing arrives on).
+fira_status tc_selftest_bounded_wait(fira_ctx* c, int rounds);
 // Names of this engine's phases in launch order (8).
 int tc_phase_names(const char** out);
 
@@ -36,9 +39,15 @@ int tc_phase_names(const char** out);
 // C[l][j] (fp32, L x r) = sum over k < D of A(k, l) B[k][j], with A taken in place from the bf16
 // matrix G (m x n, pitch ld, rows 16-byte aligned): mn_major = 1: G is [k][l] (D = m, L = n);
 // mn_major = 0: G is [l][k] (L = m, D = n).  B is bf16 [D][r].  r % 128 == 0.
+// Split-precision products: with nseg > 1 the product runs over nseg k-segments that accumulate into
+// the same output; segment s takes A from G (bit s of asel clear) or G_lo (set) and B from B (bsel
+// clear) or B_lo (set).  G_lo / B_lo have the shapes and pitches of G / B.  For an fp32 matrix
+// X = X_hi + X_lo (two bf16 parts), segments (hi,hi), (hi,lo), (lo,hi) give X Y to about 2^-16.
 struct TcGemmJob {
   const void* G; long long ld; int m, n; int mn_major;
   const void* B; float* C; int r;
+  const void* G_lo; const void* B_lo;
+  int nseg; unsigned asel, bsel;
 };
 // Device bytes of the tables (tensor maps, tile records) of a job list.
 size_t tc_gemm_table_bytes(const TcGemmJob* jobs, int njobs);

@@ -23,7 +23,8 @@
 // barrier, so that the MMA issuer waits on one barrier per stage); 1 MMA issuer (even
 // CTA only) and TMEM owner; 2 epilogue loader (TMA); 3-10 epilogue; 11-12 one thread
 // each that stores a group's finished W boxes (TMA) and hands the buffers back to the
-// loader.
+// loader.  (Issuing the two boxes of a stage from two threads changed nothing: the
+// stages wait for the data, not for the issuing thread.)
 constexpr int K2_STAGES = 5;
 constexpr int K2_STAGE_BYTES = 2 * A_STAGE_BYTES;       // A: 128 x 64, B half: 128 x 64
 constexpr int K2_GROUPS = 2;
@@ -135,10 +136,10 @@ k_tc_back_project(const TcMaps* __restrict__ maps, const BackTileDesc* __restric
           if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
           // all four boxes of the pair complete on the even CTA's barrier
           const uint32_t fb = ptx::map_to_cta(ptx::smem_u32(&ctl->full[stage]), 0);
-          const uint32_t sa = tiles_u32 + stage * K2_STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+          const uint32_t sa = tiles_u32 + stage * K2_STAGE_BYTES;
           if (rank == 0) ptx::mbar_expect_tx(ptx::smem_u32(&ctl->full[stage]), 2 * K2_STAGE_BYTES);
           ptx::tma_load_2d_pair(sa, &mp->g2a, fb, kb * BK, i0);
-          ptx::tma_load_2d_pair(sb, &mp->g2b, fb, kb * BK, jb0);
+          ptx::tma_load_2d_pair(sa + A_STAGE_BYTES, &mp->g2b, fb, kb * BK, jb0);
           if (++stage == K2_STAGES) { stage = 0; phase ^= 1u; }
         }
       }

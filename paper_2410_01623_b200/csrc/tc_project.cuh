@@ -56,7 +56,8 @@ static_assert(K1_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 // Per-tile record (256 l x BN r), built on the host once (32 bytes).
 struct ProjTileDesc {
-  float* colpart;      // partial sums of the tile's matrix: [2 part + which][l]
+  float* colpart;      // partial sums of the tile's matrix: [2 part + which][l]; EPI_PLAIN: the k-segments
+                       // of a split-precision product instead (see seg_word)
   int slot;            // index into the tensor-map table and the fast-scalar table
   int l0, r0;          // first unprojected index / first rank index of the tile
   int nkb;             // k-blocks: ceil(d / 64)
@@ -65,6 +66,16 @@ struct ProjTileDesc {
 };
 static_assert(sizeof(ProjTileDesc) == 32, "ProjTileDesc layout");
 constexpr int PROJ_A_CHUNKED = 1 << 30;
+
+// EPI_PLAIN products may run over up to three k-segments that accumulate into the same tile: segment
+// s multiplies A taken through the map g1a (bit s of asel clear) or g2a (set) with B taken through
+// g1b or g2b (bsel), each over the same nkb_seg k-blocks.  With an fp32 matrix split into a bf16 high
+// part and a bf16 remainder this gives hi*hi + hi*lo + lo*hi, a product good to about 2^-16.  The
+// word travels in the record's pointer field: bits 0-31 nkb_seg (0: one segment over all k-blocks),
+// 32-34 asel, 35-37 bsel.
+__host__ __device__ inline unsigned long long seg_word(int nkb_seg, unsigned asel, unsigned bsel) {
+  return (unsigned long long)(unsigned)nkb_seg | ((unsigned long long)(asel & 7u) << 32) | ((unsigned long long)(bsel & 7u) << 35);
+}
 
 struct ProjCtl {
   uint64_t full[K1_STAGES];     // (even CTA) both CTAs' operands of a stage have landed
@@ -170,10 +181,14 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         const int left = d.bn_left < 0;
         const int bn = d.bn_left & 0xffff;
         const int l0 = d.l0 + BM * (int)rank;             // this CTA's unprojected indices
-        const int rb0 = d.r0 + (bn / 2) * (int)rank;      // this CTA's half of the rank range
         const int nparts = (d.bn_left >> 16) & 0xff;
         int gturn = EPI == EPI_ADAM ? d.r0 / bn : -1;     // next k-block that the G^2 warps read
         const uint32_t bytes = 2 * (A_STAGE_BYTES + (bn / 2) * BK * 2);   // both CTAs together
+        const unsigned long long sw = EPI == EPI_PLAIN ? reinterpret_cast<unsigned long long>(d.colpart) : 0ull;
+        const int nkb_seg = (int)(sw & 0xffffffffu) ? (int)(sw & 0xffffffffu) : d.nkb;
+        const unsigned asel = (unsigned)(sw >> 32) & 7u, bsel = (unsigned)(sw >> 35) & 7u;
+        const int rb0 = d.r0 + (bn / 2) * (int)rank;      // this CTA's half of the rank range
+        int seg = 0, kk = 0;
         for (int kb = 0; kb < d.nkb; ++kb) {
           if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
           if ((gmask >> stage) & 1u) {                     // the previous occupant is still being squared
@@ -183,18 +198,21 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           if (kb == gturn) { gturn += nparts; gmask |= 1u << stage; } else { gmask &= ~(1u << stage); }
           // all boxes of the pair complete on the even CTA's barrier
           const uint32_t fb = ptx::map_to_cta(ptx::smem_u32(&ctl->full[stage]), 0);
-          const uint32_t sa = tiles_u32 + stage * K1_STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+          const uint32_t sa = tiles_u32 + stage * K1_STAGE_BYTES;
           if (rank == 0) ptx::mbar_expect_tx(ptx::smem_u32(&ctl->full[stage]), bytes);
-          const int k0 = kb * BK;
+          const int k0 = kk * BK;
+          const CUtensorMap* am = ((asel >> seg) & 1u) ? &mp->g2a : &mp->g1a;
+          const CUtensorMap* bm = ((bsel >> seg) & 1u) ? &mp->g2b : &mp->g1b;
+          if (++kk == nkb_seg) { kk = 0; ++seg; }
           if (d.bn_left & PROJ_A_CHUNKED) {
-            ptx::tma_load_3d_pair(sa, &mp->g1a, fb, 0, k0, l0 >> 6);
+            ptx::tma_load_3d_pair(sa, am, fb, 0, k0, l0 >> 6);
           } else if (left) {
-            ptx::tma_load_2d_pair(sa, &mp->g1a, fb, l0, k0);
-            ptx::tma_load_2d_pair(sa + CHUNK_BYTES, &mp->g1a, fb, l0 + 64, k0);
+            ptx::tma_load_2d_pair(sa, am, fb, l0, k0);
+            ptx::tma_load_2d_pair(sa + CHUNK_BYTES, am, fb, l0 + 64, k0);
           } else {
-            ptx::tma_load_2d_pair(sa, &mp->g1a, fb, k0, l0);
+            ptx::tma_load_2d_pair(sa, am, fb, k0, l0);
           }
-          ptx::tma_load_3d_pair(sb, &mp->g1b, fb, 0, k0, rb0 >> 6);
+          ptx::tma_load_3d_pair(sa + A_STAGE_BYTES, bm, fb, 0, k0, rb0 >> 6);
           if (++stage == K1_STAGES) { stage = 0; phase ^= 1u; }
         }
       }

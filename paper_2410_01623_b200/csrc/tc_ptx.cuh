@@ -42,10 +42,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // beyond any legitimate wait (one tile takes tens of microseconds).
 constexpr uint32_t kSpinLimit = 1u << 24;
 
-// Waits for the phase with the given parity.  Returns false if the CTA is aborting
-// (this wait ran out, or another role's did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+// Waits for the phase with the given parity, for at most `limit` tries.  Returns false if the CTA
+// is aborting (this wait ran out, or another role's did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t limit = kSpinLimit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 255u && *abort_flag) return false;
   }

@@ -93,7 +93,43 @@ def test_ablation_variants(flags, dtype):
         assert any(l < 1.0 for row in tr.lams for l in row)
 
 
+@pytest.mark.parametrize("flags", [fb.FLAG_ONLY_SCALING, fb.FLAG_ONLY_SCALING | fb.FLAG_MATRIX_SCALING])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_only_scaling_variant(flags, dtype):
+    """Fira-only-scaling, W <- W - eta phi(R) G, column and matrix level, both orientations: the
+    factors multiply the whole gradient, there is no P N term, and the limiter acts on ||G diag k||."""
+    tr = _random_case([(150, 333), (333, 150), (64, 200)], [37, 37, 16], dtype, steps=5, seed=53,
+                      spike=(4,), flags=flags)
+    tr.assert_ok()
+    assert any(l < 1.0 for row in tr.lams for l in row)
+    for i in range(3):
+        d = tr.f.diagnostics(i)
+        assert d["t"] == 5
+        assert d["norm_prev"] == pytest.approx(tr.st[i].prev_norm, rel=1e-3 if dtype == torch.float32 else 2e-2)
+        M, V, pn, t = tr.f.get_state(i)                    # the moments advance as in the ordinary step
+        Mo = tr.st[i].M.T if tr.shapes[i][0] <= tr.shapes[i][1] else tr.st[i].M
+        assert rel_err(to_np64(M), Mo) < 1e-4
+
+
+def test_only_scaling_printed_equation_on_the_device():
+    """alpha dropped from the scaled term and gamma = inf: (W_0 - W_1) / eta is G with column j
+    multiplied by k_j, element by element."""
+    hp = fb.make_hparams(lr=0.05, gamma=math.inf, flags=fb.FLAG_ONLY_SCALING | fb.FLAG_ALPHA_LOWRANK_ONLY)
+    tr = _random_case([(96, 160)], 16, torch.float32, steps=1, seed=59, hp=hp)
+    tr.assert_ok()
+    assert all(l == 1.0 for row in tr.lams for l in row)
+    d = tr.f.diagnostics(0)
+    assert d["k_max"] > d["k_min"] > 0
+    # every column of the update is a multiple of the same column of G, with a factor inside [k_min, k_max]
+    upd = (tr.W0[0] - to_np64(tr.W[0])) / 0.05
+    Wo_upd = (tr.W0[0] - tr.Wo[0]) / 0.05
+    kcol = (upd * Wo_upd).sum(axis=0) / (Wo_upd * Wo_upd).sum(axis=0)
+    np.testing.assert_allclose(kcol, 1.0, rtol=1e-5)
+
+
 def test_variant_flags_that_exclude_each_other_are_rejected():
+    with pytest.raises(fb.FiraError):
+        fb.Fira([(64, 96)], 8, torch.float32, fb.make_hparams(flags=fb.FLAG_ONLY_SCALING | fb.FLAG_NO_RESIDUAL))
     with pytest.raises(fb.FiraError):
         fb.Fira([(64, 96)], 8, torch.float32, fb.make_hparams(flags=fb.FLAG_MATRIX_SCALING | fb.FLAG_NO_SCALING))
     with pytest.raises(fb.FiraError):
