@@ -164,11 +164,14 @@ FIRA_API fira_status fira_adam_dense(const fira_hparams* hp, int32_t count, void
 /* The same pass as fira_step() (Algorithm 1's loop body) for callers whose weights
  * and gradients live in HOST memory: W_host and G_host are host arrays of `count`
  * host pointers (m x ld elements each; page-locked memory makes the copies
- * asynchronous).  Every G and W is copied into staging_dev, the step runs there,
- * and every W is copied back, all on the context's stream.  staging_dev is a
- * 256-byte aligned device buffer of at least fira_staging_bytes() bytes, owned by
- * the caller.  The host W buffers hold the result once the stream has been
- * synchronised. */
+ * asynchronous).  The matrix list is cut into chunks of consecutive matrices: while
+ * one chunk steps, the next one's G and W are on their way into staging_dev and the
+ * previous one's W on its way back, on two copy streams that the library creates on
+ * the first call and orders against the context's stream with events.  staging_dev
+ * is a 256-byte aligned device buffer of at least fira_staging_bytes() bytes, owned
+ * by the caller.  The host W buffers hold the result once the context's stream has
+ * been synchronised.  The state after the call equals that after fira_step() on the
+ * same data.  FIRA_FLAG_AUTO_REFRESH is not supported here (FIRA_ERR_UNSUPPORTED). */
 FIRA_API fira_status fira_step_host(fira_ctx* ctx, void* const* W_host, const void* const* G_host,
                                     float lr, void* staging_dev, size_t staging_bytes);
 FIRA_API size_t fira_staging_bytes(const fira_ctx* ctx);

@@ -5,6 +5,15 @@
 
 namespace fira { struct TcPlan; }
 
+namespace fira {
+// Streams and events of fira_step_host(): created on its first call.
+struct HostPipe {
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, out_done = nullptr;
+  std::vector<cudaEvent_t> in_done, stepped;     // per chunk
+};
+}  // namespace fira
+
 struct fira_ctx {
   fira_hparams hp;
   std::vector<fira_matrix_desc> descs;
@@ -31,7 +40,9 @@ struct fira_ctx {
   std::vector<int> simt_list, tc_list;
   std::vector<long long> t_host;         // host mirror of every matrix's step count
   fira::PhaseTimer timer;
+  fira::HostPipe pipe;
   bool table_dirty = true;
+  bool proj_weights_dirty = true;        // tensor-core path: column norms of the stored projections to be retaken
   int last_launches = 0;
 };
 

@@ -259,6 +259,7 @@ fira_status fira_init(fira_ctx** out, const fira_hparams* hp, const fira_matrix_
     c->simt.row_start = c->ints_dev + o_rs; c->simt.rows_total = rs.back();
     c->simt.w_tile_start = c->ints_dev + o_wt; c->simt.w_tiles = wt.back();
     c->simt.npart = c->ints_dev + o_np;
+    c->simt.h_proj_tile_start = pt; c->simt.h_row_start = rs; c->simt.h_w_tile_start = wt;
   }
   fira_status ts = tc_build_plan(c, ints);
   if (ts != FIRA_OK) { tc_destroy_plan(c); delete c; return ts; }
@@ -282,9 +283,59 @@ fira_status fira_init(fira_ctx** out, const fira_hparams* hp, const fira_matrix_
   return FIRA_OK;
 }
 
-fira_status fira_step(fira_ctx* c, void* const* W_dev, const void* const* G_dev, float lr) {
-  if (!c || !W_dev || !G_dev) { set_error("null argument"); return FIRA_ERR_INVALID_ARG; }
+// Registers the caller's W and G pointers (re-encoding what depends on them).
+static fira_status set_pointers(fira_ctx* c, void* const* W_dev, const void* const* G_dev) {
+  const int count = (int)c->mats.size();
+  bool ptr_changed = false;
+  for (int i = 0; i < count; ++i) {
+    if (c->mats[i].W != W_dev[i] || c->mats[i].G != G_dev[i]) {
+      c->mats[i].W = W_dev[i]; c->mats[i].G = G_dev[i];
+      ptr_changed = true;
+    }
+  }
+  if (ptr_changed) {
+    c->table_dirty = true;
+    fira_status s = tc_update_pointers(c);
+    if (s != FIRA_OK) return s;
+  }
+  if (c->table_dirty) { fira_status s = upload_table(c); if (s != FIRA_OK) return s; }
+  return FIRA_OK;
+}
+
+// Enqueues the step of the matrices [i0, i1) (both engines' lists are ascending, so the range maps
+// to one sub-range of each); returns the number of launches or -1.
+static int launch_range(fira_ctx* c, const Hyper& h, int i0, int i1, bool whole) {
+  if (whole) {
+    int launches = launch_simt_step(c->simt, h, c->status_dev, c->stream, &c->timer);
+    if (c->simt.nlist == 0) c->timer.mark(c->stream);
+    const int tcl = launch_tc_step(c, h);
+    return tcl < 0 ? -1 : launches + tcl;
+  }
+  auto sub = [&](const std::vector<int>& lst, int& qa, int& qb) {
+    qa = (int)(std::lower_bound(lst.begin(), lst.end(), i0) - lst.begin());
+    qb = (int)(std::lower_bound(lst.begin(), lst.end(), i1) - lst.begin());
+  };
+  int qa, qb, launches = 0;
+  sub(c->simt_list, qa, qb);
+  if (qb > qa) launches += launch_simt_step(c->simt, h, c->status_dev, c->stream, &c->timer, qa, qb);
+  sub(c->tc_list, qa, qb);
+  if (qb > qa) {
+    const int tcl = launch_tc_step(c, h, qa, qb);
+    if (tcl < 0) return -1;
+    launches += tcl;
+  }
+  return launches;
+}
+
+static fira_status check_step_args(fira_ctx* c, void* const* W, const void* const* G, float lr) {
+  if (!c || !W || !G) { set_error("null argument"); return FIRA_ERR_INVALID_ARG; }
   if (!(lr < 0.f) && !isfinite(lr)) { set_error("lr must be finite"); return FIRA_ERR_INVALID_ARG; }
+  return FIRA_OK;
+}
+
+fira_status fira_step(fira_ctx* c, void* const* W_dev, const void* const* G_dev, float lr) {
+  fira_status as = check_step_args(c, W_dev, G_dev, lr);
+  if (as != FIRA_OK) return as;
   const int count = (int)c->mats.size();
   for (int i = 0; i < count; ++i) {
     if (!W_dev[i] || !G_dev[i] || ((uintptr_t)W_dev[i] & 15) || ((uintptr_t)G_dev[i] & 15)) {
@@ -300,26 +351,12 @@ fira_status fira_step(fira_ctx* c, void* const* W_dev, const void* const* G_dev,
       if (rs != FIRA_OK) return rs;
     }
   }
-  bool ptr_changed = false;
-  for (int i = 0; i < count; ++i) {
-    if (c->mats[i].W != W_dev[i] || c->mats[i].G != G_dev[i]) {
-      c->mats[i].W = W_dev[i]; c->mats[i].G = G_dev[i];
-      ptr_changed = true;
-    }
-  }
-  if (ptr_changed) {
-    c->table_dirty = true;
-    fira_status s = tc_update_pointers(c);
-    if (s != FIRA_OK) return s;
-  }
-  if (c->table_dirty) { fira_status s = upload_table(c); if (s != FIRA_OK) return s; }
+  fira_status ps = set_pointers(c, W_dev, G_dev);
+  if (ps != FIRA_OK) return ps;
   const Hyper h = make_hyper(c->hp, lr);
   c->timer.begin_step();
-  int launches = launch_simt_step(c->simt, h, c->status_dev, c->stream, &c->timer);
-  if (c->simt.nlist == 0) c->timer.mark(c->stream);
-  const int tcl = launch_tc_step(c, h);
-  if (tcl < 0) return FIRA_ERR_CUDA;
-  launches += tcl;
+  const int launches = launch_range(c, h, 0, count, true);
+  if (launches < 0) return FIRA_ERR_CUDA;
   if (c->timer.on) c->timer.steps += 1;
   c->last_launches = launches;
   for (int i = 0; i < count; ++i) c->t_host[i] += 1;
@@ -336,7 +373,9 @@ size_t fira_staging_bytes(const fira_ctx* c) {
 
 fira_status fira_step_host(fira_ctx* c, void* const* W_host, const void* const* G_host, float lr,
                            void* staging_dev, size_t staging_bytes) {
-  if (!c || !W_host || !G_host || !staging_dev) { set_error("null argument"); return FIRA_ERR_INVALID_ARG; }
+  fira_status as = check_step_args(c, W_host, G_host, lr);
+  if (as != FIRA_OK) return as;
+  if (!staging_dev) { set_error("null argument"); return FIRA_ERR_INVALID_ARG; }
   if (((uintptr_t)staging_dev & 255) || staging_bytes < fira_staging_bytes(c)) {
     set_error("staging buffer must be 256-byte aligned and hold fira_staging_bytes() bytes");
     return FIRA_ERR_WORKSPACE_TOO_SMALL;
@@ -346,16 +385,78 @@ fira_status fira_step_host(fira_ctx* c, void* const* W_host, const void* const* 
     if (!W_host[i] || !G_host[i]) { set_error("null host matrix"); return FIRA_ERR_INVALID_ARG; }
   std::vector<void*> Wd(count);
   std::vector<const void*> Gd(count);
-  char* p = (char*)staging_dev;
-  for (int i = 0; i < count; ++i) {
-    const size_t bytes = matrix_bytes(c->mats[i]);
-    Gd[i] = p; FIRA_CUDA(cudaMemcpyAsync(p, G_host[i], bytes, cudaMemcpyHostToDevice, c->stream)); p += align_up(bytes);
-    Wd[i] = p; FIRA_CUDA(cudaMemcpyAsync(p, W_host[i], bytes, cudaMemcpyHostToDevice, c->stream)); p += align_up(bytes);
+  size_t total = 0;
+  {
+    char* p = (char*)staging_dev;
+    for (int i = 0; i < count; ++i) {
+      const size_t bytes = matrix_bytes(c->mats[i]);
+      Gd[i] = p; p += align_up(bytes);
+      Wd[i] = p; p += align_up(bytes);
+      total += bytes;
+    }
   }
-  fira_status s = fira_step(c, Wd.data(), Gd.data(), lr);
-  if (s != FIRA_OK) return s;
-  for (int i = 0; i < count; ++i)
-    FIRA_CUDA(cudaMemcpyAsync(W_host[i], Wd[i], matrix_bytes(c->mats[i]), cudaMemcpyDeviceToHost, c->stream));
+  // Chunks of consecutive matrices: while chunk q steps, chunk q + 1 is on its way in and the
+  // weights of chunk q - 1 on their way out (the link carries both directions at once).  Two
+  // side streams carry the copies; events order them against the context's stream.
+  HostPipe& hp_ = c->pipe;
+  if (!hp_.in) {
+    FIRA_CUDA(cudaStreamCreateWithFlags(&hp_.in, cudaStreamNonBlocking));
+    FIRA_CUDA(cudaStreamCreateWithFlags(&hp_.out, cudaStreamNonBlocking));
+    FIRA_CUDA(cudaEventCreateWithFlags(&hp_.start, cudaEventDisableTiming));
+    FIRA_CUDA(cudaEventCreateWithFlags(&hp_.out_done, cudaEventDisableTiming));
+  }
+  std::vector<int> cut{0};
+  {
+    const size_t target = std::max<size_t>(total / 32, (size_t)32 << 20);   // about 32 chunks, 32 MiB at least
+    size_t acc = 0;
+    for (int i = 0; i < count; ++i) {
+      acc += matrix_bytes(c->mats[i]);
+      if (acc >= target || i + 1 == count) { cut.push_back(i + 1); acc = 0; }
+    }
+  }
+  const int nchunk = (int)cut.size() - 1;
+  while ((int)hp_.in_done.size() < nchunk) {
+    cudaEvent_t a, b;
+    FIRA_CUDA(cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
+    FIRA_CUDA(cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
+    hp_.in_done.push_back(a); hp_.stepped.push_back(b);
+  }
+  if ((c->hp.flags & FIRA_FLAG_AUTO_REFRESH) && c->hp.T > 0) {
+    set_error("fira_step_host: FIRA_FLAG_AUTO_REFRESH is not supported with host buffers (refresh needs G on the device)");
+    return FIRA_ERR_UNSUPPORTED;
+  }
+  fira_status ps = set_pointers(c, Wd.data(), Gd.data());
+  if (ps != FIRA_OK) return ps;
+  const Hyper h = make_hyper(c->hp, lr);
+  // the copies start once everything enqueued so far on the context's stream has run (an earlier
+  // call's kernels may still be reading the staging buffer)
+  FIRA_CUDA(cudaEventRecord(hp_.start, c->stream));
+  FIRA_CUDA(cudaStreamWaitEvent(hp_.in, hp_.start, 0));
+  FIRA_CUDA(cudaStreamWaitEvent(hp_.out, hp_.start, 0));
+  c->timer.begin_step();
+  int launches = 0;
+  for (int q = 0; q < nchunk; ++q) {
+    for (int i = cut[q]; i < cut[q + 1]; ++i) {
+      const size_t bytes = matrix_bytes(c->mats[i]);
+      FIRA_CUDA(cudaMemcpyAsync(const_cast<void*>(Gd[i]), G_host[i], bytes, cudaMemcpyHostToDevice, hp_.in));
+      FIRA_CUDA(cudaMemcpyAsync(Wd[i], W_host[i], bytes, cudaMemcpyHostToDevice, hp_.in));
+    }
+    FIRA_CUDA(cudaEventRecord(hp_.in_done[q], hp_.in));
+    FIRA_CUDA(cudaStreamWaitEvent(c->stream, hp_.in_done[q], 0));
+    const int l = launch_range(c, h, cut[q], cut[q + 1], nchunk == 1);
+    if (l < 0) return FIRA_ERR_CUDA;
+    launches += l;
+    FIRA_CUDA(cudaEventRecord(hp_.stepped[q], c->stream));
+    FIRA_CUDA(cudaStreamWaitEvent(hp_.out, hp_.stepped[q], 0));
+    for (int i = cut[q]; i < cut[q + 1]; ++i)
+      FIRA_CUDA(cudaMemcpyAsync(W_host[i], Wd[i], matrix_bytes(c->mats[i]), cudaMemcpyDeviceToHost, hp_.out));
+  }
+  // the context's stream is done when the last weights have arrived
+  FIRA_CUDA(cudaEventRecord(hp_.out_done, hp_.out));
+  FIRA_CUDA(cudaStreamWaitEvent(c->stream, hp_.out_done, 0));
+  c->last_launches = launches;
+  for (int i = 0; i < count; ++i) c->t_host[i] += 1;
+  FIRA_CUDA(cudaGetLastError());
   return FIRA_OK;
 }
 
@@ -399,6 +500,7 @@ fira_status fira_set_projection(fira_ctx* c, int32_t idx, const void* P_dev) {
   const MatDev& mt = c->mats[idx];
   const size_t bytes = (size_t)mt.d * mt.r * (mt.bf16 ? 2 : 4);
   FIRA_CUDA(cudaMemcpyAsync(mt.P, P_dev, bytes, cudaMemcpyDeviceToDevice, c->stream));
+  c->proj_weights_dirty = true;
   return FIRA_OK;
 }
 
@@ -543,6 +645,12 @@ const char* fira_last_error(void) { return g_last_error.c_str(); }
 void fira_destroy(fira_ctx* c) {
   if (!c) return;
   tc_destroy_plan(c);
+  if (c->pipe.in) {
+    cudaStreamDestroy(c->pipe.in); cudaStreamDestroy(c->pipe.out);
+    cudaEventDestroy(c->pipe.start); cudaEventDestroy(c->pipe.out_done);
+    for (auto& ev : c->pipe.in_done) cudaEventDestroy(ev);
+    for (auto& ev : c->pipe.stepped) cudaEventDestroy(ev);
+  }
   for (auto& ev : c->timer.events) cudaEventDestroy(ev);
   delete c;
 }

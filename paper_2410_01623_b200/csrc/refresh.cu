@@ -51,6 +51,7 @@ struct RefreshMat {
   __nv_bfloat16* Zl;
   __nv_bfloat16* Ul;
   float* out32;        // optional copy of the kept basis in fp32, before it is rounded for storage
+  float* info;         // a few floats of the Cholesky factorisation (pivot floor)
   int tc;              // every product of this matrix runs on the tensor cores
   long long ld;
   int d, l, r;
@@ -137,109 +138,138 @@ k_rgemm(const GemmDesc* __restrict__ descs, int ndesc, const int* __restrict__ t
 }
 
 // ------------------------------------------------------------------ Cholesky
-// One cluster of CHOL_CTAS blocks per matrix: C (r x r, symmetric, row major) -> lower factor L in
-// place (the strict upper triangle is left as it was).  Left-looking over 64-wide block columns:
-// the row tiles of the panel update and the rows of the solve below the diagonal block are dealt
-// out to the blocks of the cluster, which meet at a cluster barrier (release/acquire, so that what
-// one block wrote to C is what the others read) after each phase; every block factors the 64 x 64
-// diagonal block for itself in shared memory.  shift_rel * trace(C)/r is added to the diagonal
-// first.  A non-positive or non-finite pivot is replaced and flagged.
+// C (r x r, symmetric, row major) -> lower factor L in place (the strict upper triangle is left as
+// it was), for all matrices of a chunk at once, right-looking over block columns of CB = 64.  Three
+// launches per block column, each over every matrix:
+//   k_chol_diag   one block per matrix factors the CB x CB diagonal block in shared memory
+//   k_chol_panel  the rows below it: L[i, J] = C[i, J] L_JJ^-T, 64 rows per block
+//   k_chol_update the trailing matrix: C[I, K] -= L[I, J] L[K, J]^T on 128 x 128 tiles of its lower half
+// On the first block column k_chol_diag also adds shift_rel * trace(C)/r to the whole diagonal and
+// notes the pivot floor in info[0].  A non-positive or non-finite pivot is replaced and flagged.
+// Matrices whose r does not reach the block column do nothing.
 constexpr int CB = 64;
-constexpr int CHOL_CTAS = 8;
 
-__device__ __forceinline__ void cluster_barrier() {
-  __threadfence();
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
-__global__ void __cluster_dims__(CHOL_CTAS, 1, 1) __launch_bounds__(GEMM_THREADS)
-k_cholesky(const RefreshMat* __restrict__ rm, float shift_rel, unsigned* __restrict__ status) {
-  __shared__ __align__(16) float As[TK][TM + 4];
-  __shared__ __align__(16) float Bs[TK][TN + 4];
+__global__ void __launch_bounds__(GEMM_THREADS)
+k_chol_diag(const RefreshMat* __restrict__ rm, int J0, float shift_rel, unsigned* __restrict__ status) {
   __shared__ float D[CB][CB + 1];
   __shared__ float red[GEMM_THREADS];
-  const RefreshMat m = rm[blockIdx.x / CHOL_CTAS];
-  const int rank = blockIdx.x % CHOL_CTAS;
+  const RefreshMat m = rm[blockIdx.x];
   const int r = m.r;
+  if (J0 >= r) return;
   float* C = m.C;
   const int tid = threadIdx.x;
-  float tr = 0.f;
-  for (int i = tid; i < r; i += GEMM_THREADS) tr += C[(long long)i * r + i];
-  red[tid] = tr;
+  float floor_pivot;
+  if (J0 == 0) {
+    float tr = 0.f;
+    for (int i = tid; i < r; i += GEMM_THREADS) tr += C[(long long)i * r + i];
+    red[tid] = tr;
+    __syncthreads();
+    for (int o = GEMM_THREADS / 2; o > 0; o >>= 1) {
+      if (tid < o) red[tid] += red[tid + o];
+      __syncthreads();
+    }
+    const float mean_diag = red[0] / (float)r;
+    const float shift = shift_rel * mean_diag;
+    floor_pivot = fmaxf(1e-30f, 1e-12f * mean_diag);
+    if (tid == 0) m.info[0] = floor_pivot;
+    for (int i = tid; i < r; i += GEMM_THREADS) C[(long long)i * r + i] += shift;
+    __syncthreads();                       // this block reads its own writes back below
+  } else {
+    floor_pivot = m.info[0];
+  }
+  const int jb = min(CB, r - J0);
+  for (int e = tid; e < CB * CB; e += GEMM_THREADS) {
+    const int i = e / CB, j = e % CB;
+    D[i][j] = (i < jb && j < jb) ? C[(long long)(J0 + i) * r + J0 + j] : (i == j ? 1.f : 0.f);
+  }
   __syncthreads();
-  for (int o = GEMM_THREADS / 2; o > 0; o >>= 1) {
-    if (tid < o) red[tid] += red[tid + o];
+  for (int k = 0; k < jb; ++k) {
+    if (tid == 0) {
+      float pv = D[k][k];
+      if (!(pv > floor_pivot) || !isfinite(pv)) { pv = floor_pivot; atomicOr(status, DEV_STATUS_NONFINITE); }
+      D[k][k] = sqrtf(pv);
+    }
+    __syncthreads();
+    const float dk = D[k][k];
+    if (tid > k && tid < jb) D[tid][k] /= dk;
+    __syncthreads();
+    const int rem = jb - k - 1;
+    for (int e = tid; e < rem * rem; e += GEMM_THREADS) {
+      const int i = k + 1 + e / rem, j = k + 1 + e % rem;
+      if (j <= i) D[i][j] -= D[i][k] * D[j][k];
+    }
     __syncthreads();
   }
-  const float mean_diag = red[0] / (float)r;
-  const float shift = shift_rel * mean_diag;
-  const float floor_pivot = fmaxf(1e-30f, 1e-12f * mean_diag);
-  cluster_barrier();                       // every block has read the unshifted diagonal
-  if (rank == 0)
-    for (int i = tid; i < r; i += GEMM_THREADS) C[(long long)i * r + i] += shift;
-  cluster_barrier();
+  for (int e = tid; e < jb * jb; e += GEMM_THREADS) {
+    const int i = e / jb, j = e % jb;
+    if (j <= i) C[(long long)(J0 + i) * r + J0 + j] = D[i][j];
+  }
+}
 
-  const int tx = tid & 15, ty = tid >> 4;
-  for (int J0 = 0; J0 < r; J0 += CB) {
-    const int jb = min(CB, r - J0);
-    // (a) C[I, J] -= L[I, :J0] L[J, :J0]^T for the row tiles I >= J, dealt out to the blocks
-    for (int I0 = J0 + TM * rank; I0 < r; I0 += TM * CHOL_CTAS) {
-      float acc[4][4] = {};
-      gemm_tile<1, float, float>(C, r, 1, C, 1, r, r, J0 + jb, J0, I0, J0, acc, As, Bs);
+// Rows below the diagonal block: one block per 64 rows (tiles_per_matrix of them per matrix),
+// one thread per row for the substitution.
+__global__ void __launch_bounds__(64)
+k_chol_panel(const RefreshMat* __restrict__ rm, int J0, int tiles_per_matrix) {
+  __shared__ float D[CB][CB + 1];
+  __shared__ float T[64][CB + 1];
+  const RefreshMat m = rm[blockIdx.x / tiles_per_matrix];
+  const int r = m.r;
+  const int jb = min(CB, r - J0);
+  const int I0 = J0 + CB + (blockIdx.x % tiles_per_matrix) * 64;
+  if (J0 >= r || I0 >= r) return;
+  float* C = m.C;
+  const int tid = threadIdx.x;
+  for (int e = tid; e < CB * CB; e += 64) {
+    const int i = e / CB, j = e % CB;
+    D[i][j] = (i < jb && j < jb) ? C[(long long)(J0 + i) * r + J0 + j] : (i == j ? 1.f : 0.f);
+    T[i][j] = (I0 + i < r && j < jb) ? C[(long long)(I0 + i) * r + J0 + j] : 0.f;
+  }
+  __syncthreads();
+  if (I0 + tid < r) {
+    float* row = T[tid];
+    for (int c = 0; c < jb; ++c) {
+      float v = row[c];
+      for (int k = 0; k < c; ++k) v -= row[k] * D[c][k];
+      row[c] = v / D[c][c];
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e < CB * CB; e += 64) {
+    const int i = e / CB, j = e % CB;
+    if (I0 + i < r && j < jb) C[(long long)(I0 + i) * r + J0 + j] = T[i][j];
+  }
+}
+
+// Trailing update on the 128 x 128 tiles (I >= K) of the part below and right of the panel.
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
+k_chol_update(const RefreshMat* __restrict__ rm, int J0, int nt) {
+  __shared__ __align__(16) float As[TK][SIMT_TILE + 4];
+  __shared__ __align__(16) float Bs[TK][SIMT_TILE + 4];
+  const int per = nt * (nt + 1) / 2;
+  const RefreshMat m = rm[blockIdx.x / per];
+  const int r = m.r;
+  if (J0 + CB >= r) return;
+  int p = blockIdx.x % per, ti = 0;
+  while (p > ti) { p -= ti + 1; ++ti; }        // tile row ti, tile column p <= ti
+  const int first = ((J0 + CB) / SIMT_TILE) * SIMT_TILE;      // tiles start at a multiple of 128 at or below the panel's end
+  const int I0 = first + ti * SIMT_TILE, K0 = first + p * SIMT_TILE;
+  if (I0 >= r) return;
+  float* C = m.C;
+  const int jb = min(CB, r - J0);
+  float acc[4 * SIMT_Q][4 * SIMT_Q] = {};
+  // A(i, k) = C[i][J0 + k], B(k, j) = C[j][J0 + k]
+  gemm_tile<SIMT_Q, float, float>(C + J0, r, 1, C + J0, 1, r, r, r, jb, I0, K0, acc, As, Bs);
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int lo = J0 + CB;                      // only rows and columns past the panel change
 #pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        const int i = I0 + ty * 4 + x;
-        if (i >= r) continue;
+  for (int x = 0; x < 4 * SIMT_Q; ++x) {
+    const int i = I0 + tile_coord(ty, x);
+    if (i >= r || i < lo) continue;
 #pragma unroll
-        for (int y = 0; y < 4; ++y) {
-          const int j = J0 + tx * 4 + y;
-          if (j < J0 + jb) C[(long long)i * r + j] -= acc[x][y];
-        }
-      }
+    for (int y = 0; y < 4 * SIMT_Q; ++y) {
+      const int j = K0 + tile_coord(tx, y);
+      if (j <= i && j >= lo) C[(long long)i * r + j] -= acc[x][y];
     }
-    cluster_barrier();
-    // (b) every block factors the diagonal block in its own shared memory
-    for (int e = tid; e < CB * CB; e += GEMM_THREADS) {
-      const int i = e / CB, j = e % CB;
-      D[i][j] = (i < jb && j < jb) ? C[(long long)(J0 + i) * r + J0 + j] : (i == j ? 1.f : 0.f);
-    }
-    __syncthreads();
-    for (int k = 0; k < jb; ++k) {
-      if (tid == 0) {
-        float pv = D[k][k];
-        if (!(pv > floor_pivot) || !isfinite(pv)) { pv = floor_pivot; if (rank == 0) atomicOr(status, DEV_STATUS_NONFINITE); }
-        D[k][k] = sqrtf(pv);
-      }
-      __syncthreads();
-      const float dk = D[k][k];
-      if (tid > k && tid < jb) D[tid][k] /= dk;
-      __syncthreads();
-      const int rem = jb - k - 1;
-      for (int e = tid; e < rem * rem; e += GEMM_THREADS) {
-        const int i = k + 1 + e / rem, j = k + 1 + e % rem;
-        if (j <= i) D[i][j] -= D[i][k] * D[j][k];
-      }
-      __syncthreads();
-    }
-    // all blocks have copied the unfactored block before block 0 overwrites it
-    cluster_barrier();
-    if (rank == 0) {
-      for (int e = tid; e < jb * jb; e += GEMM_THREADS) {
-        const int i = e / jb, j = e % jb;
-        if (j <= i) C[(long long)(J0 + i) * r + J0 + j] = D[i][j];
-      }
-    }
-    // (c) rows below: L[i, J] = C[i, J] L_JJ^-T, one thread per row, rows dealt out to the blocks
-    for (int i = J0 + jb + rank * GEMM_THREADS + tid; i < r; i += GEMM_THREADS * CHOL_CTAS) {
-      float* row = C + (long long)i * r + J0;
-      for (int c = 0; c < jb; ++c) {
-        float v = row[c];
-        for (int k = 0; k < c; ++k) v -= row[k] * D[c][k];
-        row[c] = v / D[c][c];
-      }
-    }
-    cluster_barrier();
   }
 }
 
@@ -388,7 +418,7 @@ static TcGemmJob refresh_job(const fira_matrix_desc& dsc, int kind) {
 
 static size_t refresh_data_bytes(const fira_matrix_desc& d) {
   const size_t dd = std::min(d.m, d.n), ll = std::max(d.m, d.n), r = d.r;
-  size_t b = align_up(dd * r * 4) + align_up(ll * r * 4) + align_up(r * r * 4);
+  size_t b = align_up(dd * r * 4) + align_up(ll * r * 4) + align_up(r * r * 4) + 256;
   if (refresh_on_tc(d)) {
     b += align_up(r * r * 4) + 2 * (align_up(dd * r * 2) + align_up(ll * r * 2) + align_up(r * r * 2));
     for (int k = 0; k < JOB_KINDS; ++k) { const TcGemmJob j = refresh_job(d, k); b += tc_gemm_table_bytes(&j, 1); }
@@ -416,6 +446,7 @@ size_t refresh_bytes_per_matrix(const fira_matrix_desc& d) {
 fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vector<int>& which,
                          uint64_t seed, int iters, float* const* basis_out) {
   if (iters < 0) iters = 4;
+  c->proj_weights_dirty = true;
   cudaStream_t st = c->stream;
   size_t pos = 0;
   while (pos < which.size()) {
@@ -444,6 +475,7 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
       rm.Y = (float*)base; base += align_up((size_t)mt.d * r * 4);
       rm.Z = (float*)base; base += align_up((size_t)mt.l * r * 4);
       rm.C = (float*)base; base += align_up(r * r * 4);
+      rm.info = (float*)base; base += 256;
       rm.tc = refresh_on_tc(c->descs[idx]) ? 1 : 0;
       if (rm.tc) {
         rm.U = (float*)base; base += align_up(r * r * 4);
@@ -545,6 +577,8 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
         tp += bytes;
       }
     }
+    int rmax = 0;
+    for (const RefreshMat& m : rms) rmax = std::max(rmax, m.r);
     const dim3 ew_grid(296, nm);      // element-wise helpers: every matrix of the chunk, tc ones act
     // A Z -> Y and A^T Y -> Z.  precise: the iterate enters with its bf16 remainder as a second k-segment.
     auto product = [&](bool az, bool precise) -> fira_status {
@@ -570,7 +604,14 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
           const fira_status gs = tc_gemm_run(c, tab[y ? JOB_GRAM_Y : JOB_GRAM_Z], ntc, jtiles[y ? JOB_GRAM_Y : JOB_GRAM_Z]);
           if (gs != FIRA_OK) return gs;
         }
-        k_cholesky<<<nm * CHOL_CTAS, GEMM_THREADS, 0, st>>>(rm_dev, pass == 0 ? 1e-6f : 0.f, c->status_dev);
+        for (int J0 = 0; J0 < rmax; J0 += CB) {
+          k_chol_diag<<<nm, GEMM_THREADS, 0, st>>>(rm_dev, J0, pass == 0 ? 1e-6f : 0.f, c->status_dev);
+          if (J0 + CB < rmax) {
+            k_chol_panel<<<nm * ((rmax - J0 - CB + 63) / 64), 64, 0, st>>>(rm_dev, J0, (rmax - J0 - CB + 63) / 64);
+            const int nt = (rmax - ((J0 + CB) / SIMT_TILE) * SIMT_TILE + SIMT_TILE - 1) / SIMT_TILE;
+            k_chol_update<<<nm * (nt * (nt + 1) / 2), GEMM_THREADS, 0, st>>>(rm_dev, J0, nt);
+          }
+        }
         if (nsimt) {
           if (y) k_trsm_rows<<<sTY.back(), GEMM_THREADS, 0, st>>>(dTY, nsimt, dsTY);
           else k_trsm_rows<<<sTZ.back(), GEMM_THREADS, 0, st>>>(dTZ, nsimt, dsTZ);

@@ -48,12 +48,13 @@ __device__ __forceinline__ void project_tile(const MatDev& mt, int tile, float (
 
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
 k_project(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
-          const int* __restrict__ tile_start) {
+          const int* __restrict__ tile_start, int first) {
   __shared__ __align__(16) float As[TK][SIMT_TILE + 4];
   __shared__ __align__(16) float Bs[TK][SIMT_TILE + 4];
-  const int p = find_matrix(tile_start, nlist, blockIdx.x);
+  const int gt = blockIdx.x + first;
+  const int p = find_matrix(tile_start, nlist, gt);
   const MatDev mt = mats[list[p]];
-  const int tile = blockIdx.x - tile_start[p];
+  const int tile = gt - tile_start[p];
   if (mt.bf16) project_tile<__nv_bfloat16>(mt, tile, As, Bs);
   else project_tile<float>(mt, tile, As, Bs);
 }
@@ -62,10 +63,10 @@ k_project(const MatDev* __restrict__ mats, const int* __restrict__ list, int nli
 // One warp per unprojected index l.  N goes to Xt.
 __global__ void __launch_bounds__(256)
 k_adam_rows(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
-            const int* __restrict__ row_start, int rows_total, Hyper hp) {
+            const int* __restrict__ row_start, int first_row, int rows_total, Hyper hp) {
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  const int row = first_row + blockIdx.x * warps_per_block + (threadIdx.x >> 5);
   if (row >= rows_total) return;
   const int p = find_matrix(row_start, nlist, row);
   const MatDev mt = mats[list[p]];
@@ -171,13 +172,14 @@ __device__ __forceinline__ void back_tile(const MatDev& mt, int tile, float lr, 
 template <int MODE>
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
 k_back_project(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
-               const int* __restrict__ tile_start, float lr, float a_res) {
+               const int* __restrict__ tile_start, int first, float lr, float a_res) {
   __shared__ __align__(16) float As[TK][SIMT_TILE + 4];
   __shared__ __align__(16) float Bs[TK][SIMT_TILE + 4];
   __shared__ float red[GEMM_THREADS / 32];
-  const int p = find_matrix(tile_start, nlist, blockIdx.x);
+  const int gt = blockIdx.x + first;
+  const int p = find_matrix(tile_start, nlist, gt);
   const MatDev mt = mats[list[p]];
-  const int tile = blockIdx.x - tile_start[p];
+  const int tile = gt - tile_start[p];
   if (mt.bf16) back_tile<__nv_bfloat16, MODE>(mt, tile, lr, a_res, As, Bs, red);
   else back_tile<float, MODE>(mt, tile, lr, a_res, As, Bs, red);
 }
@@ -185,9 +187,9 @@ k_back_project(const MatDev* __restrict__ mats, const int* __restrict__ list, in
 // ---------------------------------------------------------------- phase 5
 __global__ void __launch_bounds__(256)
 k_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
-         const int* __restrict__ row_start, int rows_total, float a_low, float a_res) {
+         const int* __restrict__ row_start, int first_row, int rows_total, float a_low, float a_res) {
   const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int row = first_row + blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= rows_total) return;
   const int p = find_matrix(row_start, nlist, row);
   const MatDev mt = mats[list[p]];
@@ -223,11 +225,12 @@ __device__ __forceinline__ float scaled_gradient_tile(const MatDev& mt, int i0, 
 template <int UPDATE>
 __global__ void __launch_bounds__(256)
 k_scaled_gradient(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
-                  const int* __restrict__ tile_start, int tile, float lr, float a_res) {
+                  const int* __restrict__ tile_start, int first, int tile, float lr, float a_res) {
   __shared__ float red[8];
-  const int p = find_matrix(tile_start, nlist, blockIdx.x);
+  const int gt = blockIdx.x + first;
+  const int p = find_matrix(tile_start, nlist, gt);
   const MatDev mt = mats[list[p]];
-  const int t = blockIdx.x - tile_start[p];
+  const int t = gt - tile_start[p];
   const int ct = (mt.n + tile - 1) / tile;
   const int i0 = (t / ct) * tile, j0 = (t % ct) * tile;
   const float c = UPDATE ? lr * a_res * mt.sc->lambda : 0.f;
@@ -248,11 +251,11 @@ k_scaled_gradient(const MatDev* __restrict__ mats, const int* __restrict__ list,
 
 }  // namespace
 
-void launch_scaled_gradient(const MatDev* mats, const int* list, int nlist, const int* tile_start, int tiles,
-                            int tile, int update, float lr, float a_res, cudaStream_t st) {
+void launch_scaled_gradient(const MatDev* mats, const int* list, int nlist, const int* tile_start, int first,
+                            int tiles, int tile, int update, float lr, float a_res, cudaStream_t st) {
   if (tiles <= 0) return;
-  if (update) k_scaled_gradient<1><<<tiles, 256, 0, st>>>(mats, list, nlist, tile_start, tile, lr, a_res);
-  else k_scaled_gradient<0><<<tiles, 256, 0, st>>>(mats, list, nlist, tile_start, tile, lr, a_res);
+  if (update) k_scaled_gradient<1><<<tiles, 256, 0, st>>>(mats, list, nlist, tile_start, first, tile, lr, a_res);
+  else k_scaled_gradient<0><<<tiles, 256, 0, st>>>(mats, list, nlist, tile_start, first, tile, lr, a_res);
 }
 
 // ---------------------------------------------------------------- phase 4
@@ -328,35 +331,46 @@ const char* const kSimtPhaseNames[6] = {"k_project", "k_adam_rows", "k_back_proj
                                         "k_finalize", "k_form_x", "k_back_project<update>"};
 
 int launch_simt_step(const SimtPlan& pl, const Hyper& hp, unsigned* status_dev, cudaStream_t st,
-                     PhaseTimer* tm) {
+                     PhaseTimer* tm, int qa, int qb) {
   if (pl.nlist == 0) return 0;
+  // the sub-range [qa, qb) of the list: first tile / row and their counts from the host copies of
+  // the prefix arrays; the kernels still search the whole arrays with absolute indices
+  int pt0 = 0, pt1 = pl.proj_tiles, r0 = 0, r1 = pl.rows_total, wt0 = 0, wt1 = pl.w_tiles, nq = pl.nlist;
+  if (qb >= 0) {
+    if (qa >= qb) return 0;
+    pt0 = pl.h_proj_tile_start[qa]; pt1 = pl.h_proj_tile_start[qb];
+    r0 = pl.h_row_start[qa]; r1 = pl.h_row_start[qb];
+    wt0 = pl.h_w_tile_start[qa]; wt1 = pl.h_w_tile_start[qb];
+    nq = qb - qa;
+  } else {
+    qa = 0;
+  }
   tm->mark(st);
-  k_project<<<pl.proj_tiles, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.proj_tile_start);
+  k_project<<<pt1 - pt0, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.proj_tile_start, pt0);
   tm->mark(st);
-  const int row_blocks = (pl.rows_total + 7) / 8;
-  k_adam_rows<<<row_blocks, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.row_start, pl.rows_total, hp);
+  const int row_blocks = (r1 - r0 + 7) / 8;
+  k_adam_rows<<<row_blocks, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.row_start, r0, r1, hp);
   tm->mark(st);
   if (hp.mode & HYPER_ONLY_SCALING) {
     // W <- W - lr phi(R) G: the norm of the scaled gradient, the limiter, the element-wise update
-    launch_scaled_gradient(pl.mats, pl.list, pl.nlist, pl.w_tile_start, pl.w_tiles, SIMT_TILE, 0, 0.f, hp.a_res, st);
+    launch_scaled_gradient(pl.mats, pl.list, pl.nlist, pl.w_tile_start, wt0, wt1 - wt0, SIMT_TILE, 0, 0.f, hp.a_res, st);
     tm->mark(st);
-    k_finalize<<<pl.nlist, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.npart, hp, status_dev);
+    k_finalize<<<nq, 256, 0, st>>>(pl.mats, pl.list + qa, nq, pl.npart + qa, hp, status_dev);
     tm->mark(st);
     tm->mark(st);
-    launch_scaled_gradient(pl.mats, pl.list, pl.nlist, pl.w_tile_start, pl.w_tiles, SIMT_TILE, 1, hp.lr, hp.a_res, st);
+    launch_scaled_gradient(pl.mats, pl.list, pl.nlist, pl.w_tile_start, wt0, wt1 - wt0, SIMT_TILE, 1, hp.lr, hp.a_res, st);
     tm->mark(st);
     return 5;
   }
-  k_back_project<MODE_NORM><<<pl.w_tiles, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist,
-                                                                 pl.w_tile_start, 0.f, hp.a_res);
+  k_back_project<MODE_NORM><<<wt1 - wt0, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist,
+                                                                pl.w_tile_start, wt0, 0.f, hp.a_res);
   tm->mark(st);
-  k_finalize<<<pl.nlist, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.npart, hp, status_dev);
+  k_finalize<<<nq, 256, 0, st>>>(pl.mats, pl.list + qa, nq, pl.npart + qa, hp, status_dev);
   tm->mark(st);
-  k_form_x<<<row_blocks, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.row_start, pl.rows_total,
-                                       hp.a_low, hp.a_res);
+  k_form_x<<<row_blocks, 256, 0, st>>>(pl.mats, pl.list, pl.nlist, pl.row_start, r0, r1, hp.a_low, hp.a_res);
   tm->mark(st);
-  k_back_project<MODE_UPDATE><<<pl.w_tiles, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist,
-                                                                   pl.w_tile_start, hp.lr, hp.a_res);
+  k_back_project<MODE_UPDATE><<<wt1 - wt0, GEMM_THREADS, 0, st>>>(pl.mats, pl.list, pl.nlist,
+                                                                  pl.w_tile_start, wt0, hp.lr, hp.a_res);
   tm->mark(st);
   return 6;
 }

@@ -17,11 +17,14 @@ struct SimtPlan {
   const int* w_tile_start = nullptr;     // 64 x 64 tiles of W (m x n)
   int w_tiles = 0;
   const int* npart = nullptr;            // partial sums per matrix (= its W tiles)
+  // host copies of the three prefix arrays (needed only to step a sub-range of the list)
+  std::vector<int> h_proj_tile_start, h_row_start, h_w_tile_start;
 };
 
-// Enqueues the six phases; returns the number of launches.
+// Enqueues the six phases for the matrices [qa, qb) of the list (qb < 0: the whole list); returns
+// the number of launches.
 int launch_simt_step(const SimtPlan& pl, const Hyper& hp, unsigned* status_dev, cudaStream_t st,
-                     PhaseTimer* tm);
+                     PhaseTimer* tm, int qa = 0, int qb = -1);
 extern const char* const kSimtPhaseNames[6];
 
 // One block of 256 threads per matrix of the list: sums the matrix's partial sums
@@ -32,10 +35,10 @@ __global__ void k_finalize(const MatDev* __restrict__ mats, const int* __restric
                            const int* __restrict__ npart_of, Hyper hp, unsigned* __restrict__ status);
 
 // Fira-only-scaling, element-wise over tiles of `tile` x `tile` elements of W (one block of 256
-// threads per tile; tile_start holds nlist + 1 ascending tile counts; first_block is added to the
-// block index).  update = 0: part[tile] = sum over the tile of (k_l G)^2, the norm that the
+// threads per tile; tile_start holds nlist + 1 ascending tile counts; `first` is added to the
+// block index, `tiles` blocks are launched).  update = 0: part[tile] = sum over the tile of (k_l G)^2, the norm that the
 // limiter sees; update = 1: W <- W - lr a_res lambda k_l G.
-void launch_scaled_gradient(const MatDev* mats, const int* list, int nlist, const int* tile_start, int tiles,
-                            int tile, int update, float lr, float a_res, cudaStream_t st);
+void launch_scaled_gradient(const MatDev* mats, const int* list, int nlist, const int* tile_start, int first,
+                            int tiles, int tile, int update, float lr, float a_res, cudaStream_t st);
 
 }  // namespace fira

@@ -13,9 +13,14 @@
 //   k_tc_form_x        X = a_low N - a_res lambda k_l R  (bf16)
 //   k_tc_back_project  D = Pi X on the tensor cores; epilogue: W -= lr (D + a_res lambda k_l G)
 //
-// ||S_l||^2 = ||G_l||^2 - ||R_l||^2 holds for a projection with orthonormal columns;
-// with a bf16-rounded projection it is exact to about 2^-8 ||R_l||^2.  It only enters
-// the limiter factor lambda and the remembered norm.
+// ||S_l||^2 = ||G_l - Pi R_l||^2 = ||G_l||^2 - 2 ||R_l||^2 + R_l^T (Pi^T Pi) R_l.  For orthonormal
+// columns this is ||G_l||^2 - ||R_l||^2; the stored projection is rounded to bf16, and where its
+// columns are concentrated on a few coordinates (outlier columns of G) their norms are off by up
+// to 2^-8, which matters because ||S||^2 is a small difference when the subspace holds most of
+// the energy.  The kernels therefore use the diagonal of Pi^T Pi: ||S_l||^2 = ||G_l||^2 -
+// sum_j (2 - ||pi_j||^2) R_lj^2, with the column norms of the stored projection recomputed
+// whenever it changes (k_tc_proj_weights); what is left is the off-diagonal part, which
+// averages out.  It only enters the limiter factor lambda and the remembered norm.
 //
 // Both tensor-core kernels run on CTA pairs (clusters of two, tcgen05 cta_group::2):
 // tiles of 256 x BN <= 256 accumulator elements per pair, 64 (one 128-byte swizzle row of
@@ -83,9 +88,31 @@ __device__ __forceinline__ void unpack8_bf16(const uint4& u, float (&v)[8]) {
 #include "tc_back_project.cuh"
 
 // ============================================================================ small kernels
-__global__ void k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist, Hyper hp,
+// w_j = 2 - ||pi_j||^2 for the columns of the stored projection [d][r]: 128 columns per block,
+// two threads per column (even and odd rows), fp32 sums in a fixed order.
+__global__ void __launch_bounds__(256)
+k_tc_proj_weights(const MatDev* __restrict__ mats, const int* __restrict__ list, const int* __restrict__ wq_off,
+                  const int* __restrict__ blk_start, int nlist, float* __restrict__ wq_all) {
+  __shared__ float part[256];
+  const int p = find_matrix(blk_start, nlist, blockIdx.x);
+  const MatDev& mt = mats[list[p]];
+  const int j = (blockIdx.x - blk_start[p]) * 128 + (threadIdx.x & 127);
+  const int half = threadIdx.x >> 7;
+  const __nv_bfloat16* P = static_cast<const __nv_bfloat16*>(mt.P);
+  float acc = 0.f;
+  if (j < mt.r)
+    for (int i = half; i < mt.d; i += 2) {
+      const float v = __bfloat162float(P[(long long)i * mt.r + j]);
+      acc = fmaf(v, v, acc);
+    }
+  part[threadIdx.x] = acc;
+  __syncthreads();
+  if (half == 0 && j < mt.r) wq_all[wq_off[p] + j] = 2.f - (part[threadIdx.x] + part[threadIdx.x + 128]);
+}
+
+__global__ void k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict__ list, int first, int nlist, Hyper hp,
                           float* __restrict__ fast) {
-  const int p = blockIdx.x * blockDim.x + threadIdx.x;
+  const int p = first + blockIdx.x * blockDim.x + threadIdx.x;
   if (p >= nlist) return;
   const MatDev& mt = mats[list[p]];
   const double s = (double)(mt.sc->t + 1);
@@ -143,10 +170,11 @@ __device__ __forceinline__ void copy_row_from_aligned(unsigned short* __restrict
 
 __global__ void __launch_bounds__(256)
 k_tc_stage(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
-           const int* __restrict__ row_start, int dir) {
-  const int p = find_matrix(row_start, nlist, blockIdx.x);
+           const int* __restrict__ row_start, int first_row, int dir) {
+  const int gr = blockIdx.x + first_row;
+  const int p = find_matrix(row_start, nlist, gr);
   const MatDev& mt = mats[list[p]];
-  const long long i = blockIdx.x - row_start[p];
+  const long long i = gr - row_start[p];
   const unsigned short* g = static_cast<const unsigned short*>(mt.G) + i * mt.ld;
   unsigned short* w = static_cast<unsigned short*>(mt.W) + i * mt.ld;
   unsigned short* gs = reinterpret_cast<unsigned short*>(mt.Gs) + i * mt.lds;
@@ -162,11 +190,12 @@ k_tc_stage(const MatDev* __restrict__ mats, const int* __restrict__ list, int nl
 // k_l and the partial sums of ||S||^2, 256 values of l per block.
 __global__ void __launch_bounds__(256)
 k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
-                const int* __restrict__ start, Hyper hp) {
+                const int* __restrict__ start, int first, Hyper hp) {
   __shared__ float red[8];
-  const int p = find_matrix(start, nlist, blockIdx.x);
+  const int gb = blockIdx.x + first;
+  const int p = find_matrix(start, nlist, gb);
   const MatDev& mt = mats[list[p]];
-  const int b = blockIdx.x - start[p];
+  const int b = gb - start[p];
   const int l = b * 256 + threadIdx.x;
   float contrib = 0.f;
   if (l < mt.l) {
@@ -177,12 +206,14 @@ k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, i
       rn += mt.colpart[(long long)(2 * q + 1) * mt.l + l];
     }
     for (int q = 2 * nparts; q < (2 + K1_GSQ_SPLIT) * nparts; ++q) gs += mt.colpart[(long long)q * mt.l + l];   // ||G_l||^2 in parts
+    float rw = 0.f;                                      // sum_j (2 - ||pi_j||^2) R_lj^2
+    for (int q = 0; q < nparts; ++q) rw += mt.colpart[(long long)((2 + K1_GSQ_SPLIT) * nparts + q) * mt.l + l];
     float k = sqrtf(nn) / (sqrtf(rn) + hp.eps);
     if (hp.mode & HYPER_MATRIX_SCALING) { mt.aux[l] = nn; mt.aux[mt.l + l] = rn; k = 1.f; }   // see k_finalize
     if (hp.mode & HYPER_NO_SCALING) k = 1.f;
     mt.kvec[l] = k;
     // only-scaling: S = G diag(k), so ||S_l||^2 = k_l^2 ||G_l||^2
-    contrib = k * k * ((hp.mode & HYPER_ONLY_SCALING) ? gs : fmaxf(gs - rn, 0.f));
+    contrib = k * k * ((hp.mode & HYPER_ONLY_SCALING) ? gs : fmaxf(gs - rw, 0.f));
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xffffffffu, contrib, o);
@@ -198,10 +229,10 @@ k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, i
 // X = a_low N - a_res lambda k_l R in bf16, one warp per l.
 __global__ void __launch_bounds__(256)
 k_tc_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
-            const int* __restrict__ row_start, int rows_total, float a_low, float a_res,
+            const int* __restrict__ row_start, int first_row, int rows_total, float a_low, float a_res,
             float* __restrict__ fast) {
   const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int row = first_row + blockIdx.x * 8 + (threadIdx.x >> 5);
   if (row >= rows_total) return;
   const int p = find_matrix(row_start, nlist, row);
   const MatDev& mt = mats[list[p]];
@@ -317,8 +348,14 @@ struct TcPlan {
   ProjTileDesc* td1_dev = nullptr;   // per-tile records of the projection
   BackTileDesc* td2_dev = nullptr;   // per-tile records of the back-projection
   float* fast_dev = nullptr;         // per matrix of the list: {bias factor, lambda}
+  float* wq_dev = nullptr;           // weights 2 - ||pi_j||^2 of all matrices of the list, r floats each
+  const int* wq_off = nullptr;       // per matrix: its offset into wq_dev
+  const int* wq_blk = nullptr;       // prefix sums of the blocks of k_tc_proj_weights
+  int wq_blocks = 0;
   int num_sms = 148;
   bool attrs_set = false;
+  // host copies of the prefix arrays (needed only to step a sub-range of the list)
+  std::vector<int> h_k1, h_k2, h_cs, h_rs, h_sl, h_ss;
 };
 
 bool tc_supported(const fira_matrix_desc& d) {
@@ -333,7 +370,7 @@ long long tc_staging_pitch(const fira_matrix_desc& d) {
 
 size_t tc_colpart_floats(const fira_matrix_desc& d) {
   const size_t l = std::max(d.m, d.n);
-  return (2 + K1_GSQ_SPLIT) * (size_t)(d.r / host_tile_bn(d.r)) * l;   // N^2 and R^2 per r-tile, then the partial G^2
+  return (3 + K1_GSQ_SPLIT) * (size_t)(d.r / host_tile_bn(d.r)) * l;   // N^2 and R^2 per r-tile, the partial G^2, the weighted R^2
 }
 
 size_t tc_part_floats(const fira_matrix_desc& d) { return ((size_t)std::max(d.m, d.n) + 255) / 256; }
@@ -349,11 +386,11 @@ static size_t back_tiles(const fira_matrix_desc& d) {
 
 // Device tables of this engine: tensor maps, fast scalars, back-projection tile records.
 size_t tc_tables_bytes(const fira_hparams& hp, const fira_matrix_desc* descs, int count) {
-  size_t ntc = 0, tiles2 = 0, tiles1 = 0;
+  size_t ntc = 0, tiles2 = 0, tiles1 = 0, rsum = 0;
   for (int i = 0; i < count; ++i)
-    if (engine_for(hp, descs[i]) == 1) { ++ntc; tiles2 += back_tiles(descs[i]); tiles1 += proj_tiles(descs[i]); }
+    if (engine_for(hp, descs[i]) == 1) { ++ntc; tiles2 += back_tiles(descs[i]); tiles1 += proj_tiles(descs[i]); rsum += descs[i].r; }
   return align_up(sizeof(TcMaps) * ntc) + align_up(2 * sizeof(float) * ntc) +
-         align_up(sizeof(BackTileDesc) * tiles2) + align_up(sizeof(ProjTileDesc) * tiles1);
+         align_up(sizeof(BackTileDesc) * tiles2) + align_up(sizeof(ProjTileDesc) * tiles1) + align_up(sizeof(float) * rsum);
 }
 
 static bool encode_matrix_maps(const MatDev& mt0, TcMaps& mp, bool only_g) {
@@ -386,7 +423,8 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
   c->tc = pl;
   cudaDeviceGetAttribute(&pl->num_sms, cudaDevAttrMultiProcessorCount, c->device);
   const std::vector<int>& lst = c->tc_list;
-  std::vector<int> k1{0}, k2{0}, cs{0}, rs{0}, np, sl, ss{0};
+  std::vector<int> k1{0}, k2{0}, cs{0}, rs{0}, np, sl, ss{0}, wo, wb{0};
+  int wsum = 0;
   for (int i : lst) {
     const MatDev& mt = c->mats[i];
     if (mt.Gs) { sl.push_back(i); ss.push_back(ss.back() + mt.m); }
@@ -397,6 +435,8 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
     cs.push_back(cs.back() + cb);
     rs.push_back(rs.back() + mt.l);
     np.push_back(cb);
+    wo.push_back(wsum); wsum += mt.r;
+    wb.push_back(wb.back() + (mt.r + 127) / 128);
   }
   auto push_block = [&](const std::vector<int>& v) {
     size_t o = ints.size();
@@ -405,7 +445,8 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
   };
   const size_t o_list = push_block(lst), o_k1 = push_block(k1), o_k2 = push_block(k2),
                o_cs = push_block(cs), o_rs = push_block(rs), o_np = push_block(np),
-               o_sl = push_block(sl), o_ss = push_block(ss);
+               o_sl = push_block(sl), o_ss = push_block(ss), o_wo = push_block(wo), o_wb = push_block(wb);
+  pl->wq_off = c->ints_dev + o_wo; pl->wq_blk = c->ints_dev + o_wb; pl->wq_blocks = wb.back();
   pl->list = c->ints_dev + o_list; pl->nlist = (int)lst.size();
   pl->k1_start = c->ints_dev + o_k1; pl->k1_tiles = k1.back();
   pl->k2_start = c->ints_dev + o_k2; pl->k2_tiles = k2.back();
@@ -414,12 +455,14 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
   pl->npart = c->ints_dev + o_np;
   pl->stage_list = c->ints_dev + o_sl; pl->stage_start = c->ints_dev + o_ss;
   pl->nstage = (int)sl.size(); pl->stage_rows = ss.back();
+  pl->h_k1 = k1; pl->h_k2 = k2; pl->h_cs = cs; pl->h_rs = rs; pl->h_sl = sl; pl->h_ss = ss;
   pl->maps.resize(lst.size());
   char* tab = c->tc_maps_dev;
   pl->maps_dev = reinterpret_cast<TcMaps*>(tab); tab += align_up(sizeof(TcMaps) * lst.size());
   pl->fast_dev = reinterpret_cast<float*>(tab); tab += align_up(2 * sizeof(float) * lst.size());
   pl->td2_dev = reinterpret_cast<BackTileDesc*>(tab); tab += align_up(sizeof(BackTileDesc) * (size_t)pl->k2_tiles);
-  pl->td1_dev = reinterpret_cast<ProjTileDesc*>(tab);
+  pl->td1_dev = reinterpret_cast<ProjTileDesc*>(tab); tab += align_up(sizeof(ProjTileDesc) * (size_t)pl->k1_tiles);
+  pl->wq_dev = reinterpret_cast<float*>(tab);
   {
     std::vector<BackTileDesc> td;
     td.reserve(pl->k2_tiles);
@@ -564,7 +607,7 @@ fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntile
   const ProjTileDesc* tiles = reinterpret_cast<const ProjTileDesc*>(table_dev + align_up(sizeof(TcMaps) * (size_t)njobs));
   Hyper hp{};
   k_tc_project<EPI_PLAIN, PSI_ADAM><<<2 * std::min(ntiles, num_sms / 2), K1_THREADS, K1_SMEM_BYTES, c->stream>>>(
-      maps, tiles, ntiles, nullptr, hp, c->status_dev);
+      maps, tiles, ntiles, nullptr, nullptr, nullptr, hp, c->status_dev);
   return FIRA_OK;
 }
 
@@ -582,7 +625,7 @@ int tc_phase_names(const char** out) {
   return 8;
 }
 
-int launch_tc_step(fira_ctx* c, const Hyper& hp) {
+int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
   TcPlan* pl = c->tc;
   if (!pl || pl->nlist == 0) return 0;
   cudaStream_t st = c->stream;
@@ -597,46 +640,67 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp) {
     }
     pl->attrs_set = true;
   }
+  // the sub-range [qa, qb) of the list (qb < 0: all of it): first tile / block / row of every kernel
+  // and their counts from the host copies of the prefix arrays
+  if (qb < 0) { qa = 0; qb = pl->nlist; }
+  if (qa >= qb) return 0;
+  const int nq = qb - qa;
+  const int k1a = pl->h_k1[qa], k1n = pl->h_k1[qb] - k1a;
+  const int k2a = pl->h_k2[qa], k2n = pl->h_k2[qb] - k2a;
+  const int csa = pl->h_cs[qa], csn = pl->h_cs[qb] - csa;
+  const int rsa = pl->h_rs[qa], rsb = pl->h_rs[qb];
+  // staged matrices (a subset of the list, both ascending) that fall into the range
+  int sa = 0, sb = 0;
+  for (int q = 0; q < pl->nstage; ++q) {
+    if (pl->h_sl[q] < c->tc_list[qa]) ++sa;
+    if (pl->h_sl[q] <= c->tc_list[qb - 1]) ++sb;
+  }
+  const int sra = pl->nstage ? pl->h_ss[sa] : 0, srn = pl->nstage ? pl->h_ss[sb] - sra : 0;
   PhaseTimer* tm = &c->timer;
   const MatDev* mats = c->mats_dev;
-  if (pl->nstage) k_tc_stage<<<pl->stage_rows, 256, 0, st>>>(mats, pl->stage_list, pl->nstage, pl->stage_start, 0);
+  if (c->proj_weights_dirty) {        // the stored projection has changed since the weights were taken
+    k_tc_proj_weights<<<pl->wq_blocks, 256, 0, st>>>(mats, pl->list, pl->wq_off, pl->wq_blk, pl->nlist, pl->wq_dev);
+    c->proj_weights_dirty = false;
+  }
+  if (srn) k_tc_stage<<<srn, 256, 0, st>>>(mats, pl->stage_list, pl->nstage, pl->stage_start, sra, 0);
   tm->mark(st);
-  k_tc_prep<<<(pl->nlist + 127) / 128, 128, 0, st>>>(mats, pl->list, pl->nlist, hp, pl->fast_dev);
+  k_tc_prep<<<(nq + 127) / 128, 128, 0, st>>>(mats, pl->list, qa, qb, hp, pl->fast_dev);
   tm->mark(st);
   // both tensor kernels: clusters of two CTAs, at most one CTA per SM
-  const int k1_grid = 2 * std::min(pl->k1_tiles, pl->num_sms / 2);
+  const int k1_grid = 2 * std::min(k1n, pl->num_sms / 2);
+  const ProjTileDesc* td1 = pl->td1_dev + k1a;
   if (hp.mode & HYPER_PSI_RMSPROP)
     k_tc_project<EPI_ADAM, PSI_RMSPROP><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(
-        pl->maps_dev, pl->td1_dev, pl->k1_tiles, pl->fast_dev, hp, c->status_dev);
+        pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev);
   else if (hp.mode & HYPER_PSI_ADAGRAD)
     k_tc_project<EPI_ADAM, PSI_ADAGRAD><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(
-        pl->maps_dev, pl->td1_dev, pl->k1_tiles, pl->fast_dev, hp, c->status_dev);
+        pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev);
   else
     k_tc_project<EPI_ADAM, PSI_ADAM><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(
-        pl->maps_dev, pl->td1_dev, pl->k1_tiles, pl->fast_dev, hp, c->status_dev);
+        pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev);
   tm->mark(st);
-  k_tc_colfactors<<<pl->col_blocks, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->col_start, hp);
+  k_tc_colfactors<<<csn, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->col_start, csa, hp);
   tm->mark(st);
-  k_finalize<<<pl->nlist, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->npart, hp, c->status_dev);
+  k_finalize<<<nq, 256, 0, st>>>(mats, pl->list + qa, nq, pl->npart + qa, hp, c->status_dev);
   tm->mark(st);
   if (hp.mode & HYPER_ONLY_SCALING) {
     // W <- W - lr phi(R) G: no back-projection; the element-wise update works on the caller's W and
     // G in place (whatever their pitch), so nothing is copied back from the aligned copies
     tm->mark(st);
-    launch_scaled_gradient(mats, pl->list, pl->nlist, pl->k2_start, pl->k2_tiles, 2 * BM, 1, hp.lr, hp.a_res, st);
+    launch_scaled_gradient(mats, pl->list, pl->nlist, pl->k2_start, k2a, k2n, 2 * BM, 1, hp.lr, hp.a_res, st);
     tm->mark(st);
     tm->mark(st);
-    return pl->nstage ? 6 : 5;
+    return srn ? 6 : 5;
   }
-  k_tc_form_x<<<(pl->rows_total + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start,
-                                                        pl->rows_total, hp.a_low, hp.a_res, pl->fast_dev);
+  k_tc_form_x<<<(rsb - rsa + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start, rsa, rsb,
+                                                   hp.a_low, hp.a_res, pl->fast_dev);
   tm->mark(st);
-  k_tc_back_project<<<2 * std::min(pl->k2_tiles, pl->num_sms / 2), K2_THREADS, K2_SMEM_BYTES, st>>>(
-      pl->maps_dev, pl->td2_dev, pl->k2_tiles, pl->fast_dev, hp, c->status_dev);
+  k_tc_back_project<<<2 * std::min(k2n, pl->num_sms / 2), K2_THREADS, K2_SMEM_BYTES, st>>>(
+      pl->maps_dev, pl->td2_dev + k2a, k2n, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);
-  if (pl->nstage) k_tc_stage<<<pl->stage_rows, 256, 0, st>>>(mats, pl->stage_list, pl->nstage, pl->stage_start, 1);
+  if (srn) k_tc_stage<<<srn, 256, 0, st>>>(mats, pl->stage_list, pl->nstage, pl->stage_start, sra, 1);
   tm->mark(st);
-  return pl->nstage ? 8 : 6;
+  return srn ? 8 : 6;
 }
 
 }  // namespace fira

@@ -26,9 +26,9 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints);
 void tc_destroy_plan(fira_ctx* c);
 // Called when W / G pointers changed: re-encodes what depends on them.
 fira_status tc_update_pointers(fira_ctx* c);
-// Enqueues the tensor-core phases for the matrices of the tc list; returns the
-// number of launches (negative: error, message set).
-int launch_tc_step(fira_ctx* c, const Hyper& hp);
+// Enqueues the tensor-core phases for the matrices [qa, qb) of the tc list (qb < 0: all of it);
+// returns the number of launches (negative: error, message set).
+int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa = 0, int qb = -1);
 // Launches the self-test kernel of the bounded waits (one block; sets the time-out bit of the
 // context's status word after `rounds` tries on a barrier that nothing arrives on).
 fira_status tc_selftest_bounded_wait(fira_ctx* c, int rounds);

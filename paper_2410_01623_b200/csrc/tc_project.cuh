@@ -3,8 +3,10 @@
 //
 //   Rt[l][j] = sum_d G(d,l) Pi[d][j]          (R = P^T G, stored with the rank index contiguous)
 //   M <- b1 M + (1-b1) R,  V <- b2 V + (1-b2) R^2,  N = bias M / (sqrt V + eps)     (Eq. 2-4)
-//   writes M, V (fp32), N, R (bf16), the per-l partial sums ||N_l||^2, ||R_l||^2 and, from the
-//   tiles of the first r range, the per-l sums ||G_l||^2 (needed for ||S||)
+//   writes M, V (fp32), N, R (bf16), the per-l partial sums ||N_l||^2, ||R_l||^2 and
+//   sum_j w_j R_lj^2 with w_j = 2 - ||pi_j||^2 (pi_j = column j of the stored projection), and the
+//   per-l sums ||G_l||^2: together they give ||S_l||^2 = ||G_l||^2 - sum_j w_j R_lj^2, which is
+//   ||G_l - Pi R_l||^2 up to the off-diagonal part of Pi^T Pi - I
 //
 // CTA pairs (clusters of two, one CTA per SM) walk tiles of 256 l x BN r with
 // tcgen05.mma.cta_group::2.  A = G: for m <= n an MN-major operand (G is [d][l], l
@@ -123,7 +125,8 @@ enum { PSI_ADAM = 0, PSI_RMSPROP = 1, PSI_ADAGRAD = 2 };
 template <int EPI, int PSI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(K1_THREADS, 1)
 k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ tdesc, int total_tiles,
-             const float* __restrict__ fast, Hyper hp, unsigned* __restrict__ status) {
+             const float* __restrict__ fast, const float* __restrict__ wq_all, const int* __restrict__ wq_off,
+             Hyper hp, unsigned* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* tiles = smem_raw;
   unsigned char* mvbuf = tiles + (size_t)K1_STAGES * K1_STAGE_BYTES;
@@ -433,12 +436,13 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
       const int bn = d.bn_left & 0xffff;
       const int l = d.l0 + BM * (int)rank + row;
       const float bias = EPI == EPI_ADAM ? fast[2 * d.slot] : 0.f;
+      const float* wrow = EPI == EPI_ADAM ? wq_all + wq_off[d.slot] + d.r0 : nullptr;   // weights of this tile's rank range
       if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->tmem_full[buf]), bphase, abort_flag)) break;
       ptx::tc_fence_after();
       const uint32_t tcol = tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX;
       const uint32_t te = buf ? tmem_empty1 : tmem_empty0;
       const int nch = bn / K1_ECOLS;
-      float nn = 0.f, rn = 0.f;
+      float nn = 0.f, rn = 0.f, rw = 0.f;
       for (int c = 0; c < nch; ++c) {
         uint32_t rr[32];
         __syncwarp();
@@ -470,6 +474,9 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           const float4 v1 = *reinterpret_cast<const float4*>(vb + f1);
           float mo[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
           float vo[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+          const float4 w0 = __ldg(reinterpret_cast<const float4*>(wrow + K1_ECOLS * c + 8 * q));      // same for every lane
+          const float4 w1 = __ldg(reinterpret_cast<const float4*>(wrow + K1_ECOLS * c + 8 * q + 4));
+          const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
           float rv[8], nv[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
@@ -484,6 +491,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
             }
             nn = fmaf(nv[e], nv[e], nn);
             rn = fmaf(rv[e], rv[e], rn);
+            rw = fmaf(wv[e] * rv[e], rv[e], rw);
           }
           *reinterpret_cast<float4*>(mb + f0) = make_float4(mo[0], mo[1], mo[2], mo[3]);
           *reinterpret_cast<float4*>(mb + f1) = make_float4(mo[4], mo[5], mo[6], mo[7]);
@@ -504,10 +512,12 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         if (++mvuse == K1_MVBUFS) { mvuse = 0; mvphase ^= 1u; }
       }
       if (EPI == EPI_ADAM && ok && l < d.L) {
-        // colpart[2 part][l] = partial ||N_l||^2, colpart[2 part + 1][l] = partial ||R_l||^2
-        const int part = d.r0 / bn;
+        // colpart[2 part][l] = partial ||N_l||^2, colpart[2 part + 1][l] = partial ||R_l||^2; after the
+        // sums of G^2: colpart[(2 + K1_GSQ_SPLIT) nparts + part][l] = partial sum_j w_j R_lj^2
+        const int part = d.r0 / bn, nparts = (d.bn_left >> 16) & 0xff;
         d.colpart[(long long)(2 * part) * d.L + l] = nn;
         d.colpart[(long long)(2 * part + 1) * d.L + l] = rn;
+        d.colpart[(long long)((2 + K1_GSQ_SPLIT) * nparts + part) * d.L + l] = rw;
       }
       if (++buf == 2) { buf = 0; bphase ^= 1u; }
     }

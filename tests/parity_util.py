@@ -22,24 +22,30 @@ TOL_W = {"f32": 1e-5, "bf16": 2e-2}
 # flips of W.
 TOL_DW = {"f32": 2e-4, "bf16": 3e-2}
 # A Frobenius ratio over a whole matrix cannot see one wrong column, row or tile, so three local
-# measures are bounded as well (derivations in the design notes; all on the accumulated update
-# dW = W_t - W_0 or on single elements of W):
-#  * col / row: the largest error norm of any one COLUMN (ROW) of dW relative to that column's (row's)
-#    own norm, the denominator floored at half the median column (row) norm.  The floor is there
-#    because the error of the bf16 path is absolute: the rank-r operand X of the back-projection is
-#    rounded to bf16, which puts about 2^-9 of the typical size of (Pi X) into every element of W,
-#    however small the exact update of a particular column may be (a gradient column of tiny scale
-#    in the right orientation, say).  Measured: median 6e-3, worst 2e-2 per column over 100 steps.
-#  * fp32: elem = the largest |W_gpu - W_oracle| over all elements, relative to max |W|.
-#  * bf16: elem = the largest of |W_gpu - W_oracle| / (U(t) ulp + 0.1 s) over all elements, which
-#    must stay below 1.  ulp is one bf16 spacing at the largest magnitude the element has had so far;
-#    after one step the two sides round nearly equal numbers and differ by one spacing at most (two
-#    across a binade boundary), and over t steps the difference performs a lazy random walk (about
-#    one element in ten moves per step), hence U(t) = 2 + 1.5 sqrt(t - 1).  s is the rms size of the
-#    update in the element's column or row (the larger; floored as above): an element may be off by
-#    a tenth of that (the arithmetic error of one element is about 1 % of s, the maximum over 10^7
-#    elements about 6 %), whereas an element of a misplaced or stale tile is off by about s itself.
-TOL_COL = {"f32": 5e-4, "bf16": 5e-2}
+# measures are bounded as well, each as a ratio (error / allowance) that must stay below 1; all are
+# taken on the accumulated update dW = W_t - W_0 or on single elements of W.  Two effects make up the
+# allowance on the bf16 path:
+#   (a) arithmetic: the rank-r operand X of the back-projection (and N, R before it) is rounded to
+#       bf16, which puts an error of about 2^-9 of the typical size of (Pi X) into every element of
+#       W, however small the exact update of a particular column may be (so norms of columns and
+#       rows of dW are floored at half their median).  Measured: 0.6 % of a column's norm (median),
+#       2 % (worst column over 100 steps);
+#   (b) storage: W is rounded to bf16 once per step on both sides.  After one step the two sides
+#       round nearly equal numbers and differ by one spacing (ulp) at most (two across a binade
+#       boundary), in a few per cent of the elements; over t steps the difference of an element
+#       performs a lazy random walk, so its rms grows like sqrt(t) spacings (measured: about
+#       0.3 sqrt(t)).  The spacing is taken at the largest magnitude the element has had so far.
+#  * col / row: ||err_col|| / (COL_ARITH ||dW_col|| + COL_WALK sqrt(t) ||ulp_col||), largest over the
+#    columns (rows).  A stale or misplaced column has ||err_col|| = ||dW_col||: a ratio of 5 to 30.
+#  * bf16 elem: |err| / (U(t) ulp + ELEM_UPDATE_SHARE s) over all elements, U(t) = 2 + 1.5 sqrt(t - 1)
+#    (the maximum of the walk over 10^7 elements), s the rms size of the update in the element's
+#    column or row (the larger): the arithmetic error of one element is about 1 % of s, its maximum
+#    over 10^7 elements about 6 %, whereas an element of a misplaced or stale tile is off by about s.
+#  * fp32: no storage term; col / row relative to TOL_COL_F32 ||dW_col||; elem = the largest
+#    |W_gpu - W_oracle| relative to max |W|, bounded by TOL_ELEM_F32.
+COL_ARITH = 0.03
+COL_WALK = 0.6
+TOL_COL_F32 = 5e-4
 TOL_ELEM_F32 = 1e-5
 ELEM_UPDATE_SHARE = 0.1
 
@@ -65,25 +71,31 @@ def bf16_ulp(x: np.ndarray) -> np.ndarray:
 
 
 def local_errors(Wg: np.ndarray, Wo: np.ndarray, W0: np.ndarray, wmax: np.ndarray, kind: str, steps: int) -> dict:
-    """Column-, row- and element-wise differences between the library's W and the oracle's (see the
-    bounds above).  wmax is the largest |W| that the oracle has held in each element so far."""
+    """Column-, row- and element-wise differences between the library's W and the oracle's, each
+    divided by its allowance (see above).  wmax is the largest |W| that the oracle has held in each
+    element so far."""
     err = Wg - Wo
     dO = Wo - W0
     e2, d2 = err * err, dO * dO
+    ulp = bf16_ulp(wmax) if kind == "bf16" else None
     out, rms = {}, {}
     for name, ax in (("col", 0), ("row", 1)):
         den = np.sqrt(d2.sum(axis=ax))
         den = np.maximum(den, max(0.5 * float(np.median(den)), 1e-300))
-        out[name] = float((np.sqrt(e2.sum(axis=ax)) / den).max())
         rms[name] = den / math.sqrt(err.shape[ax])
+        if kind == "bf16":
+            allow = COL_ARITH * den + COL_WALK * math.sqrt(steps) * np.sqrt((ulp * ulp).sum(axis=ax))
+        else:
+            allow = TOL_COL_F32 * den
+        out[name] = float((np.sqrt(e2.sum(axis=ax)) / allow).max())
     aerr = np.abs(err)
     if kind == "bf16":
         s = np.maximum(rms["col"][None, :], rms["row"][:, None])
-        out["elem"] = float((aerr / (max_ulp_bound(steps) * bf16_ulp(wmax) + ELEM_UPDATE_SHARE * s)).max())
-        out["ulp"] = float((aerr / bf16_ulp(wmax)).max())
+        out["elem"] = float((aerr / (max_ulp_bound(steps) * ulp + ELEM_UPDATE_SHARE * s)).max())
+        out["ulp"] = float((aerr / ulp).max())
         out["frac_off"] = float(np.count_nonzero(err) / err.size)
     else:
-        out["elem"] = float(aerr.max() / max(float(np.abs(Wo).max()), 1e-300))
+        out["elem"] = float(aerr.max() / max(float(np.abs(Wo).max()), 1e-300)) / TOL_ELEM_F32
     return out
 
 
@@ -215,16 +227,15 @@ class Trajectory:
                 f"row {self.local['row']:.2e} elem {self.local['elem']:.2e} ulp {self.local['ulp']:.2f} "
                 f"off {self.local['frac_off']:.3f} marked {sum(int(v.sum()) for v in self.marked.values())}")
 
-    def assert_ok(self, tol_w=None, tol_dw=None, tol_col=None):
+    def assert_ok(self, tol_w=None, tol_dw=None):
         tol_w = TOL_W[self.kind] if tol_w is None else tol_w
         tol_dw = TOL_DW[self.kind] if tol_dw is None else tol_dw
-        tol_col = TOL_COL[self.kind] if tol_col is None else tol_col
         print("parity:", self.summary())
         assert self.f.poll() == 0
         assert math.isfinite(self.max_w) and self.max_w <= tol_w, (self.max_w, tol_w)
         assert math.isfinite(self.max_dw) and self.max_dw <= tol_dw, (self.max_dw, tol_dw)
-        assert self.local["col"] <= tol_col and self.local["row"] <= tol_col, (self.summary(), tol_col)
-        assert self.local["elem"] <= (TOL_ELEM_F32 if self.kind == "f32" else 1.0), self.summary()
+        # column, row and element errors as fractions of their allowances
+        assert self.local["col"] <= 1.0 and self.local["row"] <= 1.0 and self.local["elem"] <= 1.0, self.summary()
 
 
 def workload_trajectory(wl: wk.Workload, steps: int, device="cuda", gen_device="cpu",
