@@ -23,7 +23,7 @@ TOL_W = {"f32": 1e-5, "bf16": 2e-2}
 TOL_DW = {"f32": 2e-4, "bf16": 3e-2}
 # A Frobenius ratio over a whole matrix cannot see one wrong column, row or tile, so three local
 # measures are bounded as well, each as a ratio (error / allowance) that must stay below 1; all are
-# taken on the accumulated update dW = W_t - W_0 or on single elements of W.  Two effects make up the
+# taken on the accumulated update dW = W_t - W_0 or on single elements of W.  Three effects make up the
 # allowance on the bf16 path:
 #   (a) arithmetic: the rank-r operand X of the back-projection (and N, R before it) is rounded to
 #       bf16, which puts an error of about 2^-9 of the typical size of (Pi X) into every element of
@@ -35,9 +35,21 @@ TOL_DW = {"f32": 2e-4, "bf16": 3e-2}
 #       boundary), in a few per cent of the elements; over t steps the difference of an element
 #       performs a lazy random walk, so its rms grows like sqrt(t) spacings (measured: about
 #       0.3 sqrt(t)).  The spacing is taken at the largest magnitude the element has had so far.
-#  * col / row: ||err_col|| / (COL_ARITH ||dW_col|| + COL_WALK sqrt(t) ||ulp_col||), largest over the
+#   (c) large entries of the rank-r operand: the rounding error of X[l][q] is proportional to
+#       |X[l][q]| (and to |N|, |R|, rounded before it), not to the size of the net update.  Where the
+#       projection has a column concentrated on one coordinate d (a gradient with a few dominant
+#       columns gives such a basis) the terms k_l R_lq Pi_dq and k_l G_dl of the update nearly cancel,
+#       so X[l][q] is many times larger than the element's update and its rounding error is no
+#       longer a small share of s.  The allowance therefore carries the error model of the three
+#       roundings: per step, var(dW[d][l]) = lr^2 (2^-9)^2 / 3 * sum_q Pi_dq^2 ((a N_lq)^2 +
+#       (c_l R_lq)^2 + X_lq^2) with c_l = a lambda k_l, summed over the steps (independent roundings)
+#       into A[d][l] from the ORACLE's N, R, k, lambda; an element may be off by ELEM_MODEL_SIGMAS
+#       standard deviations sqrt(A) (the maximum of 10^7 to 10^8 samples), a column or row by
+#       LINE_MODEL_SIGMAS times the root of its summed variance.  On matrices without such entries
+#       this term is a few per cent of the others.
+#  * col / row: ||err_col|| / (COL_ARITH ||dW_col|| + COL_WALK sqrt(t) ||ulp_col|| + the (c) term), largest over the
 #    columns (rows).  A stale or misplaced column has ||err_col|| = ||dW_col||: a ratio of 5 to 30.
-#  * bf16 elem: |err| / (U(t) ulp + ELEM_UPDATE_SHARE s) over all elements, U(t) = 2 + 1.5 sqrt(t - 1)
+#  * bf16 elem: |err| / (U(t) ulp + ELEM_UPDATE_SHARE s + the (c) term) over all elements, U(t) = 2 + 1.5 sqrt(t - 1)
 #    (the maximum of the walk over 10^7 elements), s the rms size of the update in the element's
 #    column or row (the larger): the arithmetic error of one element is about 1 % of s, its maximum
 #    over 10^7 elements about 6 %, whereas an element of a misplaced or stale tile is off by about s.
@@ -48,6 +60,9 @@ COL_WALK = 0.6
 TOL_COL_F32 = 5e-4
 TOL_ELEM_F32 = 1e-5
 ELEM_UPDATE_SHARE = 0.1
+ELEM_MODEL_SIGMAS = 6.0
+LINE_MODEL_SIGMAS = 3.0
+BF16_REL_VAR = (2.0 ** -9) ** 2 / 3.0
 
 
 def max_ulp_bound(steps: int) -> float:
@@ -70,10 +85,12 @@ def bf16_ulp(x: np.ndarray) -> np.ndarray:
     return np.exp2(e - 7.0)
 
 
-def local_errors(Wg: np.ndarray, Wo: np.ndarray, W0: np.ndarray, wmax: np.ndarray, kind: str, steps: int) -> dict:
+def local_errors(Wg: np.ndarray, Wo: np.ndarray, W0: np.ndarray, wmax: np.ndarray, kind: str, steps: int,
+                 var: Optional[np.ndarray] = None, flip: Optional[np.ndarray] = None) -> dict:
     """Column-, row- and element-wise differences between the library's W and the oracle's, each
     divided by its allowance (see above).  wmax is the largest |W| that the oracle has held in each
-    element so far."""
+    element so far; var (bf16) the accumulated variance A of the operand roundings per element; flip
+    (bf16) the accumulated bound F of the changes of ill-conditioned direction elements."""
     err = Wg - Wo
     dO = Wo - W0
     e2, d2 = err * err, dO * dO
@@ -85,13 +102,22 @@ def local_errors(Wg: np.ndarray, Wo: np.ndarray, W0: np.ndarray, wmax: np.ndarra
         rms[name] = den / math.sqrt(err.shape[ax])
         if kind == "bf16":
             allow = COL_ARITH * den + COL_WALK * math.sqrt(steps) * np.sqrt((ulp * ulp).sum(axis=ax))
+            if var is not None:
+                allow = allow + LINE_MODEL_SIGMAS * np.sqrt(var.sum(axis=ax))
+            if flip is not None:
+                allow = allow + np.sqrt((flip.astype(np.float64) ** 2).sum(axis=ax))
         else:
             allow = TOL_COL_F32 * den
         out[name] = float((np.sqrt(e2.sum(axis=ax)) / allow).max())
     aerr = np.abs(err)
     if kind == "bf16":
         s = np.maximum(rms["col"][None, :], rms["row"][:, None])
-        out["elem"] = float((aerr / (max_ulp_bound(steps) * ulp + ELEM_UPDATE_SHARE * s)).max())
+        allow = max_ulp_bound(steps) * ulp + ELEM_UPDATE_SHARE * s
+        if var is not None:
+            allow = allow + ELEM_MODEL_SIGMAS * np.sqrt(var)
+        if flip is not None:
+            allow = allow + flip
+        out["elem"] = float((aerr / allow).max())
         out["ulp"] = float((aerr / ulp).max())
         out["frac_off"] = float(np.count_nonzero(err) / err.size)
     else:
@@ -109,24 +135,78 @@ def local_errors(Wg: np.ndarray, Wo: np.ndarray, W0: np.ndarray, wmax: np.ndarra
 # nothing else.  The fp32 bounds (1e-5 on W) leave no room for a single such element, so the fp32
 # comparisons leave out the unprojected indices l for which the ORACLE's own numbers predict an error
 # of N above N_ERR_MARK; how many were left out is bounded and what happened in them is checked for
-# plausibility separately.  (bf16 runs have bounds far above this effect and mark nothing.)
-N_ERR_MARK = 5e-3
-FP32_DOT_ERR = 2.0 ** -23
+# plausibility separately.
+# The tensor-core path has the same property (bf16 operands multiply exactly, the sums are fp32; the
+# measured error of its R is about 2^-22 ||G_l|| at d = 4096, taken as 2^-20 here).  Its Frobenius
+# bounds are far above the effect, but one changed direction element (q, l) moves element (d, l) of W
+# by lr a dN |Pi_dq|, which the element bound sees where r is small or the projection has large
+# entries.  Nothing is left out of the bf16 comparisons; instead the allowances carry that term: for
+# every element of N that the oracle's numbers show to be changeable (adam_direction_changes) the bound
+# lr a dN |Pi_dq| is added to the allowance F[d][l] of the elements of line l, for good (W carries the
+# difference forward; M and V do not: R is tiny there).  Lines are allowed the norm of their F entries.
+N_ERR_MARK = {"f32": 5e-3, "bf16": 2e-2}
+DOT_ERR = {"f32": 2.0 ** -23, "bf16": 2.0 ** -20}
 
 
-def adam_sensitive_indices(R, G_l_norm, M0, V0, st_t_before: int, ohp: fo.Hyper) -> np.ndarray:
-    """Boolean mask over the unprojected index l: True where |dN/dR| times the fp32 error of R
-    exceeds N_ERR_MARK for some rank index.  R, M0, V0 are r x l (the oracle's orientation); M0, V0 are
-    the moments BEFORE the step, st_t_before the steps taken before it."""
+def adam_direction_changes(R, G_l_norm, M0, V0, st_t_before: int, ohp: fo.Hyper, kind: str = "f32"):
+    """The elements (q, l) of N that an error of the computed R of the size DOT_ERR ||G_l|| can change
+    by more than a tenth of N_ERR_MARK, with the largest such change dN.  The change is evaluated, not
+    linearised (N jumps by up to 2 where R crosses zero within that error), at the elements where the
+    closeness of R to zero makes it possible at all.  R, M0, V0 are r x l (the
+    oracle's orientation); M0, V0 are the moments BEFORE the step, st_t_before the steps taken before
+    it.  Returns (q indices, l indices, dN)."""
     s = st_t_before + 1
     b = math.sqrt(1.0 - ohp.beta2 ** s) / (1.0 - ohp.beta1 ** s)
-    M = ohp.beta1 * M0 + (1.0 - ohp.beta1) * R
-    V = ohp.beta2 * V0 + (1.0 - ohp.beta2) * R * R
-    rt = np.sqrt(V)
-    den = rt + ohp.eps
-    second = np.divide(M * (1.0 - ohp.beta2) * R, rt * den * den, out=np.zeros_like(R), where=rt > 0)
-    dNdR = np.abs(b * ((1.0 - ohp.beta1) / den - second))
-    return (dNdR * (FP32_DOT_ERR * G_l_norm)[None, :]).max(axis=0) > N_ERR_MARK
+    err_l = DOT_ERR[kind] * G_l_norm
+    thr = 0.1 * N_ERR_MARK[kind]
+
+    def direction(Rx, M0x, V0x):
+        M = ohp.beta1 * M0x + (1.0 - ohp.beta1) * Rx
+        V = ohp.beta2 * V0x + (1.0 - ohp.beta2) * Rx * Rx
+        return b * M / (np.sqrt(V) + ohp.eps)
+
+    # N can be steep in R only where R itself is small (next to its own error, or next to what the
+    # moments remember of earlier small values): everything else is left out before the evaluation
+    cand = np.abs(R) < (512.0 * err_l)[None, :]
+    qs, ls = np.nonzero(cand)
+    if qs.size == 0:
+        return qs, ls, np.zeros(0)
+    Rc, Mc, Vc, ec = R[cand], M0[cand], V0[cand], err_l[ls]
+    n0 = direction(Rc, Mc, Vc)
+    dn = np.maximum(np.abs(direction(Rc + ec, Mc, Vc) - n0), np.abs(direction(Rc - ec, Mc, Vc) - n0))
+    keep = dn > thr
+    return qs[keep], ls[keep], dn[keep]
+
+
+def adam_sensitive_indices(R, G_l_norm, M0, V0, st_t_before: int, ohp: fo.Hyper, kind: str = "f32") -> np.ndarray:
+    """Boolean mask over the unprojected index l: True where some element of N can change by more than
+    N_ERR_MARK (see adam_direction_changes)."""
+    _, ls, dn = adam_direction_changes(R, G_l_norm, M0, V0, st_t_before, ohp, kind)
+    out = np.zeros(R.shape[1], dtype=bool)
+    out[np.unique(ls[dn > N_ERR_MARK[kind]])] = True
+    return out
+
+
+def rounding_variance(proj: np.ndarray, d: dict, ohp: fo.Hyper, left: bool) -> torch.Tensor:
+    """One step's variance of the error that the bf16 roundings of N, R and X = a N - c_l R put into
+    every element of W (in W's orientation, float32): lr^2 (2^-9)^2 / 3 * Pi^2 (a^2 N^2 + c^2 R^2 + X^2)
+    with the oracle's N, R (r x l), k and lambda of that step.  This allowance (a bound, not an
+    expected value) is formed with the tensor library, on the device when there is one: its one large
+    product (d x r by r x l) would otherwise cost as much as a product of the oracle itself."""
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    N = torch.from_numpy(d["N"].astype(np.float32)).to(dev)
+    R = torch.from_numpy(d["R"].astype(np.float32)).to(dev)
+    a_low = float(ohp.alpha)
+    if ohp.residual:
+        c = torch.from_numpy(((1.0 if ohp.alpha_lowrank_only else ohp.alpha) * d["lam"] * d["k"]).astype(np.float32)).to(dev)
+        cR = R * c[None, :]
+    else:
+        cR = torch.zeros_like(R)
+    aN = a_low * N
+    Y2 = aN * aN + cR * cR + (aN - cR) ** 2
+    P2 = torch.from_numpy((proj * proj).astype(np.float32)).to(dev)
+    v = (P2 @ Y2) * float(ohp.lr ** 2 * BF16_REL_VAR)                      # d x l
+    return v if left else v.T.contiguous()
 
 
 def oracle_hyper(hp: fb.Hparams) -> fo.Hyper:
@@ -164,6 +244,10 @@ class Trajectory:
         # some step (see adam_sensitive_indices); sticky, since W carries the difference forward
         self.marked = {i: np.zeros(max(self.shapes[i]), dtype=bool) for i in self.check}
         self.wmax = {i: np.abs(self.W0[i]) for i in self.check}     # largest |W| seen per element (oracle)
+        # bf16: accumulated variance of the operand roundings per element of W (see (c) above)
+        self.var = {}                                              # (device tensors, created on the first step)
+        # bf16: accumulated bound of the changes of ill-conditioned direction elements per element of W
+        self.flip = {i: np.zeros(self.shapes[i], dtype=np.float32) for i in self.check} if self.kind == "bf16" else {}
         self.lams: List[List[float]] = []
 
     def oracle_projection(self, i):
@@ -184,7 +268,7 @@ class Trajectory:
             Wprev = self.Wo[i]
             m, n = self.shapes[i]
             left = m <= n
-            track = self.kind == "f32" and ohp.psi == "adam"
+            track = ohp.psi == "adam" and not ohp.only_scaling
             if track:
                 st = self.st[i]
                 M0, V0, t0 = (st.M.copy(), st.V.copy(), st.t) if left else (st.M.T.copy(), st.V.T.copy(), st.t)
@@ -194,18 +278,30 @@ class Trajectory:
             self.wmax[i] = np.maximum(self.wmax[i], np.abs(self.Wo[i]))
             if track:
                 gn = np.sqrt((G64 * G64).sum(axis=0 if left else 1))
-                self.marked[i] |= adam_sensitive_indices(d["R"], gn, M0, V0, t0, ohp)
+                if self.kind == "f32":
+                    self.marked[i] |= adam_sensitive_indices(d["R"], gn, M0, V0, t0, ohp, self.kind)
+                else:
+                    qs, ls, dn = adam_direction_changes(d["R"], gn, M0, V0, t0, ohp, self.kind)
+                    F = self.flip[i] if left else self.flip[i].T          # d x l view
+                    for q, l, x in zip(qs, ls, dn):
+                        F[:, l] += np.float32(ohp.lr * ohp.alpha * x) * np.abs(projs[i][:, q]).astype(np.float32)
+            if self.kind == "bf16" and not ohp.only_scaling:
+                v = rounding_variance(projs[i], d, ohp, left)
+                self.var[i] = v if i not in self.var else self.var[i] + v
             if compare:
                 Wg = to_np64(self.W[i])
-                Wo, W0, wmax = self.Wo[i], self.W0[i], self.wmax[i]
+                Wo, W0, wmax, flip = self.Wo[i], self.W0[i], self.wmax[i], self.flip.get(i)
+                var = self.var[i].cpu().numpy() if i in self.var else None
                 if self.marked[i].any():
                     keep = ~self.marked[i]
                     self.check_marked(i, Wg, Wo, W0, left)
                     sel = (slice(None), keep) if left else (keep, slice(None))
                     Wg, Wo, W0, wmax = Wg[sel], Wo[sel], W0[sel], wmax[sel]
+                    var = None if var is None else var[sel]
+                    flip = None if flip is None else flip[sel]
                 self.max_w = max(self.max_w, rel_err(Wg, Wo))
                 self.max_dw = max(self.max_dw, rel_err(Wg - W0, Wo - W0))
-                for k, v in local_errors(Wg, Wo, W0, wmax, self.kind, self.nsteps).items():
+                for k, v in local_errors(Wg, Wo, W0, wmax, self.kind, self.nsteps, var, flip).items():
                     self.local[k] = max(self.local[k], v)
         self.lams.append(lam_row)
         return lam_row

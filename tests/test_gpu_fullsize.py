@@ -15,13 +15,14 @@ pytestmark = pytest.mark.gpu
 def test_llama_7b_layer_two_steps():
     wl = wk.workload("llama-7b", layers=1)
     assert wl.shapes[0] == (4096, 4096) and wl.shapes[4] == (4096, 11008) and wl.shapes[6] == (11008, 4096)
-    tr = workload_trajectory(wl, 2, gen_device="cuda", check=[0, 4, 6])
+    # two steps with seeded orthonormal projections; the right-orientation matrix is compared (the
+    # 50-step run of the same layer in test_gpu_configs.py compares all three shapes)
+    tr = workload_trajectory(wl, 2, gen_device="cuda", check=[6])
     assert [tr.f.diagnostics(i)["engine"] for i in range(7)] == [1] * 7
     tr.assert_ok()
-    for i in (0, 4, 6):
-        d = tr.f.diagnostics(i)
-        assert d["t"] == 2
-        assert d["norm_prev"] == pytest.approx(tr.st[i].prev_norm, rel=2e-2)
+    d = tr.f.diagnostics(6)
+    assert d["t"] == 2
+    assert d["norm_prev"] == pytest.approx(tr.st[6].prev_norm, rel=2e-2)
 
 
 def test_llama_1b_layer_odd_width_on_tensor_cores():
