@@ -10,7 +10,9 @@
 //                      ||G_l||^2 from the A stages in shared memory             (for ||S||)
 //   k_tc_colfactors    k_l (Eq. 11) and partial sums of ||S||^2 = sum_l k_l^2 (||G_l||^2 - ||R_l||^2)
 //   k_finalize         lambda, ||S_prev||, t (Eq. 12)
-//   k_tc_form_x        X = a_low N - a_res lambda k_l R  (bf16)
+//   k_tc_form_x        X = a_low N - a_res lambda k_l R  (bf16).  In the plain step the projection
+//                      epilogue has written X for lambda = 1 already (see tc_project.cuh) and this
+//                      kernel only touches the matrices whose limiter acted: X += a_res (1 - lambda) k_l R
 //   k_tc_back_project  D = Pi X on the tensor cores; epilogue: W -= lr (D + a_res lambda k_l G)
 //
 // ||S_l||^2 = ||G_l - Pi R_l||^2 = ||G_l||^2 - 2 ||R_l||^2 + R_l^T (Pi^T Pi) R_l.  For orthonormal
@@ -59,6 +61,7 @@ struct TcMaps {
   CUtensorMap ev;    // V [l][r] fp32, same
   CUtensorMap en;    // N [l][r] bf16, box 32 x 64, 64-byte swizzle (stored)
   CUtensorMap er;    // R [l][r] bf16, same
+  CUtensorMap ex;    // X [l][r] bf16, same (stored by the projection epilogue when it forms X itself)
 };
 static_assert(sizeof(TcMaps) % 64 == 0, "tensor maps must stay 64-byte aligned");
 
@@ -110,15 +113,22 @@ k_tc_proj_weights(const MatDev* __restrict__ mats, const int* __restrict__ list,
   if (half == 0 && j < mt.r) wq_all[wq_off[p] + j] = 2.f - (part[threadIdx.x] + part[threadIdx.x + 128]);
 }
 
-__global__ void k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict__ list, int first, int nlist, Hyper hp,
-                          float* __restrict__ fast) {
-  const int p = first + blockIdx.x * blockDim.x + threadIdx.x;
-  if (p >= nlist) return;
+__global__ void __launch_bounds__(32)
+k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict__ list, int first, Hyper hp, float* __restrict__ fast) {
+  const int p = first + blockIdx.x;            // one warp per matrix
   const MatDev& mt = mats[list[p]];
-  const double s = (double)(mt.sc->t + 1);
-  const float bias = (float)(sqrt(1.0 - pow((double)hp.beta2, s)) / (1.0 - pow((double)hp.beta1, s)));
-  mt.sc->pad = bias;
-  fast[2 * p] = bias;          // read by the projection epilogue
+  if (threadIdx.x == 0) {
+    const double s = (double)(mt.sc->t + 1);
+    const float bias = (float)(sqrt(1.0 - pow((double)hp.beta2, s)) / (1.0 - pow((double)hp.beta1, s)));
+    mt.sc->pad = bias;
+    fast[2 * p] = bias;          // read by the projection epilogue
+  }
+  // the counters through which the projection epilogues of a row of tiles tell one another that
+  // their partial sums are in place (behind the partial sums; see tc_colpart_floats)
+  const int nparts = mt.r / tile_bn(mt.r);
+  unsigned* cnt = reinterpret_cast<unsigned*>(mt.colpart + (long long)(3 + K1_GSQ_SPLIT) * nparts * mt.l);
+  const int ncnt = 8 * ((mt.l + 2 * BM - 1) / (2 * BM));
+  for (int i = threadIdx.x; i < ncnt; i += 32) cnt[i] = 0u;
 }
 
 // Copies between the caller's G and W and the copies with aligned rows, one block per row of a
@@ -230,7 +240,7 @@ k_tc_colfactors(const MatDev* __restrict__ mats, const int* __restrict__ list, i
 __global__ void __launch_bounds__(256)
 k_tc_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlist,
             const int* __restrict__ row_start, int first_row, int rows_total, float a_low, float a_res,
-            float* __restrict__ fast) {
+            float* __restrict__ fast, int fused) {
   const int lane = threadIdx.x & 31;
   const int row = first_row + blockIdx.x * 8 + (threadIdx.x >> 5);
   if (row >= rows_total) return;
@@ -238,9 +248,10 @@ k_tc_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int n
   const MatDev& mt = mats[list[p]];
   const int l = row - row_start[p];
   const float lambda = mt.sc->lambda;
+  if (fused && mt.d >= FUSE_X_MIN_D) return;           // k_tc_fix_x's matrix
   if (l == 0 && lane == 0) fast[2 * p + 1] = lambda;   // read by the back-projection epilogue
-  const float c = a_res * lambda * mt.kvec[l];
   const long long base = (long long)l * mt.r;
+  const float c = a_res * lambda * mt.kvec[l];
   for (int j = lane * 8; j < mt.r; j += 256) {
     const uint4 nu = *reinterpret_cast<const uint4*>(mt.Nb + base + j);
     const uint4 ru = *reinterpret_cast<const uint4*>(mt.Rb + base + j);
@@ -250,6 +261,34 @@ k_tc_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int n
 #pragma unroll
     for (int e = 0; e < 8; ++e) x[e] = a_low * nv[e] - c * rv[e];
     *reinterpret_cast<uint4*>(mt.Xb + base + j) = pack8_bf16(x);
+  }
+}
+
+// The matrices whose X the projection epilogue has formed for lambda = 1 (FUSE_X): where the limiter
+// acted, X += a_res (1 - lambda) k_l R; the others are left as they are.  blockIdx.y = matrix of the
+// range, the blocks of a matrix stride over its rows, one warp per row.
+__global__ void __launch_bounds__(256)
+k_tc_fix_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int first, float a_res, float* __restrict__ fast) {
+  const int p = first + blockIdx.y;
+  const MatDev& mt = mats[list[p]];
+  if (mt.d < FUSE_X_MIN_D) return;                     // k_tc_form_x's matrix
+  const float lambda = mt.sc->lambda;
+  if (blockIdx.x == 0 && threadIdx.x == 0) fast[2 * p + 1] = lambda;   // read by the back-projection epilogue
+  if (lambda == 1.f) return;
+  const int lane = threadIdx.x & 31;
+  for (int l = blockIdx.x * 8 + (threadIdx.x >> 5); l < mt.l; l += gridDim.x * 8) {
+    const float c = a_res * (1.f - lambda) * mt.kvec[l];
+    const long long base = (long long)l * mt.r;
+    for (int j = lane * 8; j < mt.r; j += 256) {
+      const uint4 xu = *reinterpret_cast<const uint4*>(mt.Xb + base + j);
+      const uint4 ru = *reinterpret_cast<const uint4*>(mt.Rb + base + j);
+      float xv[8], rv[8], x[8];
+      unpack8_bf16(xu, xv);
+      unpack8_bf16(ru, rv);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) x[e] = xv[e] + c * rv[e];
+      *reinterpret_cast<uint4*>(mt.Xb + base + j) = pack8_bf16(x);
+    }
   }
 }
 
@@ -353,6 +392,7 @@ struct TcPlan {
   const int* wq_blk = nullptr;       // prefix sums of the blocks of k_tc_proj_weights
   int wq_blocks = 0;
   int num_sms = 148;
+  int max_pairs_fused = 0;           // CTA pairs of the projection kernel that are resident at once (see launch_tc_step)
   bool attrs_set = false;
   // host copies of the prefix arrays (needed only to step a sub-range of the list)
   std::vector<int> h_k1, h_k2, h_cs, h_rs, h_sl, h_ss;
@@ -370,7 +410,9 @@ long long tc_staging_pitch(const fira_matrix_desc& d) {
 
 size_t tc_colpart_floats(const fira_matrix_desc& d) {
   const size_t l = std::max(d.m, d.n);
-  return (3 + K1_GSQ_SPLIT) * (size_t)(d.r / host_tile_bn(d.r)) * l;   // N^2 and R^2 per r-tile, the partial G^2, the weighted R^2
+  // N^2 and R^2 per r-tile, the partial G^2, the weighted R^2; then 8 counters per row of tiles
+  // ([CTA rank][lane quarter]) for the exchange of the partial sums between the projection epilogues
+  return (3 + K1_GSQ_SPLIT) * (size_t)(d.r / host_tile_bn(d.r)) * l + 8 * ((l + 2 * BM - 1) / (2 * BM));
 }
 
 size_t tc_part_floats(const fira_matrix_desc& d) { return ((size_t)std::max(d.m, d.n) + 255) / 256; }
@@ -408,6 +450,7 @@ static bool encode_matrix_maps(const MatDev& mt0, TcMaps& mp, bool only_g) {
   if (!encode_map(&mp.ev, mt.V, mt.l, mt.r, mt.r, K1_ECOLS, K1_EROWS, 1)) return false;
   if (!encode_map(&mp.en, mt.Nb, mt.l, mt.r, mt.r, K1_ECOLS, K1_EROWS, 2)) return false;
   if (!encode_map(&mp.er, mt.Rb, mt.l, mt.r, mt.r, K1_ECOLS, K1_EROWS, 2)) return false;
+  if (!encode_map(&mp.ex, mt.Xb, mt.l, mt.r, mt.r, K1_ECOLS, K1_EROWS, 2)) return false;
   if (!encode_map_chunked(&mp.g1b, mt.P, mt.d, mt.r, mt.r, 64, host_tile_bn(mt.r) / 128)) return false;
   const void* a2 = mt.left ? (const void*)mt.P : (const void*)mt.Xb;
   const void* b2 = mt.left ? (const void*)mt.Xb : (const void*)mt.P;
@@ -491,7 +534,7 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
           d.colpart = mt.colpart; d.slot = (int)q; d.l0 = a * 2 * BM; d.r0 = b * bn;
           d.nkb = (mt.d + BK - 1) / BK; d.L = mt.l;
           d.bn_left = bn | ((mt.r / bn) << 16) | (mt.left ? (int)0x80000000 : 0) |
-                      ((mt.left && mt.n % 64 == 0) ? PROJ_A_CHUNKED : 0);
+                      ((mt.left && mt.n % 64 == 0) ? PROJ_A_CHUNKED : 0) | (mt.d >= FUSE_X_MIN_D ? PROJ_FUSE_X : 0);
           tp.push_back(d);
         }
     }
@@ -596,7 +639,7 @@ fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntile
   if (c->device < 0 || c->device >= 64) { set_error("refresh product: device index out of range"); return FIRA_ERR_CUDA; }
   if (!sms_of_device[c->device]) {
     int n = 0;
-    cudaError_t e = cudaFuncSetAttribute(k_tc_project<EPI_PLAIN, PSI_ADAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(k_tc_project<EPI_PLAIN, PSI_ADAM, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, c->device);
     if (e != cudaSuccess || n <= 0) { set_error(std::string("refresh product set-up: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
     sms_of_device[c->device] = n;
@@ -606,7 +649,7 @@ fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntile
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(table_dev);
   const ProjTileDesc* tiles = reinterpret_cast<const ProjTileDesc*>(table_dev + align_up(sizeof(TcMaps) * (size_t)njobs));
   Hyper hp{};
-  k_tc_project<EPI_PLAIN, PSI_ADAM><<<2 * std::min(ntiles, num_sms / 2), K1_THREADS, K1_SMEM_BYTES, c->stream>>>(
+  k_tc_project<EPI_PLAIN, PSI_ADAM, 0><<<2 * std::min(ntiles, num_sms / 2), K1_THREADS, K1_SMEM_BYTES, c->stream>>>(
       maps, tiles, ntiles, nullptr, nullptr, nullptr, hp, c->status_dev);
   return FIRA_OK;
 }
@@ -630,13 +673,33 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
   if (!pl || pl->nlist == 0) return 0;
   cudaStream_t st = c->stream;
   if (!pl->attrs_set) {
-    cudaError_t e1 = cudaFuncSetAttribute(k_tc_project<EPI_ADAM, PSI_ADAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
-    if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(k_tc_project<EPI_ADAM, PSI_RMSPROP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
-    if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(k_tc_project<EPI_ADAM, PSI_ADAGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
+    const void* k1s[6] = {(const void*)k_tc_project<EPI_ADAM, PSI_ADAM, 0>, (const void*)k_tc_project<EPI_ADAM, PSI_RMSPROP, 0>,
+                          (const void*)k_tc_project<EPI_ADAM, PSI_ADAGRAD, 0>, (const void*)k_tc_project<EPI_ADAM, PSI_ADAM, 1>,
+                          (const void*)k_tc_project<EPI_ADAM, PSI_RMSPROP, 1>, (const void*)k_tc_project<EPI_ADAM, PSI_ADAGRAD, 1>};
+    cudaError_t e1 = cudaSuccess;
+    for (int i = 0; i < 6 && e1 == cudaSuccess; ++i)
+      e1 = cudaFuncSetAttribute(k1s[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
     cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES);
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
       set_error(std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
       return -1;
+    }
+    // The epilogues of the fused projection kernel wait for one another across CTA pairs, so every
+    // pair of its grid must be resident at once: the grid is capped at what the device can hold.
+    {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(2 * (pl->num_sms / 2)); cfg.blockDim = dim3(K1_THREADS); cfg.dynamicSmemBytes = K1_SMEM_BYTES;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      cfg.attrs = at; cfg.numAttrs = 1;
+      int nclusters = 0;
+      const cudaError_t e3 = cudaOccupancyMaxActiveClusters(&nclusters, k1s[3], &cfg);
+      if (e3 != cudaSuccess || nclusters <= 0) {
+        set_error(std::string("cudaOccupancyMaxActiveClusters: ") + cudaGetErrorString(e3));
+        return -1;
+      }
+      pl->max_pairs_fused = std::min(nclusters, pl->num_sms / 2);
     }
     pl->attrs_set = true;
   }
@@ -664,20 +727,20 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
   }
   if (srn) k_tc_stage<<<srn, 256, 0, st>>>(mats, pl->stage_list, pl->nstage, pl->stage_start, sra, 0);
   tm->mark(st);
-  k_tc_prep<<<(nq + 127) / 128, 128, 0, st>>>(mats, pl->list, qa, qb, hp, pl->fast_dev);
+  k_tc_prep<<<nq, 32, 0, st>>>(mats, pl->list, qa, hp, pl->fast_dev);
   tm->mark(st);
   // both tensor kernels: clusters of two CTAs, at most one CTA per SM
-  const int k1_grid = 2 * std::min(k1n, pl->num_sms / 2);
+  // the plain step (column factors, residual kept) forms X in the projection epilogue
+  const bool fused = (hp.mode & (HYPER_MATRIX_SCALING | HYPER_NO_SCALING | HYPER_NO_RESIDUAL | HYPER_ONLY_SCALING)) == 0;
+  const int k1_grid = 2 * std::min(k1n, fused ? pl->max_pairs_fused : pl->num_sms / 2);
   const ProjTileDesc* td1 = pl->td1_dev + k1a;
-  if (hp.mode & HYPER_PSI_RMSPROP)
-    k_tc_project<EPI_ADAM, PSI_RMSPROP><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(
-        pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev);
-  else if (hp.mode & HYPER_PSI_ADAGRAD)
-    k_tc_project<EPI_ADAM, PSI_ADAGRAD><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(
-        pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev);
-  else
-    k_tc_project<EPI_ADAM, PSI_ADAM><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(
-        pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev);
+#define FIRA_LAUNCH_K1(PSI, FUSE)                                                     \
+  k_tc_project<EPI_ADAM, PSI, FUSE><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(      \
+      pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev)
+  if (hp.mode & HYPER_PSI_RMSPROP) { if (fused) FIRA_LAUNCH_K1(PSI_RMSPROP, 1); else FIRA_LAUNCH_K1(PSI_RMSPROP, 0); }
+  else if (hp.mode & HYPER_PSI_ADAGRAD) { if (fused) FIRA_LAUNCH_K1(PSI_ADAGRAD, 1); else FIRA_LAUNCH_K1(PSI_ADAGRAD, 0); }
+  else { if (fused) FIRA_LAUNCH_K1(PSI_ADAM, 1); else FIRA_LAUNCH_K1(PSI_ADAM, 0); }
+#undef FIRA_LAUNCH_K1
   tm->mark(st);
   k_tc_colfactors<<<csn, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->col_start, csa, hp);
   tm->mark(st);
@@ -692,15 +755,22 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
     tm->mark(st);
     return srn ? 6 : 5;
   }
-  k_tc_form_x<<<(rsb - rsa + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start, rsa, rsb,
-                                                   hp.a_low, hp.a_res, pl->fast_dev);
+  // X: the matrices whose projection epilogue formed it only need the limiter's correction
+  bool any_fused = false, any_plain = false;
+  for (int q = qa; q < qb; ++q) {
+    if (fused && c->mats[c->tc_list[q]].d >= FUSE_X_MIN_D) any_fused = true; else any_plain = true;
+  }
+  if (any_plain)
+    k_tc_form_x<<<(rsb - rsa + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start, rsa, rsb,
+                                                     hp.a_low, hp.a_res, pl->fast_dev, fused ? 1 : 0);
+  if (any_fused) k_tc_fix_x<<<dim3(64, nq), 256, 0, st>>>(mats, pl->list, qa, hp.a_res, pl->fast_dev);
   tm->mark(st);
   k_tc_back_project<<<2 * std::min(k2n, pl->num_sms / 2), K2_THREADS, K2_SMEM_BYTES, st>>>(
       pl->maps_dev, pl->td2_dev + k2a, k2n, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);
   if (srn) k_tc_stage<<<srn, 256, 0, st>>>(mats, pl->stage_list, pl->nstage, pl->stage_start, sra, 1);
   tm->mark(st);
-  return srn ? 8 : 6;
+  return (srn ? 7 : 5) + (any_plain ? 1 : 0) + (any_fused ? 1 : 0);
 }
 
 }  // namespace fira

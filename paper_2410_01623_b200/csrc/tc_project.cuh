@@ -38,6 +38,21 @@
 // Warp roles: 0 operand producer (TMA); 1 MMA issuer (even CTA only) and TMEM owner;
 // 2 epilogue loader (TMA); 3-6 epilogue; 7 one thread that stores the finished boxes;
 // 8-15 sums of G^2.
+//
+// FUSE_X (the plain step: column factors, residual kept): the operand X = a_low N - a_res k_l R of the
+// back-projection is formed here, for limiter factor 1, instead of in a pass of its own over N and R.
+// k_l needs ||N_l|| and ||R_l|| over the whole rank range, i.e. over the r / BN tiles of a row of
+// tiles, which different CTA pairs compute at about the same time.  So the epilogue makes two sweeps
+// over its accumulator.  Sweep 1 does the moment update as before and puts the pair {bf16 N, bf16 R}
+// back into each accumulator cell (tcgen05.st) instead of writing N and R out; it leaves its partial
+// row sums in global memory and adds one to a counter of its (row of tiles, CTA rank, lane quarter).
+// When the counter shows every tile of the row (a bounded poll: the pairs of a row run side by side,
+// and a tile only ever waits for tiles whose index is at most three above its own, each of which
+// follows, on its pair, a tile far below it, so the waits cannot form a cycle as long as every block
+// of the grid is resident, which the launch ensures), the thread adds the partial sums in the fixed
+// order that k_tc_colfactors uses, and sweep 2 reads the pairs back and writes X (through the map of
+// the X buffer) and R (bf16, needed only where the limiter acts: there k_tc_form_x adds
+// a_res (1 - lambda) k_l R to X).
 constexpr int K1_STAGES = 5;
 constexpr int K1_STAGE_BYTES = 2 * A_STAGE_BYTES;       // A: 128 l x 64 d, B half: 128 r x 64 d
 constexpr int K1_ECOLS = 32;                            // columns per epilogue box
@@ -63,11 +78,16 @@ struct ProjTileDesc {
   int slot;            // index into the tensor-map table and the fast-scalar table
   int l0, r0;          // first unprojected index / first rank index of the tile
   int nkb;             // k-blocks: ceil(d / 64)
-  int bn_left;         // bits 0-15: BN (128 or 256); 16-23: r / BN; 30: G comes as one chunked box; 31: left
+  int bn_left;         // bits 0-15: BN (128 or 256); 16-23: r / BN; 29: the epilogue forms X; 30: G comes as one chunked box; 31: left
   int L;               // number of unprojected indices of the matrix
 };
 static_assert(sizeof(ProjTileDesc) == 32, "ProjTileDesc layout");
 constexpr int PROJ_A_CHUNKED = 1 << 30;
+constexpr int PROJ_FUSE_X = 1 << 29;      // bn_left: this tile's epilogue forms X itself (FUSE_X kernels only)
+// The second sweep lengthens the epilogue, which pays where the products of a tile take long enough
+// to hide it (measured: 7B list, d = 4096, -6 % on the step; d = 1024 and 2048: +3 to +4 %, the
+// tiles are epilogue-bound there): matrices below this projected extent keep the separate pass.
+constexpr int FUSE_X_MIN_D = 4096;
 
 // EPI_PLAIN products may run over up to three k-segments that accumulate into the same tile: segment
 // s multiplies A taken through the map g1a (bit s of asel clear) or g2a (set) with B taken through
@@ -91,6 +111,7 @@ struct ProjCtl {
   uint64_t eready[K1_MVBUFS];   // the epilogue has finished M, V (in place) and N, R of a box
   uint64_t eempty[K1_MVBUFS];   // the stores have read M and V: the buffer is free
   uint64_t nrempty[K1_NRBUFS];  // the stores have read N and R: the buffer is free
+  uint64_t xready[K1_NRBUFS];   // FUSE_X: a row half has finished an X box and an R box
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -122,7 +143,7 @@ enum { EPI_ADAM = 0, EPI_PLAIN = 1 };
 // carried through unchanged).
 enum { PSI_ADAM = 0, PSI_RMSPROP = 1, PSI_ADAGRAD = 2 };
 
-template <int EPI, int PSI>
+template <int EPI, int PSI, int FUSE_X>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(K1_THREADS, 1)
 k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ tdesc, int total_tiles,
              const float* __restrict__ fast, const float* __restrict__ wq_all, const int* __restrict__ wq_off,
@@ -154,7 +175,10 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
       ptx::mbar_init(ptx::smem_u32(&ctl->eready[b]), K1_BOX_THREADS);
       ptx::mbar_init(ptx::smem_u32(&ctl->eempty[b]), 1);
     }
-    for (int b = 0; b < K1_NRBUFS; ++b) ptx::mbar_init(ptx::smem_u32(&ctl->nrempty[b]), 1);
+    for (int b = 0; b < K1_NRBUFS; ++b) {
+      ptx::mbar_init(ptx::smem_u32(&ctl->nrempty[b]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl->xready[b]), K1_BOX_THREADS);
+    }
     ctl->abort_flag = smem_ok ? 0 : 1;
     ptx::fence_barrier_init();
   }
@@ -376,6 +400,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     // ------------------------------------------------------------ box storer
     if (lane == 0 && smem_ok) {
       int mv = 0; uint32_t mvphase = 0; bool ok = true;
+      uint32_t xphase = 0;                                // FUSE_X: parities of xready, one bit per row half
       ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
       for (int t = pair; t < total_tiles && ok; t += npairs) {
         const ProjTileDesc d = nd;
@@ -383,6 +408,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         const TcMaps* mp = &maps[d.slot];
         const int bn = d.bn_left & 0xffff;
         const int l0 = d.l0 + BM * (int)rank;
+        const bool fuse = FUSE_X && (d.bn_left & PROJ_FUSE_X);
         for (int b = 0; b < 2 * (bn / K1_ECOLS); ++b) {
           if (!ptx::mbar_wait(ptx::smem_u32(&ctl->eready[mv]), mvphase, abort_flag)) { ok = false; break; }
           const int nr = b & 1;
@@ -392,8 +418,10 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
             if (EPI == EPI_ADAM) {
               ptx::tma_store_2d(&mp->em, src, j, row);
               ptx::tma_store_2d(&mp->ev, src + K1_FBOX_BYTES, j, row);
-              ptx::tma_store_2d(&mp->en, srn, j, row);
-              ptx::tma_store_2d(&mp->er, srn + K1_HBOX_BYTES, j, row);
+              if (!fuse) {
+                ptx::tma_store_2d(&mp->en, srn, j, row);
+                ptx::tma_store_2d(&mp->er, srn + K1_HBOX_BYTES, j, row);
+              }
             } else {
               ptx::tma_store_2d(&mp->em, srn, j, row);      // the fp32 output box sits in the N/R buffer
             }
@@ -401,8 +429,25 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
             ptx::bulk_wait_group_read<0>();              // the boxes have been read: the buffers are free
           }
           ptx::mbar_arrive(ptx::smem_u32(&ctl->eempty[mv]));
-          ptx::mbar_arrive(ptx::smem_u32(&ctl->nrempty[nr]));
+          if (!fuse) ptx::mbar_arrive(ptx::smem_u32(&ctl->nrempty[nr]));
           if (++mv == K1_MVBUFS) { mv = 0; mvphase ^= 1u; }
+        }
+        if (fuse && ok) {
+          // second sweep of the epilogue: the X and R boxes of this tile, in the same order
+          for (int b = 0; b < 2 * (bn / K1_ECOLS); ++b) {
+            const int nr = b & 1;
+            if (!ptx::mbar_wait(ptx::smem_u32(&ctl->xready[nr]), (xphase >> nr) & 1u, abort_flag)) { ok = false; break; }
+            xphase ^= 1u << nr;
+            const int j = d.r0 + K1_ECOLS * (b >> 1), row = l0 + K1_EROWS * nr;
+            if (row < d.L) {
+              const uint32_t srn = nrbuf_u32 + nr * K1_NRBUF_BYTES;
+              ptx::tma_store_2d(&mp->ex, srn, j, row);
+              ptx::tma_store_2d(&mp->er, srn + K1_HBOX_BYTES, j, row);
+              ptx::bulk_commit_group();
+              ptx::bulk_wait_group_read<0>();
+            }
+            ptx::mbar_arrive(ptx::smem_u32(&ctl->nrempty[nr]));
+          }
         }
       }
       ptx::bulk_wait_group_all();
@@ -442,19 +487,20 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
       const uint32_t tcol = tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX;
       const uint32_t te = buf ? tmem_empty1 : tmem_empty0;
       const int nch = bn / K1_ECOLS;
+      const bool fuse = FUSE_X && (d.bn_left & PROJ_FUSE_X);
       float nn = 0.f, rn = 0.f, rw = 0.f;
       for (int c = 0; c < nch; ++c) {
         uint32_t rr[32];
         __syncwarp();
         ptx::tmem_ld_32x32b_x32(tcol + K1_ECOLS * c, rr);
         ptx::tmem_ld_wait();
-        if (c == nch - 1) {                              // the accumulator has been read out
+        if (!fuse && c == nch - 1) {                     // the accumulator has been read out
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive_cluster(te);
         }
         if (EPI == EPI_ADAM && !ptx::mbar_wait(ptx::smem_u32(&ctl->efull[mv][half]), mvphase, abort_flag)) { ok = false; break; }
-        if (!ptx::mbar_wait(nrempty, nrphase ^ 1u, abort_flag)) { ok = false; break; }
+        if (!fuse && !ptx::mbar_wait(nrempty, nrphase ^ 1u, abort_flag)) { ok = false; break; }
         unsigned char* mb = mvbuf + (size_t)mv * K1_MVBUF_BYTES;
         unsigned char* vb = mb + K1_FBOX_BYTES;
         if (EPI == EPI_PLAIN) {
@@ -497,16 +543,29 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           *reinterpret_cast<float4*>(mb + f1) = make_float4(mo[4], mo[5], mo[6], mo[7]);
           *reinterpret_cast<float4*>(vb + f0) = make_float4(vo[0], vo[1], vo[2], vo[3]);
           *reinterpret_cast<float4*>(vb + f1) = make_float4(vo[4], vo[5], vo[6], vo[7]);
-          const uint32_t h = hrow + (((uint32_t)q ^ hsw) << 4);
-          *reinterpret_cast<uint4*>(nb + h) = pack8_bf16(nv);
-          *reinterpret_cast<uint4*>(rb + h) = pack8_bf16(rv);
+          if (fuse) {
+            // the pair {bf16 N (low half), bf16 R (high half)} goes back into the accumulator cell
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const __nv_bfloat162 pr = __floats2bfloat162_rn(nv[e], rv[e]);
+              rr[8 * q + e] = *reinterpret_cast<const uint32_t*>(&pr);
+            }
+          } else {
+            const uint32_t h = hrow + (((uint32_t)q ^ hsw) << 4);
+            *reinterpret_cast<uint4*>(nb + h) = pack8_bf16(nv);
+            *reinterpret_cast<uint4*>(rb + h) = pack8_bf16(rv);
+          }
         }
+        }
+        if (fuse) {
+          ptx::tmem_st_32x32b_x32(tcol + K1_ECOLS * c, rr);
+          ptx::tmem_st_wait();
         }
         // hand the finished boxes to the storer: this thread's writes are visible to
         // the async proxy (TMA) before it arrives
         ptx::fence_proxy_async_smem();
         ptx::mbar_arrive(ptx::smem_u32(&ctl->eready[mv]));
-        nrphase ^= 1u;
+        if (!fuse) nrphase ^= 1u;
         mv += 2;                                         // this warp's next box is two further on
         if (mv >= K1_MVBUFS) mv -= K1_MVBUFS;
         if (++mvuse == K1_MVBUFS) { mvuse = 0; mvphase ^= 1u; }
@@ -518,6 +577,65 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         d.colpart[(long long)(2 * part) * d.L + l] = nn;
         d.colpart[(long long)(2 * part + 1) * d.L + l] = rn;
         d.colpart[(long long)((2 + K1_GSQ_SPLIT) * nparts + part) * d.L + l] = rw;
+      }
+      if (fuse && ok) {
+        // ---- the factor k_l of this thread's row, from the partial sums of every tile of the row of tiles
+        const int nparts = (d.bn_left >> 16) & 0xff;
+        float nt = 0.f, rt = 0.f;
+        if (nparts > 1) {
+          // counters behind the matrix's partial sums: [row of tiles][CTA rank][lane quarter]
+          uint32_t* cnt = reinterpret_cast<uint32_t*>(d.colpart + (long long)(3 + K1_GSQ_SPLIT) * nparts * d.L) +
+                          ((d.l0 / (2 * BM)) * 2 + (int)rank) * 4 + quarter;
+          __threadfence();                               // this thread's partial sums, before the warp's count
+          __syncwarp();
+          int got = 1;
+          if (lane == 0) {
+            ptx::signal_counter(cnt);
+            got = ptx::wait_counter(cnt, (uint32_t)nparts, abort_flag) ? 1 : 0;
+          }
+          got = __shfl_sync(0xffffffffu, got, 0);
+          if (!got) break;
+          if (l < d.L) {
+            for (int q = 0; q < nparts; ++q) {           // the order of k_tc_colfactors
+              nt += __ldcg(d.colpart + (long long)(2 * q) * d.L + l);
+              rt += __ldcg(d.colpart + (long long)(2 * q + 1) * d.L + l);
+            }
+          }
+        } else {
+          nt += nn; rt += rn;
+        }
+        const float kl = (l < d.L) ? sqrtf(nt) / (sqrtf(rt) + hp.eps) : 0.f;
+        const float ck = hp.a_res * 1.0f * kl;           // k_tc_form_x's coefficient at lambda = 1
+        // ---- sweep 2: X = a_low N - a_res k_l R and R itself, as bf16 boxes
+        for (int c = 0; c < nch; ++c) {
+          uint32_t rr[32];
+          __syncwarp();
+          ptx::tmem_ld_32x32b_x32(tcol + K1_ECOLS * c, rr);
+          ptx::tmem_ld_wait();
+          if (c == nch - 1) {                            // the accumulator has been read out
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(te);
+          }
+          if (!ptx::mbar_wait(nrempty, nrphase ^ 1u, abort_flag)) { ok = false; break; }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            float xv[8], rv[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&rr[8 * q + e]));
+              rv[e] = f.y;
+              xv[e] = hp.a_low * f.x - ck * f.y;
+            }
+            const uint32_t h = hrow + (((uint32_t)q ^ hsw) << 4);
+            *reinterpret_cast<uint4*>(nb + h) = pack8_bf16(xv);
+            *reinterpret_cast<uint4*>(rb + h) = pack8_bf16(rv);
+          }
+          ptx::fence_proxy_async_smem();
+          ptx::mbar_arrive(ptx::smem_u32(&ctl->xready[half]));
+          nrphase ^= 1u;
+        }
+        if (!ok) break;
       }
       if (++buf == 2) { buf = 0; bphase ^= 1u; }
     }

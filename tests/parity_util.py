@@ -204,6 +204,11 @@ def rounding_variance(proj: np.ndarray, d: dict, ohp: fo.Hyper, left: bool) -> t
         cR = torch.zeros_like(R)
     aN = a_low * N
     Y2 = aN * aN + cR * cR + (aN - cR) ** 2
+    if ohp.residual and d["lam"] < 1.0:
+        # the plain step forms X for lambda = 1 in the projection epilogue (one bf16 rounding) and
+        # adds a_res (1 - lambda) k_l R where the limiter acted (a second one)
+        X1 = aN - cR / float(d["lam"])
+        Y2 = Y2 + X1 * X1
     P2 = torch.from_numpy((proj * proj).astype(np.float32)).to(dev)
     v = (P2 @ Y2) * float(ohp.lr ** 2 * BF16_REL_VAR)                      # d x l
     return v if left else v.T.contiguous()
