@@ -679,7 +679,9 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
     cudaError_t e1 = cudaSuccess;
     for (int i = 0; i < 6 && e1 == cudaSuccess; ++i)
       e1 = cudaFuncSetAttribute(k1s[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
-    cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES);
+    cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project<5, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)k2_smem_bytes(5, 2));
+    if (e2 == cudaSuccess)
+      e2 = cudaFuncSetAttribute(k_tc_back_project<4, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)k2_smem_bytes(4, 3));
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
       set_error(std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
       return -1;
@@ -765,8 +767,15 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
                                                      hp.a_low, hp.a_res, pl->fast_dev, fused ? 1 : 0);
   if (any_fused) k_tc_fix_x<<<dim3(64, nq), 256, 0, st>>>(mats, pl->list, qa, hp.a_res, pl->fast_dev);
   tm->mark(st);
-  k_tc_back_project<<<2 * std::min(k2n, pl->num_sms / 2), K2_THREADS, K2_SMEM_BYTES, st>>>(
-      pl->maps_dev, pl->td2_dev + k2a, k2n, pl->fast_dev, hp, c->status_dev);
+  // long products keep five operand stages; short ones trade one for more epilogue boxes in flight
+  int rmax = 0;
+  for (int q = qa; q < qb; ++q) rmax = std::max(rmax, c->mats[c->tc_list[q]].r);
+  if (rmax >= 1024)
+    k_tc_back_project<5, 2><<<2 * std::min(k2n, pl->num_sms / 2), K2_THREADS, k2_smem_bytes(5, 2), st>>>(
+        pl->maps_dev, pl->td2_dev + k2a, k2n, pl->fast_dev, hp, c->status_dev);
+  else
+    k_tc_back_project<4, 3><<<2 * std::min(k2n, pl->num_sms / 2), K2_THREADS, k2_smem_bytes(4, 3), st>>>(
+        pl->maps_dev, pl->td2_dev + k2a, k2n, pl->fast_dev, hp, c->status_dev);
   tm->mark(st);
   if (srn) k_tc_stage<<<srn, 256, 0, st>>>(mats, pl->stage_list, pl->nstage, pl->stage_start, sra, 1);
   tm->mark(st);

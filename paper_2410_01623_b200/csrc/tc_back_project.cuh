@@ -25,10 +25,13 @@
 // each that stores a group's finished W boxes (TMA) and hands the buffers back to the
 // loader.  (Issuing the two boxes of a stage from two threads changed nothing: the
 // stages wait for the data, not for the issuing thread.)
-constexpr int K2_STAGES = 5;
+// Two splits of the shared memory between operand stages and epilogue boxes (template parameters
+// of the kernel): 5 stages + 2 boxes in flight per epilogue group for long products (r >= 1024,
+// tensor-bound), 4 stages + 3 boxes for short ones, whose tiles are bound by the rate at which the
+// epilogue streams G and W (measured: 350M list -12 %, 1B list -6 % on this kernel with 4 + 3; the
+// 7B list +3 % with it, so it keeps 5 + 2).
 constexpr int K2_STAGE_BYTES = 2 * A_STAGE_BYTES;       // A: 128 x 64, B half: 128 x 64
 constexpr int K2_GROUPS = 2;
-constexpr int K2_GBUFS = 2;                             // boxes in flight per epilogue group
 constexpr int K2_ECOLS = 32;                            // columns per epilogue box
 constexpr int K2_EBOX_BYTES = BM * K2_ECOLS * 2;        // 8 KiB
 constexpr int K2_EBUF_BYTES = 2 * K2_EBOX_BYTES;        // G box + W box
@@ -37,9 +40,10 @@ constexpr int K2_THREADS = 32 * 3 + K2_GROUPS * K2_GROUP_THREADS + 32 * K2_GROUP
 constexpr int K2_NCH = BN_MAX / K2_ECOLS;               // 8 boxes per tile
 constexpr int K2_KS_GROUP = BN_MAX / K2_GROUPS;         // k values a group needs per tile (its own boxes)
 constexpr int K2_KS_FLOATS = K2_GROUPS * 2 * K2_KS_GROUP;   // per group, two tile parities
-constexpr size_t K2_SMEM_BYTES = (size_t)K2_STAGES * K2_STAGE_BYTES +
-                                 (size_t)K2_GROUPS * K2_GBUFS * K2_EBUF_BYTES + 512 + K2_KS_FLOATS * sizeof(float);
-static_assert(K2_SMEM_BYTES <= 227 * 1024, "shared memory budget");
+constexpr size_t k2_smem_bytes(int stages, int gbufs) {
+  return (size_t)stages * K2_STAGE_BYTES + (size_t)K2_GROUPS * gbufs * K2_EBUF_BYTES + 512 + K2_KS_FLOATS * sizeof(float);
+}
+static_assert(k2_smem_bytes(5, 2) <= 227 * 1024 && k2_smem_bytes(4, 3) <= 227 * 1024, "shared memory budget");
 
 // Per-tile record (a 256 x 256 tile of W), built on the host once (32 bytes).
 struct BackTileDesc {
@@ -52,6 +56,7 @@ struct BackTileDesc {
 };
 static_assert(sizeof(BackTileDesc) == 32, "BackTileDesc layout");
 
+template <int K2_STAGES, int K2_GBUFS>
 struct BackCtl {
   uint64_t full[K2_STAGES];     // (even CTA) both CTAs' operands of a stage have landed
   uint64_t empty[K2_STAGES];    // the MMAs reading a stage are done (both CTAs are told)
@@ -64,7 +69,7 @@ struct BackCtl {
   uint32_t tmem_base;
   int abort_flag;
 };
-static_assert(sizeof(BackCtl) <= 512, "BackCtl must fit its slot");
+static_assert(sizeof(BackCtl<5, 2>) <= 512 && sizeof(BackCtl<4, 3>) <= 512, "BackCtl must fit its slot");
 
 __device__ __forceinline__ BackTileDesc load_desc(const BackTileDesc* __restrict__ td, int t) {
   const int4 a = __ldg(reinterpret_cast<const int4*>(td + t));
@@ -76,13 +81,15 @@ __device__ __forceinline__ BackTileDesc load_desc(const BackTileDesc* __restrict
   return d;
 }
 
+template <int K2_STAGES, int K2_GBUFS>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(K2_THREADS, 1)
 k_tc_back_project(const TcMaps* __restrict__ maps, const BackTileDesc* __restrict__ tdesc, int total_tiles,
                   const float* __restrict__ fast, Hyper hp, unsigned* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* tiles = smem_raw;
   unsigned char* ebuf = tiles + (size_t)K2_STAGES * K2_STAGE_BYTES;
-  BackCtl* ctl = reinterpret_cast<BackCtl*>(ebuf + (size_t)K2_GROUPS * K2_GBUFS * K2_EBUF_BYTES);
+  using Ctl = BackCtl<K2_STAGES, K2_GBUFS>;
+  Ctl* ctl = reinterpret_cast<Ctl*>(ebuf + (size_t)K2_GROUPS * K2_GBUFS * K2_EBUF_BYTES);
   float* ksm = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(ctl) + 512);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = ptx::cluster_ctarank();          // 0: issues the MMAs; 1: its partner

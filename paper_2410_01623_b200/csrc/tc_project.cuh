@@ -24,10 +24,13 @@
 // same way: ordinary global loads would be throttled by the few L1 lines that remain when
 // nearly the whole L1/shared array is configured as shared memory.  The boxes of a tile come
 // in the order (columns 0-31, rows 0-63), (columns 0-31, rows 64-127), (columns 32-63, ...):
-// epilogue warps 0-1 take the even boxes, warps 2-3 the odd ones.  Three M/V buffers rotate
-// over all boxes, so that loads run ahead; the N/R buffer of a box is the one of its row half.
-// Small boxes leave room for five operand stages: the time from a stage's release to its next
-// MMA is several thousand cycles, which four stages do not cover.
+// epilogue warps 0-1 take the even boxes, warps 2-3 the odd ones.  Five M/V buffers (an odd number,
+// so that every buffer serves both row halves in turn) rotate over all boxes, so that loads run
+// ahead; the N/R buffer of a box is the one of its row half.  Four operand stages and five M/V
+// buffers share the shared memory: the step's time does not depend on the fifth stage (measured
+// with 3 to 6 stages), while two more M/V boxes in flight raise the rate at which the epilogue
+// streams M and V, which is what bounds the lists with a short product (350M: -7 %, 1B: -5 % on
+// this kernel; 7B unchanged).
 //
 // ||G_l||^2: G passes through shared memory as the A operand anyway.  The r / BN tiles that share a
 // panel of G split its k-blocks between them (tile `part` takes k-blocks part, part + r / BN, ...):
@@ -53,13 +56,13 @@
 // order that k_tc_colfactors uses, and sweep 2 reads the pairs back and writes X (through the map of
 // the X buffer) and R (bf16, needed only where the limiter acts: there k_tc_form_x adds
 // a_res (1 - lambda) k_l R to X).
-constexpr int K1_STAGES = 5;
+constexpr int K1_STAGES = 4;
 constexpr int K1_STAGE_BYTES = 2 * A_STAGE_BYTES;       // A: 128 l x 64 d, B half: 128 r x 64 d
 constexpr int K1_ECOLS = 32;                            // columns per epilogue box
 constexpr int K1_EROWS = 64;                            // rows per epilogue box
 constexpr int K1_FBOX_BYTES = K1_EROWS * K1_ECOLS * 4;  // fp32 box: 8 KiB
 constexpr int K1_HBOX_BYTES = K1_EROWS * K1_ECOLS * 2;  // bf16 box: 4 KiB
-constexpr int K1_MVBUFS = 3;                            // {M box, V box}
+constexpr int K1_MVBUFS = 5;                            // {M box, V box}
 constexpr int K1_NRBUFS = 2;                            // {N box, R box}, one per row half
 constexpr int K1_MVBUF_BYTES = 2 * K1_FBOX_BYTES;
 constexpr int K1_NRBUF_BYTES = 2 * K1_HBOX_BYTES;
