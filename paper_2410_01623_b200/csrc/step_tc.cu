@@ -248,7 +248,7 @@ k_tc_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int n
   const MatDev& mt = mats[list[p]];
   const int l = row - row_start[p];
   const float lambda = mt.sc->lambda;
-  if (fused && mt.d >= FUSE_X_MIN_D) return;           // k_tc_fix_x's matrix
+  if (fused && fuse_x_matrix(mt.d, mt.r)) return;      // k_tc_fix_x's matrix
   if (l == 0 && lane == 0) fast[2 * p + 1] = lambda;   // read by the back-projection epilogue
   const long long base = (long long)l * mt.r;
   const float c = a_res * lambda * mt.kvec[l];
@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(256)
 k_tc_fix_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int first, float a_res, float* __restrict__ fast) {
   const int p = first + blockIdx.y;
   const MatDev& mt = mats[list[p]];
-  if (mt.d < FUSE_X_MIN_D) return;                     // k_tc_form_x's matrix
+  if (!fuse_x_matrix(mt.d, mt.r)) return;              // k_tc_form_x's matrix
   const float lambda = mt.sc->lambda;
   if (blockIdx.x == 0 && threadIdx.x == 0) fast[2 * p + 1] = lambda;   // read by the back-projection epilogue
   if (lambda == 1.f) return;
@@ -534,7 +534,7 @@ fira_status tc_build_plan(fira_ctx* c, std::vector<int>& ints) {
           d.colpart = mt.colpart; d.slot = (int)q; d.l0 = a * 2 * BM; d.r0 = b * bn;
           d.nkb = (mt.d + BK - 1) / BK; d.L = mt.l;
           d.bn_left = bn | ((mt.r / bn) << 16) | (mt.left ? (int)0x80000000 : 0) |
-                      ((mt.left && mt.n % 64 == 0) ? PROJ_A_CHUNKED : 0) | (mt.d >= FUSE_X_MIN_D ? PROJ_FUSE_X : 0);
+                      ((mt.left && mt.n % 64 == 0) ? PROJ_A_CHUNKED : 0) | (fuse_x_matrix(mt.d, mt.r) ? PROJ_FUSE_X : 0);
           tp.push_back(d);
         }
     }
@@ -760,7 +760,8 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
   // X: the matrices whose projection epilogue formed it only need the limiter's correction
   bool any_fused = false, any_plain = false;
   for (int q = qa; q < qb; ++q) {
-    if (fused && c->mats[c->tc_list[q]].d >= FUSE_X_MIN_D) any_fused = true; else any_plain = true;
+    const MatDev& mq = c->mats[c->tc_list[q]];
+    if (fused && fuse_x_matrix(mq.d, mq.r)) any_fused = true; else any_plain = true;
   }
   if (any_plain)
     k_tc_form_x<<<(rsb - rsa + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start, rsa, rsb,

@@ -87,10 +87,13 @@ struct ProjTileDesc {
 static_assert(sizeof(ProjTileDesc) == 32, "ProjTileDesc layout");
 constexpr int PROJ_A_CHUNKED = 1 << 30;
 constexpr int PROJ_FUSE_X = 1 << 29;      // bn_left: this tile's epilogue forms X itself (FUSE_X kernels only)
-// The second sweep lengthens the epilogue, which pays where the products of a tile take long enough
-// to hide it (measured: 7B list, d = 4096, -6 % on the step; d = 1024 and 2048: +3 to +4 %, the
-// tiles are epilogue-bound there): matrices below this projected extent keep the separate pass.
+// Which matrices take that route.  The second sweep lengthens the epilogue and the exchange makes the
+// pairs of a row of tiles wait for the slowest of them.  Measured: one r-tile per row (no exchange,
+// 350M list, r = 256): -8 % on the step; long products (7B list, d = 4096, four r-tiles): -6 to
+// -7 %; short products with an exchange (1B list, d = 2048, two r-tiles): +2 %, the tiles are
+// epilogue-bound and their times jitter, so those keep the separate pass.
 constexpr int FUSE_X_MIN_D = 4096;
+__host__ __device__ inline bool fuse_x_matrix(int d, int r) { return d >= FUSE_X_MIN_D || r <= 256; }
 
 // EPI_PLAIN products may run over up to three k-segments that accumulate into the same tile: segment
 // s multiplies A taken through the map g1a (bit s of asel clear) or g2a (set) with B taken through

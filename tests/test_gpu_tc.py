@@ -85,6 +85,21 @@ def test_mixed_list_left_right_square_with_limiter():
         assert d["t"] == 6
 
 
+def test_x_formed_in_the_projection_epilogue_with_ragged_rows_and_limiter():
+    """Projected extent 4096 with rank 512: two r-tiles per row of tiles, so the projection epilogues
+    of two CTA pairs exchange their partial row sums before they form X, here with a ragged last
+    row of tiles (4200 = 16 x 256 + 104), in both orientations, mixed in one list with a matrix
+    whose X still comes from the separate pass (d = 512, two r-tiles) and one with a single r-tile;
+    a jump at step 3 makes the limiter act, which exercises the correction pass on X."""
+    shapes = [(4096, 4200), (4200, 4096), (512, 1024), (640, 512)]
+    tr = _case(shapes, [512, 512, 512, 256], steps=4, seed=77, spike=(3,))
+    assert [tr.f.diagnostics(i)["engine"] for i in range(4)] == [1, 1, 1, 1]
+    tr.assert_ok()
+    assert all(l < 0.5 for l in tr.lams[2])
+    for i in range(4):
+        assert tr.f.diagnostics(i)["norm_prev"] == pytest.approx(tr.st[i].prev_norm, rel=2e-2)
+
+
 def test_odd_widths_run_on_tensor_cores_through_aligned_copies():
     """Rows of an odd-width bf16 matrix are not 16-byte aligned, which TMA needs: the library
     works on copies with an aligned pitch and writes W back.  Odd heights need nothing special."""
