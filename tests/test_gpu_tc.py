@@ -89,9 +89,9 @@ def test_x_formed_in_the_projection_epilogue_with_ragged_rows_and_limiter():
     """Projected extent 4096 with rank 512: two r-tiles per row of tiles, so the projection epilogues
     of two CTA pairs exchange their partial row sums before they form X, here with a ragged last
     row of tiles (4200 = 16 x 256 + 104), in both orientations, mixed in one list with a matrix
-    whose X still comes from the separate pass (d = 512, two r-tiles) and one with a single r-tile;
+    whose X still comes from the separate pass (d = 1024, two r-tiles) and one with a single r-tile;
     a jump at step 3 makes the limiter act, which exercises the correction pass on X."""
-    shapes = [(4096, 4200), (4200, 4096), (512, 1024), (640, 512)]
+    shapes = [(4096, 4200), (4200, 4096), (1024, 1536), (640, 512)]
     tr = _case(shapes, [512, 512, 512, 256], steps=4, seed=77, spike=(3,))
     assert [tr.f.diagnostics(i)["engine"] for i in range(4)] == [1, 1, 1, 1]
     tr.assert_ok()
