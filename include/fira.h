@@ -94,6 +94,14 @@ typedef enum { FIRA_F32 = 0, FIRA_BF16 = 1 } fira_dtype;
  * together with gamma = inf give the printed equation literally).  M and V advance as usual.
  * Excludes FIRA_FLAG_NO_RESIDUAL. */
 #define FIRA_FLAG_ONLY_SCALING 256u
+/* Layout permission (the paper has no counterpart).  A bf16 matrix whose rows start on 16-byte
+ * boundaries (ld a multiple of 8) is read and written where it is by the tensor-core kernels; if its
+ * width n is not a multiple of 8 their stores, which move whole 16-byte units, also overwrite (with
+ * zeros) the up to 7 padding elements that follow each row of W.  With this flag the caller allows
+ * that; without it such a matrix is worked on through aligned copies in the scratch buffer (two
+ * extra passes over W and one over G per step), as is every matrix whose ld is not a multiple of 8.
+ * G's padding is never read or written. */
+#define FIRA_FLAG_ROW_PADDING_WRITABLE 512u
 
 /* Inputs of Algorithm 1.  eps > 0; 0 <= beta < 1; gamma >= 1 or +inf; T >= 0 (0: never). */
 typedef struct {

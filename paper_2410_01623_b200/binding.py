@@ -22,6 +22,7 @@ FLAG_ALPHA_LOWRANK_ONLY, FLAG_AUTO_REFRESH, FLAG_FORCE_SIMT = 1, 2, 4
 FLAG_MATRIX_SCALING, FLAG_NO_SCALING, FLAG_NO_RESIDUAL = 8, 16, 32
 FLAG_PSI_RMSPROP, FLAG_PSI_ADAGRAD = 64, 128
 FLAG_ONLY_SCALING = 256
+FLAG_ROW_PADDING_WRITABLE = 512
 
 STATUS_NAMES = {0: "FIRA_OK", 1: "FIRA_ERR_INVALID_ARG", 2: "FIRA_ERR_WORKSPACE_TOO_SMALL",
                 3: "FIRA_ERR_UNSUPPORTED", 4: "FIRA_ERR_CUDA", 5: "FIRA_ERR_DEVICE_TIMEOUT",

@@ -104,7 +104,7 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
       L.offXb[i] = w; w += align_up(ll * r * 2);
       L.offColpart[i] = w; w += align_up(tc_colpart_floats(d) * 4);
       L.offPart[i] = w; w += align_up(tc_part_floats(d) * 4);
-      const size_t lds = (size_t)tc_staging_pitch(d);
+      const size_t lds = (size_t)tc_staging_pitch(d, hp.flags);
       if (lds) {
         L.offGs[i] = w; w += align_up((size_t)d.m * lds * 2);
         L.offWs[i] = w; w += align_up((size_t)d.m * lds * 2);
@@ -224,7 +224,7 @@ fira_status fira_init(fira_ctx** out, const fira_hparams* hp, const fira_matrix_
       mt.Rb = (__nv_bfloat16*)(c->work_base + L.offRb[i]);
       mt.Xb = (__nv_bfloat16*)(c->work_base + L.offXb[i]);
       mt.colpart = (float*)(c->work_base + L.offColpart[i]);
-      mt.lds = tc_staging_pitch(c->descs[i]);
+      mt.lds = tc_staging_pitch(c->descs[i], c->hp.flags);
       if (mt.lds) {
         mt.Gs = (__nv_bfloat16*)(c->work_base + L.offGs[i]);
         mt.Ws = (__nv_bfloat16*)(c->work_base + L.offWs[i]);

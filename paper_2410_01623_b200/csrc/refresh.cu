@@ -383,7 +383,7 @@ static_assert(sizeof(RefreshMat) + 4 * sizeof(GemmDesc) + 3 * sizeof(TrsmDesc) +
 
 // bf16 matrices that TMA can read in place: their products run on the tensor cores
 static bool refresh_on_tc(const fira_matrix_desc& d) {
-  return d.dtype == FIRA_BF16 && tc_supported(d) && tc_staging_pitch(d) == 0;
+  return d.dtype == FIRA_BF16 && tc_supported(d) && tc_rows_aligned(d);   // the refresh only reads G
 }
 
 // The eight kinds of tensor-core jobs of one matrix: A Z and A^T Y (plain and with a split iterate),

@@ -402,9 +402,14 @@ bool tc_supported(const fira_matrix_desc& d) {
   return d.dtype == FIRA_BF16 && d.r % 128 == 0 && d.m >= 256 && d.n >= 256;
 }
 
-long long tc_staging_pitch(const fira_matrix_desc& d) {
-  const long long ld = d.ld ? d.ld : d.n;
-  if (d.n % 8 == 0 && ld % 8 == 0) return 0;
+bool tc_rows_aligned(const fira_matrix_desc& d) { return (d.ld ? d.ld : d.n) % 8 == 0; }
+
+// TMA reads any width in place once the rows start on 16-byte boundaries (elements past the width
+// come in as zeros), but it writes whole 16-byte units: a row whose width is not a multiple of 8
+// elements gets up to 7 elements of its padding overwritten (with zeros).  Such matrices are worked
+// on in place only if the caller has declared the padding writable; otherwise through the copies.
+long long tc_staging_pitch(const fira_matrix_desc& d, uint32_t flags) {
+  if (tc_rows_aligned(d) && (d.n % 8 == 0 || (flags & FIRA_FLAG_ROW_PADDING_WRITABLE))) return 0;
   return ((long long)d.n + 63) / 64 * 64;
 }
 

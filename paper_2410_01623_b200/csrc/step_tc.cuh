@@ -13,7 +13,8 @@ namespace fira {
 bool tc_supported(const fira_matrix_desc& d);
 // Row pitch (elements) of the aligned copies of G and W that the tensor-core path makes when the
 // caller's rows are not 16-byte aligned (odd widths or pitches); 0 when TMA can read them in place.
-long long tc_staging_pitch(const fira_matrix_desc& d);
+long long tc_staging_pitch(const fira_matrix_desc& d, uint32_t flags);
+bool tc_rows_aligned(const fira_matrix_desc& d);
 // Scratch sizes (floats) of the per-(r-tile, l) column partial sums and of the
 // partial sums of ||S||^2.
 size_t tc_colpart_floats(const fira_matrix_desc& d);

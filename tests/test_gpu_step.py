@@ -301,11 +301,14 @@ def test_step_host_matches_device_step():
 
 @pytest.mark.parametrize("dtype,shape,r,pad", [(torch.float32, (150, 333), 37, 5), (torch.float32, (333, 150), 37, 3),
                                                (torch.bfloat16, (512, 768), 128, 8), (torch.bfloat16, (768, 512), 128, 64),
-                                               (torch.bfloat16, (512, 768), 128, 3), (torch.bfloat16, (300, 333), 37, 1)])
+                                               (torch.bfloat16, (512, 768), 128, 3), (torch.bfloat16, (300, 333), 37, 1),
+                                               (torch.bfloat16, (512, 765), 128, 3), (torch.bfloat16, (768, 509), 128, 3),
+                                               (torch.bfloat16, (765, 512), 128, 8)])
 def test_padded_row_pitch(dtype, shape, r, pad):
     """W and G as views of wider buffers (ld = n + pad): the CUDA-core kernels, the tensor-core
-    kernels reading in place (pitch a multiple of 8 elements) and through aligned copies (odd
-    pitch).  The padding columns must come back untouched."""
+    kernels reading in place (pitch and width multiples of 8 elements) and through aligned copies
+    (odd pitch, or an odd width without the caller's leave to write the padding).  The padding
+    columns must come back untouched."""
     m, n = shape
     ld = n + pad
     g = torch.Generator().manual_seed(m + pad)
@@ -332,3 +335,36 @@ def test_padded_row_pitch(dtype, shape, r, pad):
     assert rel_err(to_np64(Wbuf[:, :n]) - to_np64(W0), Wo - to_np64(W0)) <= (3e-2 if dtype == torch.bfloat16 else 2e-4)
     assert (Wbuf[:, n:] == 7.0).all()
 
+
+
+@pytest.mark.parametrize("shape,ld", [((512, 765), 776), ((768, 509), 520), ((765, 512), 512)])
+def test_row_padding_writable_lets_odd_widths_run_in_place(shape, ld):
+    """FIRA_FLAG_ROW_PADDING_WRITABLE: rows that start on 16-byte boundaries are worked on where they
+    are even if the width is not a multiple of 8 (no staging kernels: 6 launches, not 8); the stores
+    may then overwrite the padding up to the next multiple of 8 elements, and nothing beyond it.
+    G's padding holds NaN: it must never enter the result."""
+    m, n = shape
+    g = torch.Generator().manual_seed(m + n)
+    hp = fb.make_hparams(lr=1e-2, alpha=0.25, gamma=1.01, flags=fb.FLAG_ROW_PADDING_WRITABLE)
+    f = fb.Fira([shape], 128, torch.bfloat16, hp, lds=[ld])
+    q, _ = torch.linalg.qr(torch.randn(min(m, n), 128, generator=g, dtype=torch.float64))
+    f.set_projection(0, q.to(torch.bfloat16).cuda())
+    P = to_np64(f.get_projection(0))
+    Wbuf = torch.full((m, ld), 7.0, dtype=torch.bfloat16, device="cuda")
+    Gbuf = torch.full((m, ld), float("nan"), dtype=torch.bfloat16, device="cuda")
+    W0 = (torch.randn(m, n, generator=g) * 0.02).to(torch.bfloat16)
+    Wbuf[:, :n] = W0.cuda()
+    st = fo.new_state(m, n, 128)
+    ohp = fo.Hyper(lr=hp.lr, alpha=hp.alpha, gamma=hp.gamma, eps=hp.eps)
+    Wo = to_np64(W0)
+    for _ in range(3):
+        G = torch.randn(m, n, generator=g).to(torch.bfloat16)
+        Gbuf[:, :n] = G.cuda()
+        f.step([Wbuf[:, :n]], [Gbuf[:, :n]])
+        Wo, _ = fo.fira_step(Wo, to_np64(G), P, st, ohp, store="bf16")
+    assert f.poll() == 0 and f.diagnostics(0)["engine"] == 1
+    assert f.last_step_launches() == 6
+    assert rel_err(to_np64(Wbuf[:, :n]), Wo) <= 2e-2
+    assert rel_err(to_np64(Wbuf[:, :n]) - to_np64(W0), Wo - to_np64(W0)) <= 3e-2
+    assert (Wbuf[:, (n + 7) // 8 * 8:] == 7.0).all()
+    assert torch.isnan(Gbuf[:, n:]).all()
