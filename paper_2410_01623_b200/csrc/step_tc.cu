@@ -12,7 +12,8 @@
 //   k_finalize         lambda, ||S_prev||, t (Eq. 12)
 //   k_tc_form_x        X = a_low N - a_res lambda k_l R  (bf16).  In the plain step the projection
 //                      epilogue has written X for lambda = 1 already (see tc_project.cuh) and this
-//                      kernel only touches the matrices whose limiter acted: X += a_res (1 - lambda) k_l R
+//                      kernel only touches the matrices whose limiter acted (k_tc_fix_x):
+//                      X <- lambda X + (1 - lambda) a_low N, N rebuilt from the stored moments
 //   k_tc_back_project  D = Pi X on the tensor cores; epilogue: W -= lr (D + a_res lambda k_l G)
 //
 // ||S_l||^2 = ||G_l - Pi R_l||^2 = ||G_l||^2 - 2 ||R_l||^2 + R_l^T (Pi^T Pi) R_l.  For orthonormal
@@ -265,10 +266,13 @@ k_tc_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int n
 }
 
 // The matrices whose X the projection epilogue has formed for lambda = 1 (FUSE_X): where the limiter
-// acted, X += a_res (1 - lambda) k_l R; the others are left as they are.  blockIdx.y = matrix of the
-// range, the blocks of a matrix stride over its rows, one warp per row.
+// acted, X_lambda = a_low N - a_res lambda k_l R = lambda X + (1 - lambda) a_low N, with N rebuilt
+// from the moments that the epilogue stored, by the epilogue's own arithmetic and rounded to bf16
+// as it was there; the other matrices are left as they are.  blockIdx.y = matrix of the range, the
+// blocks of a matrix stride over its rows, one warp per row.
 __global__ void __launch_bounds__(256)
-k_tc_fix_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int first, float a_res, float* __restrict__ fast) {
+k_tc_fix_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int first, float a_low, float eps,
+           float* __restrict__ fast) {
   const int p = first + blockIdx.y;
   const MatDev& mt = mats[list[p]];
   if (!fuse_x_matrix(mt.d, mt.r)) return;              // k_tc_form_x's matrix
@@ -276,17 +280,23 @@ k_tc_fix_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int fi
   if (blockIdx.x == 0 && threadIdx.x == 0) fast[2 * p + 1] = lambda;   // read by the back-projection epilogue
   if (lambda == 1.f) return;
   const int lane = threadIdx.x & 31;
+  const float bias = fast[2 * p];                      // this step's bias factor (k_tc_prep)
+  const float cn = (1.f - lambda) * a_low;
   for (int l = blockIdx.x * 8 + (threadIdx.x >> 5); l < mt.l; l += gridDim.x * 8) {
-    const float c = a_res * (1.f - lambda) * mt.kvec[l];
     const long long base = (long long)l * mt.r;
     for (int j = lane * 8; j < mt.r; j += 256) {
       const uint4 xu = *reinterpret_cast<const uint4*>(mt.Xb + base + j);
-      const uint4 ru = *reinterpret_cast<const uint4*>(mt.Rb + base + j);
-      float xv[8], rv[8], x[8];
+      const float4 m0 = *reinterpret_cast<const float4*>(mt.M + base + j), m1 = *reinterpret_cast<const float4*>(mt.M + base + j + 4);
+      const float4 v0 = *reinterpret_cast<const float4*>(mt.V + base + j), v1 = *reinterpret_cast<const float4*>(mt.V + base + j + 4);
+      const float mo[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+      const float vo[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+      float xv[8], x[8];
       unpack8_bf16(xu, xv);
-      unpack8_bf16(ru, rv);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) x[e] = xv[e] + c * rv[e];
+      for (int e = 0; e < 8; ++e) {
+        const float nv = __bfloat162float(__float2bfloat16_rn(__fdividef(bias * mo[e], fast_sqrt(vo[e]) + eps)));
+        x[e] = lambda * xv[e] + cn * nv;
+      }
       *reinterpret_cast<uint4*>(mt.Xb + base + j) = pack8_bf16(x);
     }
   }
@@ -678,11 +688,10 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
   if (!pl || pl->nlist == 0) return 0;
   cudaStream_t st = c->stream;
   if (!pl->attrs_set) {
-    const void* k1s[6] = {(const void*)k_tc_project<EPI_ADAM, PSI_ADAM, 0>, (const void*)k_tc_project<EPI_ADAM, PSI_RMSPROP, 0>,
-                          (const void*)k_tc_project<EPI_ADAM, PSI_ADAGRAD, 0>, (const void*)k_tc_project<EPI_ADAM, PSI_ADAM, 1>,
-                          (const void*)k_tc_project<EPI_ADAM, PSI_RMSPROP, 1>, (const void*)k_tc_project<EPI_ADAM, PSI_ADAGRAD, 1>};
+    const void* k1s[4] = {(const void*)k_tc_project<EPI_ADAM, PSI_ADAM, 0>, (const void*)k_tc_project<EPI_ADAM, PSI_RMSPROP, 0>,
+                          (const void*)k_tc_project<EPI_ADAM, PSI_ADAGRAD, 0>, (const void*)k_tc_project<EPI_ADAM, PSI_ADAM, 1>};
     cudaError_t e1 = cudaSuccess;
-    for (int i = 0; i < 6 && e1 == cudaSuccess; ++i)
+    for (int i = 0; i < 4 && e1 == cudaSuccess; ++i)
       e1 = cudaFuncSetAttribute(k1s[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
     cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project<5, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)k2_smem_bytes(5, 2));
     if (e2 == cudaSuccess)
@@ -737,16 +746,18 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
   k_tc_prep<<<nq, 32, 0, st>>>(mats, pl->list, qa, hp, pl->fast_dev);
   tm->mark(st);
   // both tensor kernels: clusters of two CTAs, at most one CTA per SM
-  // the plain step (column factors, residual kept) forms X in the projection epilogue
-  const bool fused = (hp.mode & (HYPER_MATRIX_SCALING | HYPER_NO_SCALING | HYPER_NO_RESIDUAL | HYPER_ONLY_SCALING)) == 0;
+  // the plain step (Adam, column factors, residual kept) forms X in the projection epilogue
+  const bool fused = (hp.mode & (HYPER_MATRIX_SCALING | HYPER_NO_SCALING | HYPER_NO_RESIDUAL | HYPER_ONLY_SCALING |
+                                 HYPER_PSI_RMSPROP | HYPER_PSI_ADAGRAD)) == 0;
   const int k1_grid = 2 * std::min(k1n, fused ? pl->max_pairs_fused : pl->num_sms / 2);
   const ProjTileDesc* td1 = pl->td1_dev + k1a;
 #define FIRA_LAUNCH_K1(PSI, FUSE)                                                     \
   k_tc_project<EPI_ADAM, PSI, FUSE><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(      \
       pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev)
-  if (hp.mode & HYPER_PSI_RMSPROP) { if (fused) FIRA_LAUNCH_K1(PSI_RMSPROP, 1); else FIRA_LAUNCH_K1(PSI_RMSPROP, 0); }
-  else if (hp.mode & HYPER_PSI_ADAGRAD) { if (fused) FIRA_LAUNCH_K1(PSI_ADAGRAD, 1); else FIRA_LAUNCH_K1(PSI_ADAGRAD, 0); }
-  else { if (fused) FIRA_LAUNCH_K1(PSI_ADAM, 1); else FIRA_LAUNCH_K1(PSI_ADAM, 0); }
+  if (hp.mode & HYPER_PSI_RMSPROP) FIRA_LAUNCH_K1(PSI_RMSPROP, 0);
+  else if (hp.mode & HYPER_PSI_ADAGRAD) FIRA_LAUNCH_K1(PSI_ADAGRAD, 0);
+  else if (fused) FIRA_LAUNCH_K1(PSI_ADAM, 1);
+  else FIRA_LAUNCH_K1(PSI_ADAM, 0);
 #undef FIRA_LAUNCH_K1
   tm->mark(st);
   k_tc_colfactors<<<csn, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->col_start, csa, hp);
@@ -771,7 +782,7 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
   if (any_plain)
     k_tc_form_x<<<(rsb - rsa + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start, rsa, rsb,
                                                      hp.a_low, hp.a_res, pl->fast_dev, fused ? 1 : 0);
-  if (any_fused) k_tc_fix_x<<<dim3(64, nq), 256, 0, st>>>(mats, pl->list, qa, hp.a_res, pl->fast_dev);
+  if (any_fused) k_tc_fix_x<<<dim3(64, nq), 256, 0, st>>>(mats, pl->list, qa, hp.a_low, hp.eps, pl->fast_dev);
   tm->mark(st);
   // long products keep five operand stages; short ones trade one for more epilogue boxes in flight
   int rmax = 0;

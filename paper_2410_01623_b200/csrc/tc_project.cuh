@@ -54,8 +54,9 @@
 // follows, on its pair, a tile far below it, so the waits cannot form a cycle as long as every block
 // of the grid is resident, which the launch ensures), the thread adds the partial sums in the fixed
 // order that k_tc_colfactors uses, and sweep 2 reads the pairs back and writes X (through the map of
-// the X buffer) and R (bf16, needed only where the limiter acts: there k_tc_form_x adds
-// a_res (1 - lambda) k_l R to X).
+// the X buffer).  Nothing else leaves the kernel: where the limiter acts, k_tc_fix_x rebuilds N from
+// the stored moments, X_lambda = lambda X + (1 - lambda) a_low N.  (Adam only: with RMSProp or Adagrad
+// N cannot be rebuilt from V alone, and those steps keep the separate pass.)
 constexpr int K1_STAGES = 4;
 constexpr int K1_STAGE_BYTES = 2 * A_STAGE_BYTES;       // A: 128 l x 64 d, B half: 128 r x 64 d
 constexpr int K1_ECOLS = 32;                            // columns per epilogue box
@@ -117,7 +118,7 @@ struct ProjCtl {
   uint64_t eready[K1_MVBUFS];   // the epilogue has finished M, V (in place) and N, R of a box
   uint64_t eempty[K1_MVBUFS];   // the stores have read M and V: the buffer is free
   uint64_t nrempty[K1_NRBUFS];  // the stores have read N and R: the buffer is free
-  uint64_t xready[K1_NRBUFS];   // FUSE_X: a row half has finished an X box and an R box
+  uint64_t xready[K1_NRBUFS];   // FUSE_X: a row half has finished an X box
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -439,7 +440,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           if (++mv == K1_MVBUFS) { mv = 0; mvphase ^= 1u; }
         }
         if (fuse && ok) {
-          // second sweep of the epilogue: the X and R boxes of this tile, in the same order
+          // second sweep of the epilogue: the X boxes of this tile, in the same order
           for (int b = 0; b < 2 * (bn / K1_ECOLS); ++b) {
             const int nr = b & 1;
             if (!ptx::mbar_wait(ptx::smem_u32(&ctl->xready[nr]), (xphase >> nr) & 1u, abort_flag)) { ok = false; break; }
@@ -448,7 +449,6 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
             if (row < d.L) {
               const uint32_t srn = nrbuf_u32 + nr * K1_NRBUF_BYTES;
               ptx::tma_store_2d(&mp->ex, srn, j, row);
-              ptx::tma_store_2d(&mp->er, srn + K1_HBOX_BYTES, j, row);
               ptx::bulk_commit_group();
               ptx::bulk_wait_group_read<0>();
             }
@@ -612,7 +612,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         }
         const float kl = (l < d.L) ? sqrtf(nt) / (sqrtf(rt) + hp.eps) : 0.f;
         const float ck = hp.a_res * 1.0f * kl;           // k_tc_form_x's coefficient at lambda = 1
-        // ---- sweep 2: X = a_low N - a_res k_l R and R itself, as bf16 boxes
+        // ---- sweep 2: X = a_low N - a_res k_l R as bf16 boxes
         for (int c = 0; c < nch; ++c) {
           uint32_t rr[32];
           __syncwarp();
@@ -626,16 +626,13 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           if (!ptx::mbar_wait(nrempty, nrphase ^ 1u, abort_flag)) { ok = false; break; }
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            float xv[8], rv[8];
+            float xv[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
               const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&rr[8 * q + e]));
-              rv[e] = f.y;
               xv[e] = hp.a_low * f.x - ck * f.y;
             }
-            const uint32_t h = hrow + (((uint32_t)q ^ hsw) << 4);
-            *reinterpret_cast<uint4*>(nb + h) = pack8_bf16(xv);
-            *reinterpret_cast<uint4*>(rb + h) = pack8_bf16(rv);
+            *reinterpret_cast<uint4*>(nb + hrow + (((uint32_t)q ^ hsw) << 4)) = pack8_bf16(xv);
           }
           ptx::fence_proxy_async_smem();
           ptx::mbar_arrive(ptx::smem_u32(&ctl->xready[half]));
