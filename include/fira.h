@@ -231,8 +231,9 @@ FIRA_API fira_status fira_poll(fira_ctx* ctx);
 /* Self-test of the failure path of the tensor-core kernels (the paper has no counterpart).  Every
  * wait inside those kernels is bounded: a wait that runs out raises a flag that all roles of the
  * block poll, the kernel returns, and the time-out shows up in fira_poll().  This call enqueues a
- * one-block kernel whose wait can never be satisfied (a barrier that nothing arrives on, no copy in
- * flight) with a limit of `rounds` tries (1 .. 2^20), so that the path can be exercised without
+ * one-block kernel whose waits can never be satisfied (a barrier that nothing arrives on, no copy in
+ * flight; a counter in global memory that nothing raises, the form in which the projection epilogues
+ * wait for one another) with a limit of `rounds` tries (1 .. 2^20), so that the path can be exercised without
  * disturbing anything: afterwards fira_poll() returns FIRA_ERR_DEVICE_TIMEOUT once, then FIRA_OK,
  * and the context steps on as before. */
 FIRA_API fira_status fira_selftest_bounded_wait(fira_ctx* ctx, int32_t rounds);

@@ -305,9 +305,11 @@ k_tc_fix_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int fi
 // Self-test of the bounded waits: thread 0 waits on a barrier that nothing ever arrives on and gives
 // up after `rounds` tries, raising the abort flag; a thread of the second warp sits in a wait with
 // the ordinary limit, as the other roles of the product kernels do, and must leave when it sees the
-// flag.  No copy is in flight and nothing else is touched.
-__global__ void __launch_bounds__(64)
-k_selftest_bounded_wait(unsigned* __restrict__ status, uint32_t rounds) {
+// flag; a thread of the third warp polls a counter in global memory that nothing ever raises (the
+// wait of the projection epilogues for the partial sums of their row of tiles) with the same small
+// limit.  No copy is in flight and nothing else is touched.
+__global__ void __launch_bounds__(96)
+k_selftest_bounded_wait(unsigned* status, const uint32_t* never_raised, uint32_t rounds) {
   __shared__ uint64_t bars[2];
   __shared__ int abort_flag;
   if (threadIdx.x == 0) {
@@ -320,8 +322,10 @@ k_selftest_bounded_wait(unsigned* __restrict__ status, uint32_t rounds) {
   bool got = true;
   if (threadIdx.x == 0) got = ptx::mbar_wait(ptx::smem_u32(&bars[0]), 0, &abort_flag, rounds);
   if (threadIdx.x == 32) got = ptx::mbar_wait(ptx::smem_u32(&bars[1]), 0, &abort_flag);
+  __shared__ int counter_gave_up;
+  if (threadIdx.x == 64) counter_gave_up = ptx::wait_counter(never_raised, 0xffffffffu, &abort_flag, rounds) ? 0 : 1;
   __syncthreads();
-  if (threadIdx.x == 0 && !got && abort_flag) atomicOr(status, DEV_STATUS_TIMEOUT);
+  if (threadIdx.x == 0 && !got && abort_flag && counter_gave_up) atomicOr(status, DEV_STATUS_TIMEOUT);
 }
 
 // ============================================================================ host side
@@ -670,7 +674,8 @@ fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntile
 }
 
 fira_status tc_selftest_bounded_wait(fira_ctx* c, int rounds) {
-  k_selftest_bounded_wait<<<1, 64, 0, c->stream>>>(c->status_dev, (uint32_t)rounds);
+  // the status word itself serves as the counter that never reaches its target
+  k_selftest_bounded_wait<<<1, 96, 0, c->stream>>>(c->status_dev, c->status_dev, (uint32_t)rounds);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_error(std::string("bounded-wait self-test: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
   return FIRA_OK;

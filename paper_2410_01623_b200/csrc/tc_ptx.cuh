@@ -169,8 +169,9 @@ __device__ __forceinline__ void signal_counter(uint32_t* p) {
 }
 // Waits until *p >= target.  Returns false if the wait ran out (the abort flag is then raised) or
 // the block is aborting.  The pause keeps the poll off the memory system.
-__device__ __forceinline__ bool wait_counter(const uint32_t* p, uint32_t target, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < (1u << 21); ++it) {
+__device__ __forceinline__ bool wait_counter(const uint32_t* p, uint32_t target, volatile int* abort_flag,
+                                             uint32_t limit = 1u << 21) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (ld_acquire_gpu(p) >= target) return true;
     __nanosleep(it < 64 ? 64 : 256);
     if ((it & 63u) == 63u && *abort_flag) return false;
