@@ -787,7 +787,7 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
   if (any_plain)
     k_tc_form_x<<<(rsb - rsa + 7) / 8, 256, 0, st>>>(mats, pl->list, pl->nlist, pl->row_start, rsa, rsb,
                                                      hp.a_low, hp.a_res, pl->fast_dev, fused ? 1 : 0);
-  if (any_fused) k_tc_fix_x<<<dim3(64, nq), 256, 0, st>>>(mats, pl->list, qa, hp.a_low, hp.eps, pl->fast_dev);
+  if (any_fused) k_tc_fix_x<<<dim3(16, nq), 256, 0, st>>>(mats, pl->list, qa, hp.a_low, hp.eps, pl->fast_dev);
   tm->mark(st);
   // long products keep five operand stages; short ones trade one for more epilogue boxes in flight
   int rmax = 0;
