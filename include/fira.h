@@ -204,6 +204,23 @@ FIRA_API fira_status fira_refresh_projection_f32(fira_ctx* ctx, const void* cons
                                                  const int32_t* which, int32_t nwhich, uint64_t seed,
                                                  int32_t iters, float* const* basis_f32_dev);
 
+/* Eq. 7 beside the steps (the section on gradient low-rank projection notes that the refresh costs
+ * little when it runs only every T steps; this entry point takes it off the step's stream altogether).  The
+ * same iteration as fira_refresh_projection(), but nothing of the context is modified: it works in
+ * work_dev (256-byte aligned, at least fira_refresh_side_work_bytes() bytes: room for the largest
+ * matrix; more room lets it take several matrices per pass), enqueues on side_stream (a cudaStream_t
+ * other than the context's) and writes the basis of every selected matrix i to P_out_dev[i] (a host
+ * array of `count` device pointers, d x r in the matrix's dtype, 16-byte aligned).  The call may be
+ * made from another host thread while fira_step() runs on the context's stream (it reads only what
+ * fira_init() fixed); it waits for side_stream before returning.  To adopt a basis, order the
+ * context's stream after side_stream and call fira_set_projection().  Same seed, same gradients:
+ * the same bases as fira_refresh_projection(), bit for bit. */
+FIRA_API size_t fira_refresh_side_work_bytes(const fira_ctx* ctx);
+FIRA_API fira_status fira_refresh_projection_side(fira_ctx* ctx, const void* const* G_dev,
+                                                  const int32_t* which, int32_t nwhich, uint64_t seed,
+                                                  int32_t iters, void* const* P_out_dev, void* work_dev,
+                                                  size_t work_bytes, void* side_stream);
+
 /* Copy a projection (d x r, row major, the matrix's dtype) from / to device memory
  * (the P_t of Algorithm 1, given by the caller instead of Eq. 7). */
 FIRA_API fira_status fira_set_projection(fira_ctx* ctx, int32_t idx, const void* P_dev);

@@ -64,6 +64,10 @@ SIGNATURES = {
                                           C.c_int32, C.c_uint64, C.c_int32]),
     "fira_refresh_projection_f32": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_int32),
                                               C.c_int32, C.c_uint64, C.c_int32, C.POINTER(C.c_void_p)]),
+    "fira_refresh_side_work_bytes": (C.c_size_t, [C.c_void_p]),
+    "fira_refresh_projection_side": (C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_int32), C.c_int32,
+                                               C.c_uint64, C.c_int32, C.POINTER(C.c_void_p), C.c_void_p,
+                                               C.c_size_t, C.c_void_p]),
     "fira_set_projection": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "fira_get_projection": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]),
     "fira_get_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_float),
@@ -239,6 +243,22 @@ class Fira:
                                      b.shape == (self._dl(i)[0], self.ranks[i]))
             check(self.L.fira_refresh_projection_f32(self.ctx, ptr_array(Gs), w, nw, seed, iters,
                                                      ptr_array(basis_f32)))
+
+    def refresh_side_work_bytes(self) -> int:
+        return self.L.fira_refresh_side_work_bytes(self.ctx)
+
+    def refresh_projection_side(self, Gs: Sequence[Optional[torch.Tensor]], P_out: Sequence[Optional[torch.Tensor]],
+                                work: torch.Tensor, stream: "torch.cuda.Stream",
+                                which: Optional[Sequence[int]] = None, seed: int = 0, iters: int = -1):
+        """The refresh on a side stream with its own work buffer; the bases go to P_out (one (d, r)
+        tensor of the storage type per selected matrix) and the context is left as it is."""
+        w, nw = (None, 0) if which is None else ((C.c_int32 * len(which))(*which), len(which))
+        for i, p in enumerate(P_out):
+            assert p is None or (p.dtype == self.dtype and p.is_contiguous() and
+                                 p.shape == (self._dl(i)[0], self.ranks[i]))
+        check(self.L.fira_refresh_projection_side(self.ctx, ptr_array(Gs), w, nw, seed, iters, ptr_array(P_out),
+                                                  work.data_ptr(), work.numel() * work.element_size(),
+                                                  stream.cuda_stream))
 
     def set_projection(self, idx: int, P: torch.Tensor):
         d, _ = self._dl(idx)

@@ -67,7 +67,18 @@ Layout make_layout(const fira_hparams& hp, const fira_matrix_desc* descs, int32_
 size_t refresh_bytes_per_matrix(const fira_matrix_desc& d);
 int engine_for(const fira_hparams& hp, const fira_matrix_desc& d);
 
+// Where a refresh works and where its result goes.  Default: the context's own work area and
+// stream, the bases stored into the context's projections.  The side variant: a work buffer and a
+// stream of the caller's, the bases written to the caller's buffers (per matrix index, in the
+// matrix's storage type) and nothing of the context modified, so that it may run next to steps.
+struct RefreshTarget {
+  char* work_base = nullptr;
+  size_t work_bytes = 0;
+  cudaStream_t stream = nullptr;
+  void* const* P_out = nullptr;      // null: the context's projections
+};
 fira_status refresh_impl(fira_ctx* ctx, const void* const* G_dev, const std::vector<int>& which,
-                         uint64_t seed, int iters, float* const* basis_out = nullptr);
+                         uint64_t seed, int iters, float* const* basis_out = nullptr,
+                         const RefreshTarget* target = nullptr);
 
 }  // namespace fira

@@ -488,6 +488,41 @@ fira_status fira_refresh_projection_f32(fira_ctx* c, const void* const* G_dev, c
   return refresh_impl(c, G_dev, sel, seed, iters, basis_f32_dev);
 }
 
+size_t fira_refresh_side_work_bytes(const fira_ctx* c) {
+  if (!c) return 0;
+  size_t mx = 0;
+  for (const fira_matrix_desc& d : c->descs) mx = std::max(mx, refresh_bytes_per_matrix(d));
+  return align_up(mx);
+}
+
+fira_status fira_refresh_projection_side(fira_ctx* c, const void* const* G_dev, const int32_t* which, int32_t nwhich,
+                                         uint64_t seed, int32_t iters, void* const* P_out_dev, void* work_dev,
+                                         size_t work_bytes, void* side_stream) {
+  if (!c || !G_dev || !P_out_dev || !work_dev) { set_error("null argument"); return FIRA_ERR_INVALID_ARG; }
+  const int count = (int)c->mats.size();
+  std::vector<int> sel;
+  if (!which) { for (int i = 0; i < count; ++i) sel.push_back(i); }
+  else {
+    if (nwhich < 0) { set_error("nwhich < 0"); return FIRA_ERR_INVALID_ARG; }
+    for (int q = 0; q < nwhich; ++q) {
+      if (which[q] < 0 || which[q] >= count) { set_error("matrix index out of range"); return FIRA_ERR_INVALID_ARG; }
+      sel.push_back(which[q]);
+    }
+  }
+  for (int i : sel) {
+    if (!G_dev[i] || ((uintptr_t)G_dev[i] & 15)) { set_error("G must be non-null and 16-byte aligned"); return FIRA_ERR_INVALID_ARG; }
+    if (!P_out_dev[i] || ((uintptr_t)P_out_dev[i] & 15)) { set_error("projection output must be non-null and 16-byte aligned"); return FIRA_ERR_INVALID_ARG; }
+  }
+  if (((uintptr_t)work_dev & 255) || work_bytes < fira_refresh_side_work_bytes(c)) {
+    set_error("work buffer must be 256-byte aligned and hold fira_refresh_side_work_bytes() bytes");
+    return FIRA_ERR_WORKSPACE_TOO_SMALL;
+  }
+  if (sel.empty()) return FIRA_OK;
+  RefreshTarget tg;
+  tg.work_base = (char*)work_dev; tg.work_bytes = work_bytes; tg.stream = (cudaStream_t)side_stream; tg.P_out = P_out_dev;
+  return refresh_impl(c, G_dev, sel, seed, iters, nullptr, &tg);
+}
+
 static fira_status check_idx(const fira_ctx* c, int32_t idx) {
   if (!c) { set_error("null context"); return FIRA_ERR_INVALID_ARG; }
   if (idx < 0 || idx >= (int)c->mats.size()) { set_error("matrix index out of range"); return FIRA_ERR_INVALID_ARG; }

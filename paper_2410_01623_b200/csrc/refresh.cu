@@ -444,10 +444,13 @@ size_t refresh_bytes_per_matrix(const fira_matrix_desc& d) {
 // basis_out (may be null): per matrix index an optional device pointer that receives the kept
 // basis in fp32 (d x r) before it is rounded to the storage type.
 fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vector<int>& which,
-                         uint64_t seed, int iters, float* const* basis_out) {
+                         uint64_t seed, int iters, float* const* basis_out, const RefreshTarget* target) {
   if (iters < 0) iters = 4;
-  c->proj_weights_dirty = true;
-  cudaStream_t st = c->stream;
+  RefreshTarget own;
+  own.work_base = c->work_base; own.work_bytes = c->work_bytes; own.stream = c->stream;
+  const RefreshTarget& tg = target ? *target : own;
+  if (!tg.P_out) c->proj_weights_dirty = true;
+  cudaStream_t st = tg.stream;
   size_t pos = 0;
   while (pos < which.size()) {
     // ---- carve a chunk: as many matrices as fit (data regions first, then tables)
@@ -455,7 +458,7 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     size_t off = 0, q = pos;
     for (; q < which.size(); ++q) {
       const size_t data = refresh_data_bytes(c->descs[which[q]]);
-      if (off + data + (q - pos + 1) * TABLE_PER_MATRIX + TABLE_SLACK > c->work_bytes) break;
+      if (off + data + (q - pos + 1) * TABLE_PER_MATRIX + TABLE_SLACK > tg.work_bytes) break;
       offs.push_back(off);
       off += data;
     }
@@ -468,9 +471,9 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
       const MatDev& mt = c->mats[idx];
       RefreshMat rm;
       memset(&rm, 0, sizeof(rm));
-      rm.G = G_dev[idx]; rm.P = mt.P;
+      rm.G = G_dev[idx]; rm.P = tg.P_out ? tg.P_out[idx] : mt.P;
       rm.out32 = basis_out ? basis_out[idx] : nullptr;
-      char* base = c->work_base + offs[a];
+      char* base = tg.work_base + offs[a];
       const size_t r = mt.r;
       rm.Y = (float*)base; base += align_up((size_t)mt.d * r * 4);
       rm.Z = (float*)base; base += align_up((size_t)mt.l * r * 4);
@@ -486,7 +489,7 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
         rm.Ub = (__nv_bfloat16*)base; base += align_up(r * r * 2);
         rm.Ul = (__nv_bfloat16*)base; base += align_up(r * r * 2);
       }
-      data_end = std::max(data_end, (size_t)(base - c->work_base));
+      data_end = std::max(data_end, (size_t)(base - tg.work_base));
       rm.ld = mt.ld; rm.d = mt.d; rm.l = mt.l; rm.r = mt.r; rm.left = mt.left; rm.bf16 = mt.bf16;
       rm.key = seed * 0x9E3779B97F4A7C15ull + (unsigned long long)idx * 0xD1B54A32D192ED03ull + 1ull;
       rms.push_back(rm);
@@ -535,12 +538,12 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
       tY.push_back(TrsmDesc{m.Y, m.C, m.d, m.r}); sTY.push_back(sTY.back() + (m.d + TM - 1) / TM);
       tZ.push_back(TrsmDesc{m.Z, m.C, m.l, m.r}); sTZ.push_back(sTZ.back() + (m.l + TM - 1) / TM);
     }
-    char* tp = c->work_base + align_up(data_end);
+    char* tp = tg.work_base + align_up(data_end);
     cudaError_t cerr = cudaSuccess;
     auto put = [&](const void* src, size_t bytes) -> char* {
       char* dst = tp;
       if (bytes == 0) return dst;
-      if ((size_t)(tp + align_up(bytes) - c->work_base) > c->work_bytes) { cerr = cudaErrorInvalidValue; return dst; }
+      if ((size_t)(tp + align_up(bytes) - tg.work_base) > tg.work_bytes) { cerr = cudaErrorInvalidValue; return dst; }
       cudaError_t e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st);
       if (e != cudaSuccess) cerr = e;
       tp += align_up(bytes);
@@ -568,11 +571,11 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     if (ntc) {
       for (int k = 0; k < JOB_KINDS; ++k) {
         const size_t bytes = tc_gemm_table_bytes(jobs[k].data(), ntc);
-        if ((size_t)(tp + bytes - c->work_base) > c->work_bytes) {
+        if ((size_t)(tp + bytes - tg.work_base) > tg.work_bytes) {
           set_error("scratch buffer too small for the projection refresh"); return FIRA_ERR_WORKSPACE_TOO_SMALL;
         }
         tab[k] = tp;
-        const fira_status ps = tc_gemm_prepare(c, jobs[k].data(), ntc, tab[k], bytes, &jtiles[k]);
+        const fira_status ps = tc_gemm_prepare(c, jobs[k].data(), ntc, tab[k], bytes, &jtiles[k], st);
         if (ps != FIRA_OK) return ps;
         tp += bytes;
       }
@@ -589,7 +592,7 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
       if (ntc) {
         k_split_bf16<<<ew_grid, 256, 0, st>>>(rm_dev, az ? 1 : 0, precise ? 1 : 0);
         const int k = az ? (precise ? JOB_AZ_SPLIT : JOB_AZ) : (precise ? JOB_ATY_SPLIT : JOB_ATY);
-        return tc_gemm_run(c, tab[k], ntc, jtiles[k]);
+        return tc_gemm_run(c, tab[k], ntc, jtiles[k], st);
       }
       return FIRA_OK;
     };
@@ -601,7 +604,7 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
         if (nsimt) k_rgemm<<<sYY.back(), GEMM_THREADS, 0, st>>>(y ? dYY : dZZ, nsimt, dsYY);
         if (ntc) {
           k_split_bf16<<<ew_grid, 256, 0, st>>>(rm_dev, y ? 0 : 1, 1);
-          const fira_status gs = tc_gemm_run(c, tab[y ? JOB_GRAM_Y : JOB_GRAM_Z], ntc, jtiles[y ? JOB_GRAM_Y : JOB_GRAM_Z]);
+          const fira_status gs = tc_gemm_run(c, tab[y ? JOB_GRAM_Y : JOB_GRAM_Z], ntc, jtiles[y ? JOB_GRAM_Y : JOB_GRAM_Z], st);
           if (gs != FIRA_OK) return gs;
         }
         for (int J0 = 0; J0 < rmax; J0 += CB) {
@@ -620,7 +623,7 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
           k_identity<<<ew_grid, 256, 0, st>>>(rm_dev);
           k_trsm_rows<<<sTU.back(), GEMM_THREADS, 0, st>>>(dTU, ntc, dsTU);      // U = L^-T
           k_split_bf16<<<ew_grid, 256, 0, st>>>(rm_dev, 2, 1);
-          const fira_status as = tc_gemm_run(c, tab[y ? JOB_APPLY_Y : JOB_APPLY_Z], ntc, jtiles[y ? JOB_APPLY_Y : JOB_APPLY_Z]);
+          const fira_status as = tc_gemm_run(c, tab[y ? JOB_APPLY_Y : JOB_APPLY_Z], ntc, jtiles[y ? JOB_APPLY_Y : JOB_APPLY_Z], st);
           if (as != FIRA_OK) return as;
         }
       }

@@ -605,7 +605,7 @@ size_t tc_gemm_table_bytes(const TcGemmJob* jobs, int njobs) {
 }
 
 fira_status tc_gemm_prepare(fira_ctx* c, const TcGemmJob* jobs, int njobs, char* table_dev, size_t table_bytes,
-                            int* ntiles_out) {
+                            int* ntiles_out, cudaStream_t st) {
   if (tc_gemm_table_bytes(jobs, njobs) > table_bytes) { set_error("refresh: table area too small"); return FIRA_ERR_WORKSPACE_TOO_SMALL; }
   std::vector<TcMaps> maps((size_t)njobs);
   std::vector<ProjTileDesc> tiles;
@@ -644,15 +644,15 @@ fira_status tc_gemm_prepare(fira_ctx* c, const TcGemmJob* jobs, int njobs, char*
       }
   }
   char* tiles_dev = table_dev + align_up(sizeof(TcMaps) * (size_t)njobs);
-  cudaError_t e = cudaMemcpyAsync(table_dev, maps.data(), sizeof(TcMaps) * maps.size(), cudaMemcpyHostToDevice, c->stream);
+  cudaError_t e = cudaMemcpyAsync(table_dev, maps.data(), sizeof(TcMaps) * maps.size(), cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess)
-    e = cudaMemcpyAsync(tiles_dev, tiles.data(), sizeof(ProjTileDesc) * tiles.size(), cudaMemcpyHostToDevice, c->stream);
+    e = cudaMemcpyAsync(tiles_dev, tiles.data(), sizeof(ProjTileDesc) * tiles.size(), cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) { set_error(std::string("refresh tables: ") + cudaGetErrorString(e)); return FIRA_ERR_CUDA; }
   *ntiles_out = (int)tiles.size();
   return FIRA_OK;
 }
 
-fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntiles) {
+fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntiles, cudaStream_t st) {
   // the shared-memory attribute of a kernel is a per-device setting
   static int sms_of_device[64] = {};
   if (c->device < 0 || c->device >= 64) { set_error("refresh product: device index out of range"); return FIRA_ERR_CUDA; }
@@ -668,7 +668,7 @@ fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntile
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(table_dev);
   const ProjTileDesc* tiles = reinterpret_cast<const ProjTileDesc*>(table_dev + align_up(sizeof(TcMaps) * (size_t)njobs));
   Hyper hp{};
-  k_tc_project<EPI_PLAIN, PSI_ADAM, 0><<<2 * std::min(ntiles, num_sms / 2), K1_THREADS, K1_SMEM_BYTES, c->stream>>>(
+  k_tc_project<EPI_PLAIN, PSI_ADAM, 0><<<2 * std::min(ntiles, num_sms / 2), K1_THREADS, K1_SMEM_BYTES, st>>>(
       maps, tiles, ntiles, nullptr, nullptr, nullptr, hp, c->status_dev);
   return FIRA_OK;
 }

@@ -52,11 +52,11 @@ struct TcGemmJob {
 };
 // Device bytes of the tables (tensor maps, tile records) of a job list.
 size_t tc_gemm_table_bytes(const TcGemmJob* jobs, int njobs);
-// Builds the tables on the host and uploads them to table_dev (256-byte aligned) on the context's
+// Builds the tables on the host and uploads them to table_dev (256-byte aligned) on the given
 // stream; *ntiles_out is what tc_gemm_run needs.
 fira_status tc_gemm_prepare(fira_ctx* c, const TcGemmJob* jobs, int njobs, char* table_dev, size_t table_bytes,
-                            int* ntiles_out);
+                            int* ntiles_out, cudaStream_t st);
 // One grouped launch over the prepared jobs.
-fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntiles);
+fira_status tc_gemm_run(fira_ctx* c, const char* table_dev, int njobs, int ntiles, cudaStream_t st);
 
 }  // namespace fira

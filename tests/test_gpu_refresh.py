@@ -162,3 +162,82 @@ def test_auto_refresh_flag_follows_t_mod_T():
     assert torch.equal(seen[0], seen[1])                 # kept at t = 1
     assert not torch.equal(seen[1], seen[2])             # refreshed at t = 2
     assert torch.equal(seen[2], seen[3])
+
+
+def _side_case(dtype):
+    shapes = [(512, 1024), (1024, 512), (300, 333)] if dtype == torch.bfloat16 else [(200, 333), (333, 200)]
+    r = [128, 128, 37] if dtype == torch.bfloat16 else [50, 50]
+    g = torch.Generator().manual_seed(21)
+    Gs = [torch.randn(m, n, generator=g).to(dtype).cuda() for (m, n) in shapes]
+    return shapes, r, Gs
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_side_stream_refresh_gives_the_same_bases_and_leaves_the_context_alone(dtype):
+    """fira_refresh_projection_side: own work buffer (the smallest allowed, so the list goes through
+    it one matrix at a time), own stream, bases written to the caller's tensors: bit for bit the
+    bases of the in-place refresh with the same seed, and the context's projections untouched until
+    the caller sets them."""
+    shapes, r, Gs = _side_case(dtype)
+    ref = fb.Fira(shapes, r, dtype, fb.make_hparams())
+    ref.refresh_projection(Gs, seed=77, iters=3)
+    f = fb.Fira(shapes, r, dtype, fb.make_hparams())
+    work = torch.empty(f.refresh_side_work_bytes(), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    P_out = [torch.zeros(min(m, n), r[i], dtype=dtype, device="cuda") for i, (m, n) in enumerate(shapes)]
+    torch.cuda.synchronize()
+    f.refresh_projection_side(Gs, P_out, work, side, seed=77, iters=3)
+    assert f.poll() == 0
+    for i in range(len(shapes)):
+        assert torch.equal(P_out[i], ref.get_projection(i))
+        assert f.get_projection(i).abs().max() == 0
+    with pytest.raises(fb.FiraError):
+        f.refresh_projection_side(Gs, P_out, work[:1024], side, seed=77)
+
+
+def test_side_stream_refresh_runs_beside_steps():
+    """A host thread refreshes on a side stream while the main thread keeps stepping with the old
+    projection: the steps give bit for bit what they give alone, the refreshed bases are those of a
+    refresh that ran by itself, and adopting them works as set_projection always does."""
+    import threading
+    dtype = torch.bfloat16
+    shapes, r, Gs = _side_case(dtype)
+    hp = fb.make_hparams(lr=1e-2)
+    g = torch.Generator().manual_seed(5)
+    W0 = [(torch.randn(m, n, generator=g) * 0.02).to(dtype).cuda() for (m, n) in shapes]
+    P0 = [torch.linalg.qr(torch.randn(min(m, n), r[i], generator=g, dtype=torch.float64))[0].to(dtype).cuda()
+          for i, (m, n) in enumerate(shapes)]
+    steps = 40
+
+    def run(with_refresh):
+        f = fb.Fira(shapes, r, dtype, hp)
+        for i in range(len(shapes)):
+            f.set_projection(i, P0[i])
+        W = [w.clone() for w in W0]
+        P_out = [torch.zeros(p.shape, dtype=dtype, device="cuda") for p in P0]   # row major (a QR factor may not be)
+        th = None
+        if with_refresh:
+            work = torch.empty(2 * f.refresh_side_work_bytes(), dtype=torch.uint8, device="cuda")
+            side = torch.cuda.Stream()
+            torch.cuda.synchronize()
+            th = threading.Thread(target=lambda: f.refresh_projection_side(Gs, P_out, work, side, seed=9, iters=2))
+            th.start()
+        for _ in range(steps):
+            f.step(W, Gs)
+        if th is not None:
+            th.join()
+        torch.cuda.synchronize()
+        assert f.poll() == 0
+        return f, W, P_out
+
+    _, W_alone, _ = run(False)
+    f, W_beside, P_side = run(True)
+    for a, b in zip(W_alone, W_beside):
+        assert torch.equal(a, b)
+    ref = fb.Fira(shapes, r, dtype, hp)
+    ref.refresh_projection(Gs, seed=9, iters=2)
+    for i in range(len(shapes)):
+        assert torch.equal(P_side[i], ref.get_projection(i))
+        f.set_projection(i, P_side[i])
+    f.step(W_beside, Gs)
+    assert f.poll() == 0 and all(torch.isfinite(w.float()).all() for w in W_beside)
