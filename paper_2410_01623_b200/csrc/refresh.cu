@@ -18,9 +18,11 @@
 //   * A Z and A^T Y: G is exact in bf16; the iterate is rounded to bf16, and in the last round it is
 //     split into a bf16 high part and a bf16 remainder (two k-segments), so that the basis that is
 //     kept carries no bf16 rounding of the iterate;
-//   * the Gram product Y^T Y and the application of the inverse factor Y <- Y L^-T: both operands
-//     are fp32 matrices split into two bf16 parts, three k-segments (hi hi + hi lo + lo hi), which is
-//     good to about 2^-16: enough for CholeskyQR, whose second pass removes what the first left;
+//   * the Gram product Y^T Y and the application of the inverse factor Y <- Y L^-T: for the basis
+//     that is kept both operands are fp32 matrices split into two bf16 parts, three k-segments
+//     (hi hi + hi lo + lo hi), which is good to about 2^-16: enough for CholeskyQR, whose second pass
+//     removes what the first left; for the intermediate iterates plain bf16 operands (one segment):
+//     the next product rounds the iterate to bf16 anyway, and all it asks is a well-conditioned one;
 //   * L^-T itself comes from the triangular-solve kernel applied to the identity (r x r, fp32).
 // Only the Cholesky factorisation and that small solve stay on the CUDA cores.
 //
@@ -276,7 +278,10 @@ k_chol_update(const RefreshMat* __restrict__ rm, int J0, int nt) {
 // ------------------------------------------------------------------ X <- X L^-T
 // One block per tile of 64 rows of X (rows x r, in place).  For each 64-wide
 // block column J: X_J = (X_J - X_{<J} L[J, <J]^T) L_JJ^-T.
-struct TrsmDesc { float* X; const float* L; int rows, r; };
+// tri: X starts as the identity (the solve that produces L^-T itself).  The result is upper
+// triangular and stays so on the way, so a row tile starts at its own diagonal block and its
+// products run over the columns from there on: a third of the work.
+struct TrsmDesc { float* X; const float* L; int rows, r; int tri; };
 
 __global__ void __launch_bounds__(GEMM_THREADS)
 k_trsm_rows(const TrsmDesc* __restrict__ descs, int ndesc, const int* __restrict__ tile_start) {
@@ -289,10 +294,11 @@ k_trsm_rows(const TrsmDesc* __restrict__ descs, int ndesc, const int* __restrict
   const int I0 = (blockIdx.x - tile_start[p]) * TM;
   const int r = t.r;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  for (int J0 = 0; J0 < r; J0 += CB) {
+  const int K0 = t.tri ? I0 : 0;               // first column of X that can be non-zero in these rows
+  for (int J0 = K0; J0 < r; J0 += CB) {
     const int jb = min(CB, r - J0);
     float acc[4][4] = {};
-    gemm_tile<1, float, float>(t.X, r, 1, t.L, 1, r, t.rows, J0 + jb, J0, I0, J0, acc, As, Bs);
+    gemm_tile<1, float, float>(t.X + K0, r, 1, t.L + K0, 1, r, t.rows, J0 + jb, J0 - K0, I0, J0, acc, As, Bs);
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
       const int il = ty * 4 + x;
@@ -386,9 +392,13 @@ static bool refresh_on_tc(const fira_matrix_desc& d) {
   return d.dtype == FIRA_BF16 && tc_supported(d) && tc_rows_aligned(d);   // the refresh only reads G
 }
 
-// The eight kinds of tensor-core jobs of one matrix: A Z and A^T Y (plain and with a split iterate),
-// the two Gram products, the two applications of L^-T.
-enum { JOB_AZ = 0, JOB_AZ_SPLIT, JOB_ATY, JOB_ATY_SPLIT, JOB_GRAM_Y, JOB_GRAM_Z, JOB_APPLY_Y, JOB_APPLY_Z, JOB_KINDS };
+// The kinds of tensor-core jobs of one matrix: A Z and A^T Y (plain and with a split iterate), the
+// two Gram products and the two applications of L^-T, each with split operands (three k-segments,
+// for the basis that is kept) and with plain bf16 operands (one segment, for the intermediate
+// iterates, which the next product rounds to bf16 anyway and which only have to stay well
+// conditioned).
+enum { JOB_AZ = 0, JOB_AZ_SPLIT, JOB_ATY, JOB_ATY_SPLIT, JOB_GRAM_Y, JOB_GRAM_Z, JOB_APPLY_Y, JOB_APPLY_Z,
+       JOB_GRAM_Y1, JOB_GRAM_Z1, JOB_APPLY_Y1, JOB_APPLY_Z1, JOB_KINDS };
 
 static TcGemmJob refresh_job(const fira_matrix_desc& dsc, int kind) {
   TcGemmJob j;
@@ -404,13 +414,13 @@ static TcGemmJob refresh_job(const fira_matrix_desc& dsc, int kind) {
       if (kind == JOB_AZ_SPLIT || kind == JOB_ATY_SPLIT) { j.nseg = 2; j.asel = 0u; j.bsel = 2u; }   // A hi, A lo(iterate)
       break;
     }
-    case JOB_GRAM_Y: case JOB_GRAM_Z:      // C[i][j] = sum_k X[k][i] X[k][j]: "G" = X as [k][i]
-      j.m = kind == JOB_GRAM_Y ? d : l; j.n = dsc.r; j.ld = dsc.r; j.mn_major = 1;
-      j.nseg = 3; j.asel = 4u; j.bsel = 2u;   // hi hi, hi lo, lo hi
+    case JOB_GRAM_Y: case JOB_GRAM_Z: case JOB_GRAM_Y1: case JOB_GRAM_Z1:   // C[i][j] = sum_k X[k][i] X[k][j]: "G" = X as [k][i]
+      j.m = (kind == JOB_GRAM_Y || kind == JOB_GRAM_Y1) ? d : l; j.n = dsc.r; j.ld = dsc.r; j.mn_major = 1;
+      if (kind == JOB_GRAM_Y || kind == JOB_GRAM_Z) { j.nseg = 3; j.asel = 4u; j.bsel = 2u; }   // hi hi, hi lo, lo hi
       break;
     default:                               // X[i][j] = sum_k X[i][k] U[k][j]: "G" = X as [i][k]
-      j.m = kind == JOB_APPLY_Y ? d : l; j.n = dsc.r; j.ld = dsc.r; j.mn_major = 0;
-      j.nseg = 3; j.asel = 4u; j.bsel = 2u;
+      j.m = (kind == JOB_APPLY_Y || kind == JOB_APPLY_Y1) ? d : l; j.n = dsc.r; j.ld = dsc.r; j.mn_major = 0;
+      if (kind == JOB_APPLY_Y || kind == JOB_APPLY_Z) { j.nseg = 3; j.asel = 4u; j.bsel = 2u; }
       break;
   }
   return j;
@@ -513,11 +523,15 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
             case JOB_GRAM_Y: j.G = m.Yb; j.G_lo = m.Yl; j.B = m.Yb; j.B_lo = m.Yl; j.C = m.C; break;
             case JOB_GRAM_Z: j.G = m.Zb; j.G_lo = m.Zl; j.B = m.Zb; j.B_lo = m.Zl; j.C = m.C; break;
             case JOB_APPLY_Y: j.G = m.Yb; j.G_lo = m.Yl; j.B = m.Ub; j.B_lo = m.Ul; j.C = m.Y; break;
-            default: j.G = m.Zb; j.G_lo = m.Zl; j.B = m.Ub; j.B_lo = m.Ul; j.C = m.Z; break;
+            case JOB_APPLY_Z: j.G = m.Zb; j.G_lo = m.Zl; j.B = m.Ub; j.B_lo = m.Ul; j.C = m.Z; break;
+            case JOB_GRAM_Y1: j.G = m.Yb; j.B = m.Yb; j.C = m.C; break;
+            case JOB_GRAM_Z1: j.G = m.Zb; j.B = m.Zb; j.C = m.C; break;
+            case JOB_APPLY_Y1: j.G = m.Yb; j.B = m.Ub; j.C = m.Y; break;
+            default: j.G = m.Zb; j.B = m.Ub; j.C = m.Z; break;
           }
           jobs[k].push_back(j);
         }
-        tU.push_back(TrsmDesc{m.U, m.C, m.r, m.r}); sTU.push_back(sTU.back() + (m.r + TM - 1) / TM);
+        tU.push_back(TrsmDesc{m.U, m.C, m.r, m.r, 1}); sTU.push_back(sTU.back() + (m.r + TM - 1) / TM);
         continue;
       }
       GemmDesc g;
@@ -535,8 +549,8 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
       g.A = m.Y; g.B = m.Y; g.K = m.d; gYY.push_back(g);
       g.A = m.Z; g.B = m.Z; g.K = m.l; gZZ.push_back(g);
       sYY.push_back(sYY.back() + tiles(m.r, m.r));
-      tY.push_back(TrsmDesc{m.Y, m.C, m.d, m.r}); sTY.push_back(sTY.back() + (m.d + TM - 1) / TM);
-      tZ.push_back(TrsmDesc{m.Z, m.C, m.l, m.r}); sTZ.push_back(sTZ.back() + (m.l + TM - 1) / TM);
+      tY.push_back(TrsmDesc{m.Y, m.C, m.d, m.r, 0}); sTY.push_back(sTY.back() + (m.d + TM - 1) / TM);
+      tZ.push_back(TrsmDesc{m.Z, m.C, m.l, m.r, 0}); sTZ.push_back(sTZ.back() + (m.l + TM - 1) / TM);
     }
     char* tp = tg.work_base + align_up(data_end);
     cudaError_t cerr = cudaSuccess;
@@ -599,12 +613,15 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     // CholeskyQR of Y (y = true) or Z; the second pass brings the basis to fp32 orthonormality and is
     // needed only for the basis that is kept: one pass (deviation about cond^2 times the product's
     // precision) keeps an intermediate iterate well conditioned, which is all the next product asks.
-    auto orth = [&](bool y, int passes) -> fira_status {
+    // precise: split operands (the basis that is kept); otherwise plain bf16 operands.
+    auto orth = [&](bool y, int passes, bool precise) -> fira_status {
+      const int kg = y ? (precise ? JOB_GRAM_Y : JOB_GRAM_Y1) : (precise ? JOB_GRAM_Z : JOB_GRAM_Z1);
+      const int ka = y ? (precise ? JOB_APPLY_Y : JOB_APPLY_Y1) : (precise ? JOB_APPLY_Z : JOB_APPLY_Z1);
       for (int pass = 0; pass < passes; ++pass) {
         if (nsimt) k_rgemm<<<sYY.back(), GEMM_THREADS, 0, st>>>(y ? dYY : dZZ, nsimt, dsYY);
         if (ntc) {
-          k_split_bf16<<<ew_grid, 256, 0, st>>>(rm_dev, y ? 0 : 1, 1);
-          const fira_status gs = tc_gemm_run(c, tab[y ? JOB_GRAM_Y : JOB_GRAM_Z], ntc, jtiles[y ? JOB_GRAM_Y : JOB_GRAM_Z], st);
+          k_split_bf16<<<ew_grid, 256, 0, st>>>(rm_dev, y ? 0 : 1, precise ? 1 : 0);
+          const fira_status gs = tc_gemm_run(c, tab[kg], ntc, jtiles[kg], st);
           if (gs != FIRA_OK) return gs;
         }
         for (int J0 = 0; J0 < rmax; J0 += CB) {
@@ -622,8 +639,8 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
         if (ntc) {
           k_identity<<<ew_grid, 256, 0, st>>>(rm_dev);
           k_trsm_rows<<<sTU.back(), GEMM_THREADS, 0, st>>>(dTU, ntc, dsTU);      // U = L^-T
-          k_split_bf16<<<ew_grid, 256, 0, st>>>(rm_dev, 2, 1);
-          const fira_status as = tc_gemm_run(c, tab[y ? JOB_APPLY_Y : JOB_APPLY_Z], ntc, jtiles[y ? JOB_APPLY_Y : JOB_APPLY_Z], st);
+          k_split_bf16<<<ew_grid, 256, 0, st>>>(rm_dev, 2, precise ? 1 : 0);
+          const fira_status as = tc_gemm_run(c, tab[ka], ntc, jtiles[ka], st);
           if (as != FIRA_OK) return as;
         }
       }
@@ -631,13 +648,13 @@ fira_status refresh_impl(fira_ctx* c, const void* const* G_dev, const std::vecto
     };
     k_gauss<<<ew_grid, 256, 0, st>>>(rm_dev);
     fira_status prs = product(true, iters == 0);
-    if (prs == FIRA_OK) prs = orth(true, iters == 0 ? 2 : 1);
+    if (prs == FIRA_OK) prs = orth(true, iters == 0 ? 2 : 1, iters == 0);
     for (int it = 0; it < iters && prs == FIRA_OK; ++it) {
       const bool last = it + 1 == iters;
       prs = product(false, last);
-      if (prs == FIRA_OK) prs = orth(false, 1);
+      if (prs == FIRA_OK) prs = orth(false, 1, last);
       if (prs == FIRA_OK) prs = product(true, last);
-      if (prs == FIRA_OK) prs = orth(true, last ? 2 : 1);
+      if (prs == FIRA_OK) prs = orth(true, last ? 2 : 1, last);
     }
     if (prs != FIRA_OK) return prs;
     k_store_projection<<<ew_grid, 256, 0, st>>>(rm_dev);
