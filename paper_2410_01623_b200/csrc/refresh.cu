@@ -155,6 +155,7 @@ __global__ void __launch_bounds__(GEMM_THREADS)
 k_chol_diag(const RefreshMat* __restrict__ rm, int J0, float shift_rel, unsigned* __restrict__ status) {
   __shared__ float D[CB][CB + 1];
   __shared__ float red[GEMM_THREADS];
+  __shared__ float col[2][2 * CB];
   const RefreshMat m = rm[blockIdx.x];
   const int r = m.r;
   if (J0 >= r) return;
@@ -163,7 +164,7 @@ k_chol_diag(const RefreshMat* __restrict__ rm, int J0, float shift_rel, unsigned
   float floor_pivot;
   if (J0 == 0) {
     float tr = 0.f;
-    for (int i = tid; i < r; i += GEMM_THREADS) tr += C[(long long)i * r + i];
+    for (int i = tid; i < r; i += GEMM_THREADS) tr += __ldcg(C + (long long)i * r + i);
     red[tid] = tr;
     __syncthreads();
     for (int o = GEMM_THREADS / 2; o > 0; o >>= 1) {
@@ -180,66 +181,92 @@ k_chol_diag(const RefreshMat* __restrict__ rm, int J0, float shift_rel, unsigned
     floor_pivot = m.info[0];
   }
   const int jb = min(CB, r - J0);
+  // (loads through __ldcg: known to be global, so they can overlap across the stores to shared memory)
+#pragma unroll
   for (int e = tid; e < CB * CB; e += GEMM_THREADS) {
     const int i = e / CB, j = e % CB;
-    D[i][j] = (i < jb && j < jb) ? C[(long long)(J0 + i) * r + J0 + j] : (i == j ? 1.f : 0.f);
+    D[i][j] = (i < jb && j < jb) ? __ldcg(C + (long long)(J0 + i) * r + J0 + j) : (i == j ? 1.f : 0.f);
+  }
+  if (tid < 2 * CB) { col[0][tid] = 0.f; col[1][tid] = 0.f; }
+  __syncthreads();
+  // Thread i < CB keeps row i in registers, shifted left by one entry per step so that the loop body
+  // is the same for every step: at step k, a[j] is the entry of column k + j.  Every row hands its
+  // entry of column k to the others through col[] (two buffers in turn; their upper halves stay
+  // zero), forms the pivot's root, scales its entry and updates the rest of its row.  Entries right
+  // of the diagonal are updated too: they are the mirror images and are never stored.  The two warps
+  // that work meet at a barrier of their own.
+  if (tid < CB) {
+    float a[CB];
+#pragma unroll
+    for (int j = 0; j < CB; ++j) a[j] = D[tid][j];
+#pragma unroll 1
+    for (int k = 0; k < CB; ++k) {
+      float* ck = col[k & 1];
+      ck[tid] = a[0];
+      asm volatile("bar.sync 1, %0;" ::"n"(CB) : "memory");
+      float pv = ck[k];
+      if (!(pv > floor_pivot) || !isfinite(pv)) {
+        if (tid == k && k < jb) atomicOr(status, DEV_STATUS_NONFINITE);
+        pv = floor_pivot;
+      }
+      const float s = sqrtf(pv), rs = 1.f / s;
+      const float lik = (tid == k) ? s : a[0] * rs;
+      D[tid][k] = lik;
+#pragma unroll
+      for (int j = 1; j < CB; ++j) a[j - 1] = a[j] - lik * (ck[k + j] * rs);
+      a[CB - 1] = 0.f;
+    }
   }
   __syncthreads();
-  for (int k = 0; k < jb; ++k) {
-    if (tid == 0) {
-      float pv = D[k][k];
-      if (!(pv > floor_pivot) || !isfinite(pv)) { pv = floor_pivot; atomicOr(status, DEV_STATUS_NONFINITE); }
-      D[k][k] = sqrtf(pv);
-    }
-    __syncthreads();
-    const float dk = D[k][k];
-    if (tid > k && tid < jb) D[tid][k] /= dk;
-    __syncthreads();
-    const int rem = jb - k - 1;
-    for (int e = tid; e < rem * rem; e += GEMM_THREADS) {
-      const int i = k + 1 + e / rem, j = k + 1 + e % rem;
-      if (j <= i) D[i][j] -= D[i][k] * D[j][k];
-    }
-    __syncthreads();
-  }
   for (int e = tid; e < jb * jb; e += GEMM_THREADS) {
     const int i = e / jb, j = e % jb;
     if (j <= i) C[(long long)(J0 + i) * r + J0 + j] = D[i][j];
   }
 }
 
-// Rows below the diagonal block: one block per 64 rows (tiles_per_matrix of them per matrix),
-// one thread per row for the substitution.
-__global__ void __launch_bounds__(64)
+// Rows below the diagonal block: one block of CB threads per CB rows (tiles_per_matrix of them per
+// matrix); a thread is a column while loading and storing, a row while solving x <- x L_JJ^-T.  The
+// row lives in registers and moves left by one entry per step, the finished entry coming back in at
+// the right end, so that the loop body is the same for every step and the row ends up in order; the
+// CB rows of zeros under L_JJ in shared memory are what the entries that are already final meet.
+__global__ void __launch_bounds__(CB)
 k_chol_panel(const RefreshMat* __restrict__ rm, int J0, int tiles_per_matrix) {
-  __shared__ float D[CB][CB + 1];
-  __shared__ float T[64][CB + 1];
+  __shared__ float DT[2 * CB][CB + 1];    // rows < CB: L_JJ (identity past the matrix's end); the rest: the
+                                          // tile on its way in and out, zeros during the solve
   const RefreshMat m = rm[blockIdx.x / tiles_per_matrix];
   const int r = m.r;
   const int jb = min(CB, r - J0);
-  const int I0 = J0 + CB + (blockIdx.x % tiles_per_matrix) * 64;
+  const int I0 = J0 + CB + (blockIdx.x % tiles_per_matrix) * CB;
   if (J0 >= r || I0 >= r) return;
   float* C = m.C;
   const int tid = threadIdx.x;
-  for (int e = tid; e < CB * CB; e += 64) {
-    const int i = e / CB, j = e % CB;
-    D[i][j] = (i < jb && j < jb) ? C[(long long)(J0 + i) * r + J0 + j] : (i == j ? 1.f : 0.f);
-    T[i][j] = (I0 + i < r && j < jb) ? C[(long long)(I0 + i) * r + J0 + j] : 0.f;
+#pragma unroll 16
+  for (int i = 0; i < CB; ++i) {
+    DT[i][tid] = (i < jb && tid < jb) ? __ldcg(C + (long long)(J0 + i) * r + J0 + tid) : (i == tid ? 1.f : 0.f);
+    DT[CB + i][tid] = (I0 + i < r && tid < jb) ? __ldcg(C + (long long)(I0 + i) * r + J0 + tid) : 0.f;
   }
   __syncthreads();
-  if (I0 + tid < r) {
-    float* row = T[tid];
-    for (int c = 0; c < jb; ++c) {
-      float v = row[c];
-      for (int k = 0; k < c; ++k) v -= row[k] * D[c][k];
-      row[c] = v / D[c][c];
-    }
+  float a[CB];
+#pragma unroll
+  for (int j = 0; j < CB; ++j) a[j] = DT[CB + tid][j];
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < CB; ++i) DT[CB + i][tid] = 0.f;
+  __syncthreads();
+#pragma unroll 1
+  for (int c = 0; c < CB; ++c) {
+    const float x = a[0] / DT[c][c];
+#pragma unroll
+    for (int j = 1; j < CB; ++j) a[j - 1] = a[j] - x * DT[c + j][c];
+    a[CB - 1] = x;
   }
   __syncthreads();
-  for (int e = tid; e < CB * CB; e += 64) {
-    const int i = e / CB, j = e % CB;
-    if (I0 + i < r && j < jb) C[(long long)(I0 + i) * r + J0 + j] = T[i][j];
-  }
+#pragma unroll
+  for (int j = 0; j < CB; ++j) DT[CB + tid][j] = a[j];
+  __syncthreads();
+#pragma unroll 16
+  for (int i = 0; i < CB; ++i)
+    if (I0 + i < r && tid < jb) C[(long long)(I0 + i) * r + J0 + tid] = DT[CB + i][tid];
 }
 
 // Trailing update on the 128 x 128 tiles (I >= K) of the part below and right of the panel.
