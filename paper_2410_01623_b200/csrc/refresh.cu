@@ -290,6 +290,43 @@ k_chol_update(const RefreshMat* __restrict__ rm, int J0, int nt) {
   gemm_tile<SIMT_Q, float, float>(C + J0, r, 1, C + J0, 1, r, r, r, jb, I0, K0, acc, As, Bs);
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const int lo = J0 + CB;                      // only rows and columns past the panel change
+  if (r % 4 == 0) {
+    // Four rows at a time: all their loads first, then the stores (a load after a store to the same
+    // array would have to wait for it).  A group of four columns is inside the matrix or outside it
+    // as a whole; entries that must not change (above the diagonal, before the panel's end) get
+    // their old value back, and no other block touches this tile.
+#pragma unroll
+    for (int xb = 0; xb < 4 * SIMT_Q; xb += 4) {
+      float4 c[4][SIMT_Q];
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        const int i = I0 + tile_coord(ty, xb + x);
+#pragma unroll
+        for (int q = 0; q < SIMT_Q; ++q) {
+          const int j = K0 + tile_coord(tx, 4 * q);
+          c[x][q] = (i < r && j < r) ? __ldcg(reinterpret_cast<const float4*>(C + (long long)i * r + j))
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        const int i = I0 + tile_coord(ty, xb + x);
+        if (i >= r || i < lo) continue;
+#pragma unroll
+        for (int q = 0; q < SIMT_Q; ++q) {
+          const int j = K0 + tile_coord(tx, 4 * q);
+          if (j >= r || j > i || j + 3 < lo) continue;
+          float4 v = c[x][q];
+          if (j >= lo && j <= i) v.x -= acc[xb + x][4 * q];
+          if (j + 1 >= lo && j + 1 <= i) v.y -= acc[xb + x][4 * q + 1];
+          if (j + 2 >= lo && j + 2 <= i) v.z -= acc[xb + x][4 * q + 2];
+          if (j + 3 >= lo && j + 3 <= i) v.w -= acc[xb + x][4 * q + 3];
+          *reinterpret_cast<float4*>(C + (long long)i * r + j) = v;
+        }
+      }
+    }
+    return;
+  }
 #pragma unroll
   for (int x = 0; x < 4 * SIMT_Q; ++x) {
     const int i = I0 + tile_coord(ty, x);
@@ -333,13 +370,13 @@ k_trsm_rows(const TrsmDesc* __restrict__ descs, int ndesc, const int* __restrict
       for (int y = 0; y < 4; ++y) {
         const int jl = tx * 4 + y;
         float v = 0.f;
-        if (I0 + il < t.rows && jl < jb) v = t.X[(long long)(I0 + il) * r + J0 + jl] - acc[x][y];
+        if (I0 + il < t.rows && jl < jb) v = __ldcg(t.X + (long long)(I0 + il) * r + J0 + jl) - acc[x][y];
         T[il][jl] = v;
       }
     }
     for (int e = tid; e < CB * CB; e += GEMM_THREADS) {
       const int i = e / CB, j = e % CB;
-      D[i][j] = (i < jb && j < jb) ? t.L[(long long)(J0 + i) * r + J0 + j] : (i == j ? 1.f : 0.f);
+      D[i][j] = (i < jb && j < jb) ? __ldcg(t.L + (long long)(J0 + i) * r + J0 + j) : (i == j ? 1.f : 0.f);
     }
     __syncthreads();
     if (tid < TM && I0 + tid < t.rows) {
