@@ -224,11 +224,24 @@ k_chol_diag(const RefreshMat* __restrict__ rm, int J0, float shift_rel, unsigned
   }
 }
 
+// x <- x L^-T for one row x of CB entries held in registers.  Rows [0, CB) of DT hold the lower
+// triangular L (the identity past the matrix's end), rows [CB, 2 CB) zeros.  The row moves left by one
+// entry per step and the finished entry comes back in at the right end, so that the loop body is the
+// same for every step and the row ends up in order; the zeros are what the entries that are already
+// final meet.
+__device__ __forceinline__ void solve_row_shifting(float (&a)[CB], const float (*DT)[CB + 1]) {
+#pragma unroll 1
+  for (int c = 0; c < CB; ++c) {
+    const float x = a[0] / DT[c][c];
+#pragma unroll
+    for (int j = 1; j < CB; ++j) a[j - 1] = a[j] - x * DT[c + j][c];
+    a[CB - 1] = x;
+  }
+}
+
 // Rows below the diagonal block: one block of CB threads per CB rows (tiles_per_matrix of them per
-// matrix); a thread is a column while loading and storing, a row while solving x <- x L_JJ^-T.  The
-// row lives in registers and moves left by one entry per step, the finished entry coming back in at
-// the right end, so that the loop body is the same for every step and the row ends up in order; the
-// CB rows of zeros under L_JJ in shared memory are what the entries that are already final meet.
+// matrix); a thread is a column while loading and storing, a row while solving x <- x L_JJ^-T
+// (solve_row_shifting).
 __global__ void __launch_bounds__(CB)
 k_chol_panel(const RefreshMat* __restrict__ rm, int J0, int tiles_per_matrix) {
   __shared__ float DT[2 * CB][CB + 1];    // rows < CB: L_JJ (identity past the matrix's end); the rest: the
@@ -253,13 +266,7 @@ k_chol_panel(const RefreshMat* __restrict__ rm, int J0, int tiles_per_matrix) {
 #pragma unroll
   for (int i = 0; i < CB; ++i) DT[CB + i][tid] = 0.f;
   __syncthreads();
-#pragma unroll 1
-  for (int c = 0; c < CB; ++c) {
-    const float x = a[0] / DT[c][c];
-#pragma unroll
-    for (int j = 1; j < CB; ++j) a[j - 1] = a[j] - x * DT[c + j][c];
-    a[CB - 1] = x;
-  }
+  solve_row_shifting(a, DT);
   __syncthreads();
 #pragma unroll
   for (int j = 0; j < CB; ++j) DT[CB + tid][j] = a[j];
@@ -349,10 +356,11 @@ struct TrsmDesc { float* X; const float* L; int rows, r; int tri; };
 
 __global__ void __launch_bounds__(GEMM_THREADS)
 k_trsm_rows(const TrsmDesc* __restrict__ descs, int ndesc, const int* __restrict__ tile_start) {
+  static_assert(TM == CB, "one row of the tile per solving thread");
   __shared__ __align__(16) float As[TK][TM + 4];
   __shared__ __align__(16) float Bs[TK][TN + 4];
-  __shared__ float T[TM][CB + 1];
-  __shared__ float D[CB][CB + 1];
+  __shared__ float DT[2 * CB][CB + 1];         // rows < CB: L_JJ; the rest: the tile on its way in and out,
+                                               // zeros during the solve (solve_row_shifting)
   const int p = find_matrix(tile_start, ndesc, blockIdx.x);
   const TrsmDesc t = descs[p];
   const int I0 = (blockIdx.x - tile_start[p]) * TM;
@@ -363,33 +371,47 @@ k_trsm_rows(const TrsmDesc* __restrict__ descs, int ndesc, const int* __restrict
     const int jb = min(CB, r - J0);
     float acc[4][4] = {};
     gemm_tile<1, float, float>(t.X + K0, r, 1, t.L + K0, 1, r, t.rows, J0 + jb, J0 - K0, I0, J0, acc, As, Bs);
+    float xin[4][4];
 #pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      const int il = ty * 4 + x;
+    for (int x = 0; x < 4; ++x)
 #pragma unroll
       for (int y = 0; y < 4; ++y) {
-        const int jl = tx * 4 + y;
-        float v = 0.f;
-        if (I0 + il < t.rows && jl < jb) v = __ldcg(t.X + (long long)(I0 + il) * r + J0 + jl) - acc[x][y];
-        T[il][jl] = v;
+        const int il = ty * 4 + x, jl = tx * 4 + y;
+        xin[x][y] = (I0 + il < t.rows && jl < jb) ? __ldcg(t.X + (long long)(I0 + il) * r + J0 + jl) : 0.f;
       }
-    }
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int y = 0; y < 4; ++y) {
+        const int il = ty * 4 + x, jl = tx * 4 + y;
+        DT[CB + il][jl] = (I0 + il < t.rows && jl < jb) ? xin[x][y] - acc[x][y] : 0.f;
+      }
+#pragma unroll
     for (int e = tid; e < CB * CB; e += GEMM_THREADS) {
       const int i = e / CB, j = e % CB;
-      D[i][j] = (i < jb && j < jb) ? __ldcg(t.L + (long long)(J0 + i) * r + J0 + j) : (i == j ? 1.f : 0.f);
+      DT[i][j] = (i < jb && j < jb) ? __ldcg(t.L + (long long)(J0 + i) * r + J0 + j) : (i == j ? 1.f : 0.f);
     }
     __syncthreads();
-    if (tid < TM && I0 + tid < t.rows) {
-      float* row = T[tid];
-      for (int c = 0; c < jb; ++c) {
-        float v = row[c];
-        for (int k = 0; k < c; ++k) v -= row[k] * D[c][k];
-        v /= D[c][c];
-        row[c] = v;
-        t.X[(long long)(I0 + tid) * r + J0 + c] = v;
-      }
+    float a[CB];
+    if (tid < TM) {
+#pragma unroll
+      for (int j = 0; j < CB; ++j) a[j] = DT[CB + tid][j];
     }
     __syncthreads();
+    for (int e = tid; e < CB * CB; e += GEMM_THREADS) DT[CB + e / CB][e % CB] = 0.f;
+    __syncthreads();
+    if (tid < TM) solve_row_shifting(a, DT);
+    __syncthreads();
+    if (tid < TM) {
+#pragma unroll
+      for (int j = 0; j < CB; ++j) DT[CB + tid][j] = a[j];
+    }
+    __syncthreads();
+    for (int e = tid; e < TM * CB; e += GEMM_THREADS) {
+      const int i = e / CB, j = e % CB;
+      if (I0 + i < t.rows && j < jb) t.X[(long long)(I0 + i) * r + J0 + j] = DT[CB + i][j];
+    }
+    __syncthreads();                           // the next block column's product reads these columns
   }
 }
 
