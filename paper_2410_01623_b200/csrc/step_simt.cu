@@ -76,25 +76,40 @@ k_adam_rows(const MatDev* __restrict__ mats, const int* __restrict__ list, int n
   const float bias = (float)(sqrt(1.0 - pow((double)hp.beta2, s)) / (1.0 - pow((double)hp.beta1, s)));
   const long long base = (long long)l * mt.r;
   float nn = 0.f, rn = 0.f;
-  for (int j = lane; j < mt.r; j += 32) {
-    const float rv = mt.Rt[base + j];
-    float vv, nv;
-    if (hp.mode & HYPER_PSI_RMSPROP) {
-      vv = hp.beta2 * mt.V[base + j] + (1.f - hp.beta2) * rv * rv;
-      nv = rv / (sqrtf(vv) + hp.eps);
-    } else if (hp.mode & HYPER_PSI_ADAGRAD) {
-      vv = mt.V[base + j] + rv * rv;
-      nv = rv / (sqrtf(vv) + hp.eps);
-    } else {
-      const float mv = hp.beta1 * mt.M[base + j] + (1.f - hp.beta1) * rv;
-      vv = hp.beta2 * mt.V[base + j] + (1.f - hp.beta2) * rv * rv;
-      mt.M[base + j] = mv;
-      nv = bias * mv / (sqrtf(vv) + hp.eps);
+  // four entries per lane at a time, their loads before their stores (see back_tile)
+  for (int jq = lane; jq < mt.r; jq += 128) {
+    float rv4[4], m4[4], v4[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = jq + 32 * u;
+      const bool in = j < mt.r;
+      rv4[u] = in ? mt.Rt[base + j] : 0.f;
+      v4[u] = in ? mt.V[base + j] : 0.f;
+      m4[u] = (in && !(hp.mode & (HYPER_PSI_RMSPROP | HYPER_PSI_ADAGRAD))) ? mt.M[base + j] : 0.f;
     }
-    mt.V[base + j] = vv;
-    mt.Xt[base + j] = nv;
-    nn = fmaf(nv, nv, nn);
-    rn = fmaf(rv, rv, rn);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = jq + 32 * u;
+      if (j >= mt.r) continue;
+      const float rv = rv4[u];
+      float vv, nv;
+      if (hp.mode & HYPER_PSI_RMSPROP) {
+        vv = hp.beta2 * v4[u] + (1.f - hp.beta2) * rv * rv;
+        nv = rv / (sqrtf(vv) + hp.eps);
+      } else if (hp.mode & HYPER_PSI_ADAGRAD) {
+        vv = v4[u] + rv * rv;
+        nv = rv / (sqrtf(vv) + hp.eps);
+      } else {
+        const float mv = hp.beta1 * m4[u] + (1.f - hp.beta1) * rv;
+        vv = hp.beta2 * v4[u] + (1.f - hp.beta2) * rv * rv;
+        mt.M[base + j] = mv;
+        nv = bias * mv / (sqrtf(vv) + hp.eps);
+      }
+      mt.V[base + j] = vv;
+      mt.Xt[base + j] = nv;
+      nn = fmaf(nv, nv, nn);
+      rn = fmaf(rv, rv, rn);
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -136,23 +151,40 @@ __device__ __forceinline__ void back_tile(const MatDev& mt, int tile, float lr, 
   T* W = static_cast<T*>(mt.W);
   const float lam = (MODE == MODE_UPDATE) ? mt.sc->lambda : 1.f;
   float ss = 0.f;
+  // Two rows of the thread's entries at a time: every load of the pair first, then the arithmetic
+  // and the stores.  (Written element by element, each load of G and W would wait for the store
+  // before it, since the compiler cannot tell that they never overlap.)
 #pragma unroll
-  for (int x = 0; x < 4 * SIMT_Q; ++x) {
-    const int i = i0 + tile_coord(ty, x);
-    if (i >= mt.m) continue;
+  for (int xb = 0; xb < 4 * SIMT_Q; xb += 2) {
+    float g[2][4 * SIMT_Q], w[2][4 * SIMT_Q], kf[2][4 * SIMT_Q];
 #pragma unroll
-    for (int y = 0; y < 4 * SIMT_Q; ++y) {
-      const int j = j0 + tile_coord(tx, y);
-      if (j >= mt.n) continue;
-      const float kf = mt.kvec[mt.left ? j : i];
-      const long long off = (long long)i * mt.ld + j;
-      const float g = to_float<T>(G[off]);
-      if (MODE == MODE_NORM) {
-        const float sv = kf * (g - acc[x][y]);
-        ss = fmaf(sv, sv, ss);
-      } else {
-        const float w = to_float<T>(W[off]);
-        W[off] = from_float<T>(w - lr * (acc[x][y] + a_res * lam * kf * g));
+    for (int x = 0; x < 2; ++x) {
+      const int i = i0 + tile_coord(ty, xb + x);
+#pragma unroll
+      for (int y = 0; y < 4 * SIMT_Q; ++y) {
+        const int j = j0 + tile_coord(tx, y);
+        const bool in = i < mt.m && j < mt.n;
+        const long long off = (long long)i * mt.ld + j;
+        kf[x][y] = in ? mt.kvec[mt.left ? j : i] : 0.f;
+        g[x][y] = in ? to_float<T>(G[off]) : 0.f;
+        w[x][y] = (MODE == MODE_UPDATE && in) ? to_float<T>(W[off]) : 0.f;
+      }
+    }
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+      const int i = i0 + tile_coord(ty, xb + x);
+      if (i >= mt.m) continue;
+#pragma unroll
+      for (int y = 0; y < 4 * SIMT_Q; ++y) {
+        const int j = j0 + tile_coord(tx, y);
+        if (j >= mt.n) continue;
+        if (MODE == MODE_NORM) {
+          const float sv = kf[x][y] * (g[x][y] - acc[xb + x][y]);
+          ss = fmaf(sv, sv, ss);
+        } else {
+          W[(long long)i * mt.ld + j] =
+              from_float<T>(w[x][y] - lr * (acc[xb + x][y] + a_res * lam * kf[x][y] * g[x][y]));
+        }
       }
     }
   }
@@ -196,7 +228,20 @@ k_form_x(const MatDev* __restrict__ mats, const int* __restrict__ list, int nlis
   const int l = row - row_start[p];
   const float c = a_res * mt.sc->lambda * mt.kvec[l];
   const long long base = (long long)l * mt.r;
-  for (int j = lane; j < mt.r; j += 32) mt.Xt[base + j] = a_low * mt.Xt[base + j] - c * mt.Rt[base + j];
+  for (int jq = lane; jq < mt.r; jq += 128) {    // four entries per lane, loads before stores
+    float n4[4], r4[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = jq + 32 * u;
+      n4[u] = j < mt.r ? mt.Xt[base + j] : 0.f;
+      r4[u] = j < mt.r ? mt.Rt[base + j] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = jq + 32 * u;
+      if (j < mt.r) mt.Xt[base + j] = a_low * n4[u] - c * r4[u];
+    }
+  }
 }
 
 // ---------------------------------------------------------------- Fira-only-scaling
