@@ -143,7 +143,7 @@ k_rgemm(const GemmDesc* __restrict__ descs, int ndesc, const int* __restrict__ t
 // C (r x r, symmetric, row major) -> lower factor L in place (the strict upper triangle is left as
 // it was), for all matrices of a chunk at once, right-looking over block columns of CB = 64.  Three
 // launches per block column, each over every matrix:
-//   k_chol_diag   one block per matrix factors the CB x CB diagonal block in shared memory
+//   k_chol_diag   one block per matrix factors the CB x CB diagonal block, one row per thread in registers
 //   k_chol_panel  the rows below it: L[i, J] = C[i, J] L_JJ^-T, 64 rows per block
 //   k_chol_update the trailing matrix: C[I, K] -= L[I, J] L[K, J]^T on 128 x 128 tiles of its lower half
 // On the first block column k_chol_diag also adds shift_rel * trace(C)/r to the whole diagonal and
