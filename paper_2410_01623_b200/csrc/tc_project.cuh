@@ -488,6 +488,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
       const int l = d.l0 + BM * (int)rank + row;
       const float bias = EPI == EPI_ADAM ? fast[2 * d.slot] : 0.f;
       const float* wrow = EPI == EPI_ADAM ? wq_all + wq_off[d.slot] + d.r0 : nullptr;   // weights of this tile's rank range
+      if (EPI == EPI_ADAM) asm volatile("prefetch.global.L1 [%0];" ::"l"(wrow));
       if (!ptx::mbar_wait_cluster(ptx::smem_u32(&ctl->tmem_full[buf]), bphase, abort_flag)) break;
       ptx::tc_fence_after();
       const uint32_t tcol = tmem + ((uint32_t)(quarter * 32) << 16) + buf * BN_MAX;
@@ -499,6 +500,9 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         uint32_t rr[32];
         __syncwarp();
         ptx::tmem_ld_32x32b_x32(tcol + K1_ECOLS * c, rr);
+        // the next chunk's 32 weights (one 128-byte line) on their way into L1 meanwhile
+        if (EPI == EPI_ADAM && c + 1 < nch)
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(wrow + K1_ECOLS * (c + 1)));
         ptx::tmem_ld_wait();
         if (!fuse && c == nch - 1) {                     // the accumulator has been read out
           ptx::tc_fence_before();
