@@ -695,9 +695,12 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
   if (!pl->attrs_set) {
     const void* k1s[4] = {(const void*)k_tc_project<EPI_ADAM, PSI_ADAM, 0>, (const void*)k_tc_project<EPI_ADAM, PSI_RMSPROP, 0>,
                           (const void*)k_tc_project<EPI_ADAM, PSI_ADAGRAD, 0>, (const void*)k_tc_project<EPI_ADAM, PSI_ADAM, 1>};
+    const void* k1g[2] = {(const void*)k_tc_project<EPI_ADAM, PSI_ADAM, 0, 2>, (const void*)k_tc_project<EPI_ADAM, PSI_ADAM, 1, 2>};
     cudaError_t e1 = cudaSuccess;
     for (int i = 0; i < 4 && e1 == cudaSuccess; ++i)
       e1 = cudaFuncSetAttribute(k1s[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K1_SMEM_BYTES);
+    for (int i = 0; i < 2 && e1 == cudaSuccess; ++i)
+      e1 = cudaFuncSetAttribute(k1g[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)k1_smem_bytes(2));
     cudaError_t e2 = cudaFuncSetAttribute(k_tc_back_project<5, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)k2_smem_bytes(5, 2));
     if (e2 == cudaSuccess)
       e2 = cudaFuncSetAttribute(k_tc_back_project<4, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)k2_smem_bytes(4, 3));
@@ -721,6 +724,13 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
         return -1;
       }
       pl->max_pairs_fused = std::min(nclusters, pl->num_sms / 2);
+      cfg.blockDim = dim3(k1_threads(2)); cfg.dynamicSmemBytes = k1_smem_bytes(2);
+      const cudaError_t e4 = cudaOccupancyMaxActiveClusters(&nclusters, k1g[1], &cfg);
+      if (e4 != cudaSuccess || nclusters <= 0) {
+        set_error(std::string("cudaOccupancyMaxActiveClusters: ") + cudaGetErrorString(e4));
+        return -1;
+      }
+      pl->max_pairs_fused = std::min(nclusters, pl->max_pairs_fused);
     }
     pl->attrs_set = true;
   }
@@ -756,11 +766,24 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
                                  HYPER_PSI_RMSPROP | HYPER_PSI_ADAGRAD)) == 0;
   const int k1_grid = 2 * std::min(k1n, fused ? pl->max_pairs_fused : pl->num_sms / 2);
   const ProjTileDesc* td1 = pl->td1_dev + k1a;
+  int rmax = 0;
+  for (int q = qa; q < qb; ++q) rmax = std::max(rmax, c->mats[c->tc_list[q]].r);
+  // Short products are bound by the epilogue, which then runs with two groups of warps per CTA; long
+  // ones (r = 1024 lists) are bound by the tensor pipe and keep one.
+  const bool two_groups = rmax <= 512;
 #define FIRA_LAUNCH_K1(PSI, FUSE)                                                     \
   k_tc_project<EPI_ADAM, PSI, FUSE><<<k1_grid, K1_THREADS, K1_SMEM_BYTES, st>>>(      \
       pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev)
   if (hp.mode & HYPER_PSI_RMSPROP) FIRA_LAUNCH_K1(PSI_RMSPROP, 0);
   else if (hp.mode & HYPER_PSI_ADAGRAD) FIRA_LAUNCH_K1(PSI_ADAGRAD, 0);
+  else if (two_groups) {
+    if (fused)
+      k_tc_project<EPI_ADAM, PSI_ADAM, 1, 2><<<k1_grid, k1_threads(2), k1_smem_bytes(2), st>>>(
+          pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev);
+    else
+      k_tc_project<EPI_ADAM, PSI_ADAM, 0, 2><<<k1_grid, k1_threads(2), k1_smem_bytes(2), st>>>(
+          pl->maps_dev, td1, k1n, pl->fast_dev, pl->wq_dev, pl->wq_off, hp, c->status_dev);
+  }
   else if (fused) FIRA_LAUNCH_K1(PSI_ADAM, 1);
   else FIRA_LAUNCH_K1(PSI_ADAM, 0);
 #undef FIRA_LAUNCH_K1
@@ -790,8 +813,6 @@ int launch_tc_step(fira_ctx* c, const Hyper& hp, int qa, int qb) {
   if (any_fused) k_tc_fix_x<<<dim3(16, nq), 256, 0, st>>>(mats, pl->list, qa, hp.a_low, hp.eps, pl->fast_dev);
   tm->mark(st);
   // long products keep five operand stages; short ones trade one for more epilogue boxes in flight
-  int rmax = 0;
-  for (int q = qa; q < qb; ++q) rmax = std::max(rmax, c->mats[c->tc_list[q]].r);
   if (rmax >= 1024)
     k_tc_back_project<5, 2><<<2 * std::min(k2n, pl->num_sms / 2), K2_THREADS, k2_smem_bytes(5, 2), st>>>(
         pl->maps_dev, pl->td2_dev + k2a, k2n, pl->fast_dev, hp, c->status_dev);

@@ -71,9 +71,15 @@ constexpr int K1_BOX_THREADS = 64;                      // two warps work on a b
 constexpr int K1_GSQ_WARPS = 8;
 constexpr int K1_GSQ_SPLIT = K1_GSQ_WARPS / 2;          // partial sums of G^2 per tile and l
 constexpr int K1_THREADS = 32 * (8 + K1_GSQ_WARPS);
+// EG = 2: a second group of four epilogue warps (16-19).  The two groups work on the same boxes, each
+// on one half of a box's 32 columns, and hand each other their halves of the row sums through XCH.
+constexpr int K1_THREADS_EG2 = K1_THREADS + 128;
+constexpr int K1_XCH_BYTES = BM * 4 * 4;                // per row: ||N||^2, ||R||^2, weighted ||R||^2 partials, k_l
 constexpr size_t K1_SMEM_BYTES = (size_t)K1_STAGES * K1_STAGE_BYTES + (size_t)K1_MVBUFS * K1_MVBUF_BYTES +
                                  (size_t)K1_NRBUFS * K1_NRBUF_BYTES + 512;
-static_assert(K1_SMEM_BYTES <= 227 * 1024, "shared memory budget");
+static_assert(K1_SMEM_BYTES + K1_XCH_BYTES <= 227 * 1024, "shared memory budget");
+constexpr int k1_threads(int eg) { return eg == 2 ? K1_THREADS_EG2 : K1_THREADS; }
+constexpr size_t k1_smem_bytes(int eg) { return K1_SMEM_BYTES + (eg == 2 ? K1_XCH_BYTES : 0); }
 
 // Per-tile record (256 l x BN r), built on the host once (32 bytes).
 struct ProjTileDesc {
@@ -89,11 +95,12 @@ static_assert(sizeof(ProjTileDesc) == 32, "ProjTileDesc layout");
 constexpr int PROJ_A_CHUNKED = 1 << 30;
 constexpr int PROJ_FUSE_X = 1 << 29;      // bn_left: this tile's epilogue forms X itself (FUSE_X kernels only)
 // Which matrices take that route.  The second sweep lengthens the epilogue and the exchange makes the
-// pairs of a row of tiles wait for the slowest of them.  Measured: one r-tile per row (no exchange,
-// 350M list, r = 256): -8 % on the step; long products (7B list, d = 4096, four r-tiles): -6 to
-// -7 %; short products with an exchange (1B list, d = 2048, two r-tiles): +2 %, the tiles are
-// epilogue-bound and their times jitter, so those keep the separate pass.
-constexpr int FUSE_X_MIN_D = 4096;
+// pairs of a row of tiles wait for the slowest of them.  Measured on the step: one r-tile per row (no
+// exchange, 350M list, r = 256): -8 %; long products (7B list, d = 4096, four r-tiles): -6 to -7 %;
+// short products with an exchange (1B list, d = 2048, two r-tiles): -2 % once the X boxes of the
+// second sweep alternate between two buffers (+2 % before).  Shorter products with an exchange have
+// not been measured and keep the separate pass.
+constexpr int FUSE_X_MIN_D = 2048;
 __host__ __device__ inline bool fuse_x_matrix(int d, int r) { return d >= FUSE_X_MIN_D || r <= 256; }
 
 // EPI_PLAIN products may run over up to three k-segments that accumulate into the same tile: segment
@@ -118,7 +125,10 @@ struct ProjCtl {
   uint64_t eready[K1_MVBUFS];   // the epilogue has finished M, V (in place) and N, R of a box
   uint64_t eempty[K1_MVBUFS];   // the stores have read M and V: the buffer is free
   uint64_t nrempty[K1_NRBUFS];  // the stores have read N and R: the buffer is free
-  uint64_t xready[K1_NRBUFS];   // FUSE_X: a row half has finished an X box
+  uint64_t xready[K1_NRBUFS][2];  // FUSE_X: a row half has finished an X box; X boxes alternate between the N
+  uint64_t xempty[K1_NRBUFS][2];  //   and the R part of the half's buffer, each with its own pair of barriers
+  uint64_t xsum[4];             // EG = 2, one per lane quarter: the second group's row sums are in XCH
+  uint64_t xkl[4];              //   the first group has read them (and, FUSE_X, left k_l there)
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -150,8 +160,8 @@ enum { EPI_ADAM = 0, EPI_PLAIN = 1 };
 // carried through unchanged).
 enum { PSI_ADAM = 0, PSI_RMSPROP = 1, PSI_ADAGRAD = 2 };
 
-template <int EPI, int PSI, int FUSE_X>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(K1_THREADS, 1)
+template <int EPI, int PSI, int FUSE_X, int EG = 1>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(k1_threads(EG), 1)
 k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ tdesc, int total_tiles,
              const float* __restrict__ fast, const float* __restrict__ wq_all, const int* __restrict__ wq_off,
              Hyper hp, unsigned* __restrict__ status) {
@@ -160,6 +170,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
   unsigned char* mvbuf = tiles + (size_t)K1_STAGES * K1_STAGE_BYTES;
   unsigned char* nrbuf = mvbuf + (size_t)K1_MVBUFS * K1_MVBUF_BYTES;
   ProjCtl* ctl = reinterpret_cast<ProjCtl*>(nrbuf + (size_t)K1_NRBUFS * K1_NRBUF_BYTES);
+  float4* xch = reinterpret_cast<float4*>(nrbuf + (size_t)K1_NRBUFS * K1_NRBUF_BYTES + 512);   // EG = 2 only
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = ptx::cluster_ctarank();          // 0: issues the MMAs; 1: its partner
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
@@ -174,17 +185,24 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(ptx::smem_u32(&ctl->tmem_full[b]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[b]), 2 * 4);   // every epilogue warp of the pair
+      ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[b]), 2 * 4 * EG);   // every epilogue warp of the pair
     }
     for (int b = 0; b < K1_MVBUFS; ++b) {
       ptx::mbar_init(ptx::smem_u32(&ctl->efull[b][0]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctl->efull[b][1]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl->eready[b]), K1_BOX_THREADS);
+      ptx::mbar_init(ptx::smem_u32(&ctl->eready[b]), K1_BOX_THREADS * EG);
       ptx::mbar_init(ptx::smem_u32(&ctl->eempty[b]), 1);
     }
     for (int b = 0; b < K1_NRBUFS; ++b) {
       ptx::mbar_init(ptx::smem_u32(&ctl->nrempty[b]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl->xready[b]), K1_BOX_THREADS);
+      for (int x = 0; x < 2; ++x) {
+        ptx::mbar_init(ptx::smem_u32(&ctl->xready[b][x]), K1_BOX_THREADS * EG);
+        ptx::mbar_init(ptx::smem_u32(&ctl->xempty[b][x]), 1);
+      }
+    }
+    for (int b = 0; b < 4; ++b) {
+      ptx::mbar_init(ptx::smem_u32(&ctl->xsum[b]), 32);
+      ptx::mbar_init(ptx::smem_u32(&ctl->xkl[b]), 32);
     }
     ctl->abort_flag = smem_ok ? 0 : 1;
     ptx::fence_barrier_init();
@@ -320,7 +338,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         }
       }
     }
-  } else if (warp >= 8) {
+  } else if (warp >= 8 && warp < 8 + K1_GSQ_WARPS) {
     // ------------------------------------------------------------ sums of G^2 over the A stages
     if (EPI == EPI_ADAM && smem_ok) {
       const int w = warp - 8;
@@ -407,7 +425,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     // ------------------------------------------------------------ box storer
     if (lane == 0 && smem_ok) {
       int mv = 0; uint32_t mvphase = 0; bool ok = true;
-      uint32_t xphase = 0;                                // FUSE_X: parities of xready, one bit per row half
+      uint32_t xphase = 0;                                // FUSE_X: parities of xready, one bit per (row half, buffer part)
       ProjTileDesc nd = pair < total_tiles ? load_desc(tdesc, pair) : ProjTileDesc{};
       for (int t = pair; t < total_tiles && ok; t += npairs) {
         const ProjTileDesc d = nd;
@@ -442,17 +460,17 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         if (fuse && ok) {
           // second sweep of the epilogue: the X boxes of this tile, in the same order
           for (int b = 0; b < 2 * (bn / K1_ECOLS); ++b) {
-            const int nr = b & 1;
-            if (!ptx::mbar_wait(ptx::smem_u32(&ctl->xready[nr]), (xphase >> nr) & 1u, abort_flag)) { ok = false; break; }
-            xphase ^= 1u << nr;
+            const int nr = b & 1, xs = (b >> 1) & 1, xbit = 2 * nr + xs;
+            if (!ptx::mbar_wait(ptx::smem_u32(&ctl->xready[nr][xs]), (xphase >> xbit) & 1u, abort_flag)) { ok = false; break; }
+            xphase ^= 1u << xbit;
             const int j = d.r0 + K1_ECOLS * (b >> 1), row = l0 + K1_EROWS * nr;
             if (row < d.L) {
-              const uint32_t srn = nrbuf_u32 + nr * K1_NRBUF_BYTES;
+              const uint32_t srn = nrbuf_u32 + nr * K1_NRBUF_BYTES + xs * K1_HBOX_BYTES;
               ptx::tma_store_2d(&mp->ex, srn, j, row);
               ptx::bulk_commit_group();
               ptx::bulk_wait_group_read<0>();
             }
-            ptx::mbar_arrive(ptx::smem_u32(&ctl->nrempty[nr]));
+            ptx::mbar_arrive(ptx::smem_u32(&ctl->xempty[nr][xs]));
           }
         }
       }
@@ -460,6 +478,11 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     }
   } else if (smem_ok) {
     // ------------------------------------------------------------ epilogue: Adam on R
+    constexpr int GC = K1_ECOLS / EG;                   // columns of a box that one group works on
+    constexpr int QN = 4 / EG;                          //   in units of 8
+    const int grp = (EG == 2 && warp >= 8) ? 1 : 0;     // group 1: warps 16-19
+    const int q0 = QN * grp;
+    uint32_t xphase = 0;                                // EG = 2: parity of xsum / xkl (one use per tile)
     const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31
     const int row = quarter * 32 + lane;                // row of this CTA's half tile = TMEM lane
     const int half = quarter >> 1;                      // boxes with b % 2 == half are this warp's
@@ -475,6 +498,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
     // (buffer, half) barrier is used by every third of them.
     int mv = half; int mvuse = 0; uint32_t mvphase = 0;
     uint32_t nrphase = 0;                               // parity of this half's N/R buffer use
+    uint32_t xeph = 0;                                  // FUSE_X: parities of this half's two X buffer parts
     const uint32_t nrempty = ptx::smem_u32(&ctl->nrempty[half]);
     unsigned char* nb = nrbuf + (size_t)half * K1_NRBUF_BYTES;
     unsigned char* rb = nb + K1_HBOX_BYTES;
@@ -497,9 +521,9 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
       const bool fuse = FUSE_X && (d.bn_left & PROJ_FUSE_X);
       float nn = 0.f, rn = 0.f, rw = 0.f;
       for (int c = 0; c < nch; ++c) {
-        uint32_t rr[32];
+        uint32_t rr[GC];
         __syncwarp();
-        ptx::tmem_ld_32x32b_x32(tcol + K1_ECOLS * c, rr);
+        ptx::TmemCols<GC>::ld(tcol + K1_ECOLS * c + GC * grp, rr);
         // the next chunk's 32 weights (one 128-byte line) on their way into L1 meanwhile
         if (EPI == EPI_ADAM && c + 1 < nch)
           asm volatile("prefetch.global.L1 [%0];" ::"l"(wrow + K1_ECOLS * (c + 1)));
@@ -511,17 +535,24 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         }
         if (EPI == EPI_ADAM && !ptx::mbar_wait(ptx::smem_u32(&ctl->efull[mv][half]), mvphase, abort_flag)) { ok = false; break; }
         if (!fuse && !ptx::mbar_wait(nrempty, nrphase ^ 1u, abort_flag)) { ok = false; break; }
+        if (FUSE_X && !fuse && c == 0) {                 // the X boxes of an earlier tile have left the buffer too
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->xempty[half][0]), (xeph & 1u) ^ 1u, abort_flag) ||
+              !ptx::mbar_wait(ptx::smem_u32(&ctl->xempty[half][1]), ((xeph >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        }
         unsigned char* mb = mvbuf + (size_t)mv * K1_MVBUF_BYTES;
         unsigned char* vb = mb + K1_FBOX_BYTES;
         if (EPI == EPI_PLAIN) {
           // 32 fp32 values of this row: eight 16-byte slots of a 128-byte row, slot ^= row % 8
 #pragma unroll
-          for (int q = 0; q < 8; ++q)
+          for (int qq = 0; qq < 8 / EG; ++qq) {
+            const int q = qq + (8 / EG) * grp;
             *reinterpret_cast<uint4*>(nb + frow + (((uint32_t)q ^ fsw) << 4)) =
-                make_uint4(rr[4 * q], rr[4 * q + 1], rr[4 * q + 2], rr[4 * q + 3]);
+                make_uint4(rr[4 * qq], rr[4 * qq + 1], rr[4 * qq + 2], rr[4 * qq + 3]);
+          }
         } else {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {                    // 8 columns at a time
+        for (int qq = 0; qq < QN; ++qq) {                // 8 columns at a time
+          const int q = q0 + qq;
           const uint32_t f0 = frow + (((uint32_t)(2 * q) ^ fsw) << 4);
           const uint32_t f1 = frow + (((uint32_t)(2 * q + 1) ^ fsw) << 4);
           const float4 m0 = *reinterpret_cast<const float4*>(mb + f0);
@@ -536,7 +567,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
           float rv[8], nv[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
-            rv[e] = __uint_as_float(rr[8 * q + e]);
+            rv[e] = __uint_as_float(rr[8 * qq + e]);
             if (PSI == PSI_ADAM) {
               mo[e] = hp.beta1 * mo[e] + (1.f - hp.beta1) * rv[e];
               vo[e] = hp.beta2 * vo[e] + (1.f - hp.beta2) * rv[e] * rv[e];
@@ -558,7 +589,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
               const __nv_bfloat162 pr = __floats2bfloat162_rn(nv[e], rv[e]);
-              rr[8 * q + e] = *reinterpret_cast<const uint32_t*>(&pr);
+              rr[8 * qq + e] = *reinterpret_cast<const uint32_t*>(&pr);
             }
           } else {
             const uint32_t h = hrow + (((uint32_t)q ^ hsw) << 4);
@@ -568,7 +599,7 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         }
         }
         if (fuse) {
-          ptx::tmem_st_32x32b_x32(tcol + K1_ECOLS * c, rr);
+          ptx::TmemCols<GC>::st(tcol + K1_ECOLS * c + GC * grp, rr);
           ptx::tmem_st_wait();
         }
         // hand the finished boxes to the storer: this thread's writes are visible to
@@ -580,7 +611,18 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         if (mv >= K1_MVBUFS) mv -= K1_MVBUFS;
         if (++mvuse == K1_MVBUFS) { mvuse = 0; mvphase ^= 1u; }
       }
-      if (EPI == EPI_ADAM && ok && l < d.L) {
+      if (EG == 2 && EPI == EPI_ADAM && ok) {
+        // the second group hands its halves of the row sums to the first, which owns the row from here on
+        if (grp == 1) {
+          xch[row] = make_float4(nn, rn, rw, 0.f);
+          ptx::mbar_arrive(ptx::smem_u32(&ctl->xsum[quarter]));
+        } else {
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->xsum[quarter]), xphase, abort_flag)) break;
+          const float4 o = xch[row];
+          nn += o.x; rn += o.y; rw += o.z;
+        }
+      }
+      if (EPI == EPI_ADAM && ok && l < d.L && grp == 0) {
         // colpart[2 part][l] = partial ||N_l||^2, colpart[2 part + 1][l] = partial ||R_l||^2; after the
         // sums of G^2: colpart[(2 + K1_GSQ_SPLIT) nparts + part][l] = partial sum_j w_j R_lj^2
         const int part = d.r0 / bn, nparts = (d.bn_left >> 16) & 0xff;
@@ -588,7 +630,8 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         d.colpart[(long long)(2 * part + 1) * d.L + l] = rn;
         d.colpart[(long long)((2 + K1_GSQ_SPLIT) * nparts + part) * d.L + l] = rw;
       }
-      if (fuse && ok) {
+      float kl = 0.f;
+      if (fuse && ok && grp == 0) {
         // ---- the factor k_l of this thread's row, from the partial sums of every tile of the row of tiles
         const int nparts = (d.bn_left >> 16) & 0xff;
         float nt = 0.f, rt = 0.f;
@@ -614,33 +657,50 @@ k_tc_project(const TcMaps* __restrict__ maps, const ProjTileDesc* __restrict__ t
         } else {
           nt += nn; rt += rn;
         }
-        const float kl = (l < d.L) ? sqrtf(nt) / (sqrtf(rt) + hp.eps) : 0.f;
+        kl = (l < d.L) ? sqrtf(nt) / (sqrtf(rt) + hp.eps) : 0.f;
+      }
+      if (EG == 2 && EPI == EPI_ADAM && ok) {
+        // the first group has read the sums (XCH may be written again) and, FUSE_X, left k_l there
+        if (grp == 0) {
+          if (fuse) reinterpret_cast<float*>(&xch[row])[3] = kl;
+          ptx::mbar_arrive(ptx::smem_u32(&ctl->xkl[quarter]));
+        } else {
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->xkl[quarter]), xphase, abort_flag)) break;
+          if (fuse) kl = reinterpret_cast<const float*>(&xch[row])[3];
+        }
+        xphase ^= 1u;
+      }
+      if (fuse && ok) {
         const float ck = hp.a_res * 1.0f * kl;           // k_tc_form_x's coefficient at lambda = 1
         // ---- sweep 2: X = a_low N - a_res k_l R as bf16 boxes
         for (int c = 0; c < nch; ++c) {
-          uint32_t rr[32];
+          uint32_t rr[GC];
           __syncwarp();
-          ptx::tmem_ld_32x32b_x32(tcol + K1_ECOLS * c, rr);
+          ptx::TmemCols<GC>::ld(tcol + K1_ECOLS * c + GC * grp, rr);
           ptx::tmem_ld_wait();
           if (c == nch - 1) {                            // the accumulator has been read out
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(te);
           }
-          if (!ptx::mbar_wait(nrempty, nrphase ^ 1u, abort_flag)) { ok = false; break; }
+          const int xs = c & 1;                          // X boxes alternate between the two parts of the buffer
+          if (!ptx::mbar_wait(ptx::smem_u32(&ctl->xempty[half][xs]), ((xeph >> xs) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          if (c == 0 && !ptx::mbar_wait(nrempty, nrphase ^ 1u, abort_flag)) { ok = false; break; }   // N, R of an earlier tile
+          unsigned char* xb = nb + xs * K1_HBOX_BYTES;
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
+          for (int qq = 0; qq < QN; ++qq) {
+            const int q = q0 + qq;
             float xv[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-              const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&rr[8 * q + e]));
+              const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&rr[8 * qq + e]));
               xv[e] = hp.a_low * f.x - ck * f.y;
             }
-            *reinterpret_cast<uint4*>(nb + hrow + (((uint32_t)q ^ hsw) << 4)) = pack8_bf16(xv);
+            *reinterpret_cast<uint4*>(xb + hrow + (((uint32_t)q ^ hsw) << 4)) = pack8_bf16(xv);
           }
           ptx::fence_proxy_async_smem();
-          ptx::mbar_arrive(ptx::smem_u32(&ctl->xready[half]));
-          nrphase ^= 1u;
+          ptx::mbar_arrive(ptx::smem_u32(&ctl->xready[half][xs]));
+          xeph ^= 1u << xs;
         }
         if (!ok) break;
       }
