@@ -40,7 +40,10 @@
 //
 // Warp roles: 0 operand producer (TMA); 1 MMA issuer (even CTA only) and TMEM owner;
 // 2 epilogue loader (TMA); 3-6 epilogue; 7 one thread that stores the finished boxes;
-// 8-15 sums of G^2.
+// 8-15 sums of G^2; EG = 2: 16-19 a second group of epilogue warps.  A TMEM lane quarter belongs to
+// the warps w with w % 4 equal to it, so the second group splits the columns, not the rows: both
+// groups work on every box, each on 16 of its 32 columns, and the box barriers count both.  Lists
+// whose products are short (r <= 512) are bound by this epilogue and take that instance.
 //
 // FUSE_X (the plain step: column factors, residual kept): the operand X = a_low N - a_res k_l R of the
 // back-projection is formed here, for limiter factor 1, instead of in a pass of its own over N and R.
