@@ -134,49 +134,70 @@ k_tc_prep(const MatDev* __restrict__ mats, const int* __restrict__ list, int fir
 
 // Copies between the caller's G and W and the copies with aligned rows, one block per row of a
 // staged matrix.  dir 0: G -> Gs, W -> Ws; dir 1: Ws -> W.  The caller's rows start on 2-byte
-// boundaries only; the copies' rows on 128-byte ones.  Both directions move 8-byte words on the
+// boundaries only; the copies' rows on 128-byte ones.  Both directions move 16-byte words on the
 // aligned side and assemble them from (or cut them into) two neighbouring aligned words of the other
 // side; a few elements at the ends of a row move one at a time.  No byte outside a row is written,
 // and none outside [first row, last row] of either buffer is read.
 
-// Row of n elements from `src` (any 2-byte alignment) to `dst` (8-byte aligned).
+// Bytes o .. o + 15 of the 32 bytes {a, b} (o even, 0 < o < 16).
+__device__ __forceinline__ uint4 funnel16(const uint4 a, const uint4 b, int o) {
+  const unsigned long long a0 = ((unsigned long long)a.y << 32) | a.x, a1 = ((unsigned long long)a.w << 32) | a.z;
+  const unsigned long long b0 = ((unsigned long long)b.y << 32) | b.x, b1 = ((unsigned long long)b.w << 32) | b.z;
+  unsigned long long lo, hi;
+  if (o < 8) {
+    const int sh = 8 * o;
+    lo = (a0 >> sh) | (a1 << (64 - sh));
+    hi = (a1 >> sh) | (b0 << (64 - sh));
+  } else if (o == 8) {
+    lo = a1; hi = b0;
+  } else {
+    const int sh = 8 * (o - 8);
+    lo = (a1 >> sh) | (b0 << (64 - sh));
+    hi = (b0 >> sh) | (b1 << (64 - sh));
+  }
+  return make_uint4((unsigned)lo, (unsigned)(lo >> 32), (unsigned)hi, (unsigned)(hi >> 32));
+}
+
+// Row of n elements from `src` (any 2-byte alignment) to `dst` (16-byte aligned).
 __device__ __forceinline__ void copy_row_to_aligned(unsigned short* __restrict__ dst,
                                                     const unsigned short* __restrict__ src, int n, bool first_row) {
   const unsigned long long s = reinterpret_cast<unsigned long long>(src);
-  const int o = (int)(s & 7);                                   // bytes past an 8-byte boundary
-  const unsigned long long* sw = reinterpret_cast<const unsigned long long*>(s - o);
-  unsigned long long* dw = reinterpret_cast<unsigned long long*>(dst);
+  const int o = (int)(s & 15);                                  // bytes past a 16-byte boundary
+  const uint4* sw = reinterpret_cast<const uint4*>(s - o);
+  uint4* dw = reinterpret_cast<uint4*>(dst);
   // words k < nw read sw[k], sw[k + 1]: bytes up to o + 2 n of the row; word 0 reaches o bytes back
-  int nw = (o + 2 * n) / 8 - 1;
+  int nw = (o + 2 * n) / 16 - 1;
   if (nw < 0 || (o != 0 && first_row)) nw = 0;
   if (o == 0) {
-    nw = n / 4;
+    nw = n / 8;
+#pragma unroll 4
     for (int k = threadIdx.x; k < nw; k += blockDim.x) dw[k] = sw[k];
   } else {
-    const int sh = 8 * o;
-    for (int k = threadIdx.x; k < nw; k += blockDim.x) dw[k] = (sw[k] >> sh) | (sw[k + 1] << (64 - sh));
+#pragma unroll 4
+    for (int k = threadIdx.x; k < nw; k += blockDim.x) dw[k] = funnel16(sw[k], sw[k + 1], o);
   }
-  for (int jj = 4 * nw + threadIdx.x; jj < n; jj += blockDim.x) dst[jj] = src[jj];
+  for (int jj = 8 * nw + threadIdx.x; jj < n; jj += blockDim.x) dst[jj] = src[jj];
 }
 
-// Row of n elements from `src` (8-byte aligned, readable up to `pitch` elements) to `dst` (any alignment).
+// Row of n elements from `src` (16-byte aligned, readable up to `pitch` elements) to `dst` (any alignment).
 __device__ __forceinline__ void copy_row_from_aligned(unsigned short* __restrict__ dst,
                                                       const unsigned short* __restrict__ src, int n, int pitch) {
   const unsigned long long d = reinterpret_cast<unsigned long long>(dst);
-  const int head = (int)(((8 - (d & 7)) & 7) / 2);              // elements before dst's first 8-byte boundary
+  const int head = (int)(((16 - (d & 15)) & 15) / 2);           // elements before dst's first 16-byte boundary
   if (head >= n) { for (int jj = threadIdx.x; jj < n; jj += blockDim.x) dst[jj] = src[jj]; return; }
-  unsigned long long* dw = reinterpret_cast<unsigned long long*>(dst + head);
-  const unsigned long long* sw = reinterpret_cast<const unsigned long long*>(src);
-  int nw = (n - head) / 4;                                      // whole aligned words of dst
+  uint4* dw = reinterpret_cast<uint4*>(dst + head);
+  const uint4* sw = reinterpret_cast<const uint4*>(src);
+  int nw = (n - head) / 8;                                      // whole aligned words of dst
   if (head == 0) {
+#pragma unroll 4
     for (int k = threadIdx.x; k < nw; k += blockDim.x) dw[k] = sw[k];
   } else {
-    nw = min(nw, pitch / 4 - 1);                                // word k reads sw[k] and sw[k + 1]
-    const int sh = 16 * head;
-    for (int k = threadIdx.x; k < nw; k += blockDim.x) dw[k] = (sw[k] >> sh) | (sw[k + 1] << (64 - sh));
+    nw = min(nw, pitch / 8 - 1);                                // word k reads sw[k] and sw[k + 1]
+#pragma unroll 4
+    for (int k = threadIdx.x; k < nw; k += blockDim.x) dw[k] = funnel16(sw[k], sw[k + 1], 2 * head);
   }
   for (int jj = threadIdx.x; jj < head; jj += blockDim.x) dst[jj] = src[jj];
-  for (int jj = head + 4 * nw + threadIdx.x; jj < n; jj += blockDim.x) dst[jj] = src[jj];
+  for (int jj = head + 8 * nw + threadIdx.x; jj < n; jj += blockDim.x) dst[jj] = src[jj];
 }
 
 __global__ void __launch_bounds__(256)
